@@ -1,0 +1,220 @@
+"""Seeded synthetic inputs for the batched AED decoder workloads.
+
+This module only draws random numbers and shapes them: model hyper-parameters,
+weight tensors, per-utterance encoder lengths, forced output lengths and encoder
+states.  It contains none of the decoder's arithmetic, so that the CUDA path and
+the CPU checker can both be fed from it without sharing any of the method.
+
+The paper trains and evaluates on 0.5-40 s utterances (Section "Experimental
+setup", length envelope) and reports RTFx as audio seconds per wall second
+(Table "rtfx" caption).  Its data and weights are not available, so the draws
+below stand in for them: log-normal or uniform durations clipped to [1, 40] s,
+80 ms per encoder frame, and a forced transcript length of duration x U(2, 6)
+tokens (far below the paper's 25 tokens/s filter threshold).
+
+Draw order for a workload (fixed, so the same seed always gives the same data):
+durations, token-rate factors, weights (tensor by tensor in ``WEIGHT_ORDER``,
+layer by layer inside each per-layer tensor group), encoder states.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Dict, List, Optional
+
+import numpy as np
+
+FRAME_SECONDS = 0.08          # audio time covered by one encoder frame
+BASE_SEED = 20250305
+
+# (name, per_layer, shape-lambda, kind); kind: "w" weight/bias N(0, 0.02), "g" LN gamma=1, "b" LN beta=0
+_GLOBAL_TENSORS = [
+    ("embed", lambda c: (c["vocab"], c["d_model"]), "w"),
+    ("final_ln_g", lambda c: (c["d_model"],), "g"),
+    ("final_ln_b", lambda c: (c["d_model"],), "b"),
+    ("w_out", lambda c: (c["vocab"], c["d_model"]), "w"),
+]
+_LAYER_TENSORS = [
+    ("ln1_g", lambda c: (c["d_model"],), "g"),
+    ("ln1_b", lambda c: (c["d_model"],), "b"),
+    ("w_qkv", lambda c: (3 * c["d_model"], c["d_model"]), "w"),
+    ("b_qkv", lambda c: (3 * c["d_model"],), "w"),
+    ("w_o", lambda c: (c["d_model"], c["d_model"]), "w"),
+    ("b_o", lambda c: (c["d_model"],), "w"),
+    ("ln2_g", lambda c: (c["d_model"],), "g"),
+    ("ln2_b", lambda c: (c["d_model"],), "b"),
+    ("w_q_c", lambda c: (c["d_model"], c["d_model"]), "w"),
+    ("b_q_c", lambda c: (c["d_model"],), "w"),
+    ("w_kv_c", lambda c: (2 * c["d_model"], c["d_enc"]), "w"),
+    ("b_kv_c", lambda c: (2 * c["d_model"],), "w"),
+    ("w_o_c", lambda c: (c["d_model"], c["d_model"]), "w"),
+    ("b_o_c", lambda c: (c["d_model"],), "w"),
+    ("ln3_g", lambda c: (c["d_model"],), "g"),
+    ("ln3_b", lambda c: (c["d_model"],), "b"),
+    ("w_ff1", lambda c: (c["d_ffn"], c["d_model"]), "w"),
+    ("b_ff1", lambda c: (c["d_ffn"],), "w"),
+    ("w_ff2", lambda c: (c["d_model"], c["d_ffn"]), "w"),
+    ("b_ff2", lambda c: (c["d_model"],), "w"),
+]
+GLOBAL_NAMES = [t[0] for t in _GLOBAL_TENSORS]
+LAYER_NAMES = [t[0] for t in _LAYER_TENSORS]
+WEIGHT_ORDER = GLOBAL_NAMES + LAYER_NAMES
+
+
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest bfloat16 (ties to even); result stays float32."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    u = a.view(np.uint32)
+    rounded = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return rounded.view(np.float32)
+
+
+def bf16_bits(a: np.ndarray) -> np.ndarray:
+    """The uint16 bit patterns of float32 values that are already bf16-representable."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return (a.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+MODELS: Dict[str, Dict[str, int]] = {
+    # 2-layer fp32 parity model
+    "tiny": dict(n_layers=2, d_model=256, n_heads=4, d_ffn=1024, vocab=1024, d_enc=256),
+    # Canary-1B-like 24-layer decoder (16 d^2 = 16.8M weights per layer at d=1024, F=4096)
+    "canary24": dict(n_layers=24, d_model=1024, n_heads=16, d_ffn=4096, vocab=16384, d_enc=1024),
+    # shallow decoder of the "+small decoder" / Flash variants
+    "flash4": dict(n_layers=4, d_model=1024, n_heads=16, d_ffn=4096, vocab=16384, d_enc=1024),
+}
+
+# name -> (model, dtype, batch, duration law)
+CONFIGS = {
+    "cfg1": dict(model="tiny", dtype="fp32", batch=4, lengths="tiny"),
+    "cfg2": dict(model="canary24", dtype="bf16", batch=64, lengths="lognormal"),
+    "cfg3": dict(model="flash4", dtype="bf16", batch=128, lengths="lognormal"),
+    "cfg4": dict(model="canary24", dtype="bf16", batch=512, lengths="uniform"),
+    "cfg5": dict(model="flash4", dtype="bf16", batch=4096, lengths="lognormal"),
+}
+_CONFIG_INDEX = {"cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}
+
+
+@dataclasses.dataclass
+class Workload:
+    name: str
+    model: Dict[str, int]          # n_layers, d_model, n_heads, d_ffn, vocab, d_enc
+    dtype: str                     # "fp32" or "bf16" (values are bf16-representable float32)
+    seed: int
+    enc_lens: np.ndarray           # int32 [B]
+    dec_lens: np.ndarray           # int32 [B], forced output lengths
+    durations: np.ndarray          # float64 [B], seconds
+    weights: Optional[Dict[str, object]]   # name -> float32 array, or list of arrays per layer
+    enc: Optional[np.ndarray]      # float32 [sum(enc_lens), d_enc], utterances back to back
+    bos_id: int = 1
+    eos_id: int = -1
+    ln_eps: float = 1e-5
+
+    @property
+    def batch(self) -> int:
+        return int(self.enc_lens.shape[0])
+
+    @property
+    def enc_offsets(self) -> np.ndarray:
+        off = np.zeros(self.batch + 1, dtype=np.int64)
+        np.cumsum(self.enc_lens, out=off[1:])
+        return off
+
+    @property
+    def audio_seconds(self) -> float:
+        return float(self.enc_lens.sum()) * FRAME_SECONDS
+
+    def subset(self, rows) -> "Workload":
+        """The same model with only the given utterances (in the given order)."""
+        rows = [int(r) for r in rows]
+        off = self.enc_offsets
+        enc = None
+        if self.enc is not None:
+            enc = np.concatenate([self.enc[off[r]:off[r + 1]] for r in rows], axis=0) if rows else \
+                np.zeros((0, self.model["d_enc"]), np.float32)
+        return dataclasses.replace(self, enc_lens=self.enc_lens[rows].copy(), dec_lens=self.dec_lens[rows].copy(),
+                                   durations=self.durations[rows].copy(), enc=enc)
+
+
+def draw_lengths(rng: np.random.Generator, batch: int, law: str):
+    """Durations (s), encoder lengths (frames) and forced output lengths (tokens)."""
+    if law == "tiny":
+        enc_lens = rng.integers(20, 61, size=batch)
+        dec_lens = rng.integers(8, 33, size=batch)
+        durations = enc_lens * FRAME_SECONDS
+        return durations.astype(np.float64), enc_lens.astype(np.int32), dec_lens.astype(np.int32)
+    if law == "lognormal":
+        # median 8 s; sigma 0.7 in log space is this build's reading (the spread is not given)
+        durations = np.exp(rng.normal(math.log(8.0), 0.7, size=batch))
+    elif law == "uniform":
+        durations = rng.uniform(1.0, 40.0, size=batch)
+    else:
+        raise ValueError(law)
+    durations = np.clip(durations, 1.0, 40.0)
+    rate = rng.uniform(2.0, 6.0, size=batch)
+    enc_lens = np.ceil(durations / FRAME_SECONDS - 1e-9).astype(np.int32)
+    dec_lens = np.maximum(1, np.rint(durations * rate)).astype(np.int32)
+    return durations, enc_lens, dec_lens
+
+
+def draw_weights(rng: np.random.Generator, model: Dict[str, int], dtype: str, bias_std: float = 0.02):
+    """All decoder tensors as float32 (bf16-representable when dtype == 'bf16')."""
+    def one(shape, kind):
+        if kind == "g":
+            return np.ones(shape, np.float32)
+        if kind == "b":
+            return np.zeros(shape, np.float32)
+        std = 0.02 if len(shape) == 2 else bias_std
+        a = rng.standard_normal(size=shape, dtype=np.float32)
+        a *= np.float32(std)
+        return round_to_bf16(a) if dtype == "bf16" else a
+
+    w: Dict[str, object] = {}
+    for name, shape_fn, kind in _GLOBAL_TENSORS:
+        w[name] = one(shape_fn(model), kind)
+    for name, shape_fn, kind in _LAYER_TENSORS:
+        w[name] = [one(shape_fn(model), kind) for _ in range(model["n_layers"])]
+    w["b_out"] = None
+    return w
+
+
+def draw_encoder_states(rng: np.random.Generator, total_frames: int, d_enc: int, dtype: str) -> np.ndarray:
+    enc = rng.standard_normal(size=(int(total_frames), d_enc), dtype=np.float32)
+    return round_to_bf16(enc) if dtype == "bf16" else enc
+
+
+def make_workload(name: str, *, seed: Optional[int] = None, batch: Optional[int] = None,
+                  with_weights: bool = True, with_enc: bool = True,
+                  model_override: Optional[Dict[str, int]] = None,
+                  dtype: Optional[str] = None) -> Workload:
+    """Build one of the named workloads ('cfg1' .. 'cfg5')."""
+    spec = CONFIGS[name]
+    model = dict(MODELS[spec["model"]])
+    if model_override:
+        model.update(model_override)
+    dt = dtype or spec["dtype"]
+    seed = BASE_SEED + _CONFIG_INDEX[name] if seed is None else int(seed)
+    rng = np.random.default_rng(seed)
+    b = int(batch) if batch is not None else spec["batch"]
+    durations, enc_lens, dec_lens = draw_lengths(rng, b, spec["lengths"])
+    weights = draw_weights(rng, model, dt) if with_weights else None
+    enc = draw_encoder_states(rng, int(enc_lens.sum()), model["d_enc"], dt) if with_enc else None
+    return Workload(name=name, model=model, dtype=dt, seed=seed, enc_lens=enc_lens, dec_lens=dec_lens,
+                    durations=durations, weights=weights, enc=enc)
+
+
+def make_custom(model: Dict[str, int], enc_lens, dec_lens, *, dtype: str = "fp32", seed: int = 0,
+                bias_std: float = 0.02, name: str = "custom") -> Workload:
+    """A workload with explicit lengths (edge cases, property tests)."""
+    rng = np.random.default_rng(seed)
+    enc_lens = np.asarray(enc_lens, dtype=np.int32)
+    dec_lens = np.asarray(dec_lens, dtype=np.int32)
+    weights = draw_weights(rng, model, dtype, bias_std=bias_std)
+    enc = draw_encoder_states(rng, int(enc_lens.sum()), model["d_enc"], dtype)
+    return Workload(name=name, model=dict(model), dtype=dtype, seed=seed, enc_lens=enc_lens, dec_lens=dec_lens,
+                    durations=enc_lens.astype(np.float64) * FRAME_SECONDS, weights=weights, enc=enc)
+
+
+def layer_param_count(model: Dict[str, int]) -> int:
+    """Number of parameters (weights, biases, LN) in one decoder layer."""
+    return int(sum(int(np.prod(fn(model))) for _, fn, _ in _LAYER_TENSORS))

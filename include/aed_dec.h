@@ -1,0 +1,175 @@
+/*
+ * aed_dec.h — C ABI of the batched autoregressive decoder for attention
+ * encoder-decoder (AED) speech models on NVIDIA B200 (sm_100a).
+ *
+ * The paper (Section "Methods", paragraph "Transferring model capacity from
+ * decoder to encoder"; abstract) identifies the autoregressive cross-attention
+ * Transformer decoder as the inference bottleneck of models such as Canary-1B
+ * and measures the effect of its depth (24 vs 4 layers, Table "rtfx").  This
+ * library runs exactly that part: greedy decoding steps of a pre-LN Transformer
+ * decoder for a batch of utterances with ragged encoder lengths (the paper's
+ * two padding axes, Section "Introduction" and Figure "efficiency_cubes", are
+ * both handled without padding: encoder frames are packed, and finished
+ * utterances are compacted away on the device).
+ *
+ * One decoding step, per active utterance u with t_u tokens already consumed:
+ *   x  = E[token] * sqrt(d) + PE(t_u)                      (sinusoidal positions)
+ *   per layer:  x += Wo  . selfattn (LN1(x))   over the t_u+1 cached positions
+ *               x += Woc . crossattn(LN2(x))   over the T_u encoder frames of u
+ *               x += W2 . relu(W1 . LN3(x) + b1) + b2
+ *   logits = LNf(x) . Wout^T (+ bout);   next = lowest index of the maximum
+ *
+ * General rules
+ *   - Every pointer marked DEVICE is device memory owned by the caller and must
+ *     stay valid while the handle uses it; HOST pointers are read during the
+ *     call only.  The library allocates no device memory: all of its device
+ *     state lives in the caller's workspace.
+ *   - All work is enqueued on the stream given at creation.  Calls return once
+ *     the work is enqueued, except aed_dec_greedy_decode, which synchronises
+ *     the stream once before returning its status.
+ *   - Utterances are addressed by their index in the batch given to
+ *     aed_dec_precompute_cross_kv; compaction of finished rows is internal.
+ *   - No call throws or aborts; every failure is a negative aed_status_t and
+ *     leaves the decode state unchanged.  aed_dec_last_error gives the text.
+ *   - Matrices are row-major [out_features, in_features].  With dtype
+ *     AED_DTYPE_F32 every tensor (weights, biases, LayerNorm parameters,
+ *     embedding, encoder states, K/V caches) is fp32 and all arithmetic is fp32
+ *     FMA.  With AED_DTYPE_BF16 every tensor is bf16; accumulation, LayerNorm
+ *     statistics, softmax and the residual stream stay fp32.
+ */
+#ifndef AED_DEC_H_
+#define AED_DEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct aed_dec aed_dec_t; /* opaque handle; host memory owned by the library */
+
+typedef enum {
+    AED_OK = 0,
+    AED_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, length 0, d_model not divisible by heads ... */
+    AED_ERR_CAPACITY = -2,    /* batch, frame count or step count beyond what the handle was created for */
+    AED_ERR_STATE = -3,       /* call out of order, e.g. a step before any precompute */
+    AED_ERR_CUDA = -4,        /* a CUDA runtime call or launch failed */
+    AED_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired */
+    AED_ERR_UNSUPPORTED = -6  /* shape outside what the kernels support (see aed_dec_create) */
+} aed_status_t;
+
+enum { AED_DTYPE_F32 = 0, AED_DTYPE_BF16 = 1 };
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, d_ffn, vocab, d_enc;
+    int32_t dtype;                /* AED_DTYPE_F32 or AED_DTYPE_BF16 */
+    int32_t max_batch;            /* most utterances in one batch */
+    int32_t max_total_enc_frames; /* most encoder frames in one batch, summed over utterances */
+    int32_t max_enc_len;          /* most encoder frames of one utterance */
+    int32_t max_dec_len;          /* most decoding steps of one utterance */
+    int32_t bos_id;               /* start token of aed_dec_greedy_decode */
+    int32_t eos_id;               /* < 0: no end-of-sequence stopping */
+    float ln_eps;                 /* LayerNorm epsilon (biased variance) */
+    void *workspace;              /* DEVICE, 256-byte aligned, at least aed_dec_workspace_bytes() */
+    size_t workspace_bytes;
+    void *stream;                 /* cudaStream_t of the caller (NULL = default stream) */
+} aed_dec_config_t;
+
+/* All members are DEVICE pointers to tensors of the configured dtype.  The per-layer members are HOST arrays
+ * of n_layers DEVICE pointers (the arrays are copied at creation, the tensors are borrowed).  A NULL bias
+ * pointer (or a NULL per-layer bias array) means "no bias".
+ * w_qkv rows: d query rows, then d key rows, then d value rows.  w_kv_c rows: d key rows, then d value rows. */
+typedef struct {
+    const void *embed;      /* [vocab, d_model] */
+    const void *final_ln_g; /* [d_model] */
+    const void *final_ln_b; /* [d_model] */
+    const void *w_out;      /* [vocab, d_model] */
+    const void *b_out;      /* [vocab] or NULL */
+    const void *const *ln1_g, *const *ln1_b;   /* [d_model] */
+    const void *const *w_qkv, *const *b_qkv;   /* [3 d_model, d_model], [3 d_model] */
+    const void *const *w_o, *const *b_o;       /* [d_model, d_model], [d_model] */
+    const void *const *ln2_g, *const *ln2_b;   /* [d_model] */
+    const void *const *w_q_c, *const *b_q_c;   /* [d_model, d_model], [d_model] */
+    const void *const *w_kv_c, *const *b_kv_c; /* [2 d_model, d_enc], [2 d_model] */
+    const void *const *w_o_c, *const *b_o_c;   /* [d_model, d_model], [d_model] */
+    const void *const *ln3_g, *const *ln3_b;   /* [d_model] */
+    const void *const *w_ff1, *const *b_ff1;   /* [d_ffn, d_model], [d_ffn] */
+    const void *const *w_ff2, *const *b_ff2;   /* [d_model, d_ffn], [d_model] */
+} aed_dec_weights_t;
+
+/*
+ * Bytes of device workspace a handle with this configuration needs (the workspace and stream members are
+ * ignored).  Returns 0 if the configuration is invalid or unsupported.
+ */
+size_t aed_dec_workspace_bytes(const aed_dec_config_t *config);
+
+/*
+ * Create a decoder for one model (the decoder definition above; depth and width per the paper's Table
+ * "rtfx" variants are free parameters).  Validates the configuration, carves the caller's workspace into
+ * self-attention K/V caches, the cross-attention K/V store, activation buffers and decode state, and fills
+ * the positional table.  Supported shapes: head_dim = d_model / n_heads == 64; d_model, d_ffn, d_enc
+ * multiples of 64; vocab >= 2.  Otherwise AED_ERR_UNSUPPORTED.  On success *out receives the handle.
+ */
+aed_status_t aed_dec_create(const aed_dec_config_t *config, const aed_dec_weights_t *weights, aed_dec_t **out);
+
+/*
+ * Start a new batch: compute the cross-attention keys and values of every layer,
+ *   Kc = X Wkc^T + bkc,  Vc = X Wvc^T + bvc,
+ * once for all packed encoder frames (they depend only on the encoder output, which the paper's decoder
+ * attends to at every step), and reset the decode state (t_u = 0, every utterance active).
+ *   enc_packed  DEVICE [sum(enc_lens), d_enc], configured dtype, utterance after utterance, no padding
+ *   enc_lens    HOST   [batch], each in 1..max_enc_len
+ *   batch       1..max_batch
+ */
+aed_status_t aed_dec_precompute_cross_kv(aed_dec_t *dec, const void *enc_packed, const int32_t *enc_lens,
+                                         int32_t batch);
+
+/*
+ * One decoding step (the per-token computation the paper names as the bottleneck) for every utterance that
+ * takes part: consumes tokens_in[u] at position t_u, appends its self-attention key/value to the cache, and
+ * advances t_u by one.
+ *   tokens_in   DEVICE int32 [batch], indexed by utterance; entries of idle utterances are ignored
+ *   active      DEVICE uint8 [batch] or NULL; an utterance takes part if it is not retired and (active == NULL
+ *               or active[u] != 0).  Utterances are retired only by aed_dec_greedy_decode.
+ *   logits_out  DEVICE float [batch, vocab] or NULL; rows of idle utterances are left untouched
+ *   next_out    DEVICE int32 [batch] or NULL; greedy choice (lowest index on ties); idle entries untouched
+ * Errors: AED_ERR_STATE before a precompute; AED_ERR_CAPACITY if a participating utterance already holds
+ * max_dec_len tokens (checked on the host from the steps issued so far, so only reliable when every step uses
+ * active == NULL; with masks the device also refuses to write past the cache and raises a sticky error that
+ * the next aed_dec_greedy_decode or aed_dec_sync_status reports).
+ */
+aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, const uint8_t *active, float *logits_out,
+                          int32_t *next_out);
+
+/*
+ * Greedy decoding of the whole batch from the start token: step, feed each argmax back as the next input,
+ * retire an utterance once it produced max_len[u] tokens (or, when eos_id >= 0, right after it emitted eos_id),
+ * compact the remaining rows on the device, and stop when none is left.  Must directly follow a precompute.
+ *   max_len     HOST   [batch], each in 1..max_dec_len
+ *   tokens_out  DEVICE int32 [batch, max_dec_len]; tokens_out[u][j] is the argmax after consuming j+1 inputs;
+ *               entries at and beyond out_lens[u] are set to -1
+ *   out_lens    DEVICE int32 [batch]
+ * Synchronises the stream before returning.
+ */
+aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max_len, int32_t *tokens_out, int32_t *out_lens);
+
+/* Synchronise the stream and report any sticky device-side error (AED_OK if none). */
+aed_status_t aed_dec_sync_status(aed_dec_t *dec);
+
+/* Number of kernels the handle has launched so far (host-side count, for benchmarks). */
+int64_t aed_dec_launch_count(const aed_dec_t *dec);
+
+/* Free the handle's host state.  NULL is allowed.  Device memory is the caller's and is not touched. */
+void aed_dec_destroy(aed_dec_t *dec);
+
+/* Text of the last error of this handle ("" if none); valid until the next call on the handle. */
+const char *aed_dec_last_error(const aed_dec_t *dec);
+
+/* Text of the last error of a failed aed_dec_create on this thread. */
+const char *aed_dec_create_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AED_DEC_H_ */

@@ -1,0 +1,88 @@
+// Shared device helpers for the AED decoder kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace aed {
+
+constexpr int kHeadDim = 64;        // every supported model has head_dim 64
+constexpr int kAttnChunk = 64;      // positions per flash-decoding work item
+constexpr int kPartialStride = 66;  // floats per attention partial: max, sum, 64 accumulators
+
+// Device-resident decode state (lives in the caller's workspace).
+struct DecState {
+    int32_t n_active;    // rows taking part in the current step
+    int32_t error;       // sticky: 0 ok, 1 = a row would have overflowed the self-attention cache
+    int32_t n_retired;   // utterances retired so far
+    int32_t pad;
+};
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// 8 consecutive elements of type T, starting at a 16-byte (bf16) / 32-byte (fp32) aligned address, as floats.
+__device__ __forceinline__ void load8(const float *p, float (&v)[8])
+{
+    float4 a = *reinterpret_cast<const float4 *>(p);
+    float4 b = *reinterpret_cast<const float4 *>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8])
+{
+    uint4 raw = *reinterpret_cast<const uint4 *>(p);
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+
+// 4 consecutive elements as floats (16-byte aligned for fp32, 8-byte aligned for bf16).
+__device__ __forceinline__ void load4(const float *p, float (&v)[4])
+{
+    float4 a = *reinterpret_cast<const float4 *>(p);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16 *p, float (&v)[4])
+{
+    uint2 raw = *reinterpret_cast<const uint2 *>(p);
+    v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Monotone map float -> uint32 (larger float => larger key), used to take an argmax with integer atomics.
+__device__ __forceinline__ uint32_t float_order_key(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+// (value, index) packed so that the maximum key is the largest value and, among equals, the lowest index.
+__device__ __forceinline__ unsigned long long argmax_key(float f, uint32_t idx)
+{
+    return (static_cast<unsigned long long>(float_order_key(f)) << 32) | (0xFFFFFFFFu - idx);
+}
+__device__ __forceinline__ int32_t argmax_key_index(unsigned long long key)
+{
+    return static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(key & 0xFFFFFFFFull));
+}
+
+}  // namespace aed

@@ -1,0 +1,397 @@
+// Per-step kernels of the AED decoder: row bookkeeping, embedding, LayerNorm, CUDA-core GEMM with fused
+// epilogues (fp32 mode and fallback shapes), flash-decoding attention over ragged caches, argmax finalisation.
+#pragma once
+#include "common.cuh"
+
+namespace aed {
+
+// ------------------------------------------------------------------------------------------------------------
+// Row bookkeeping: stable compaction of the utterances that take part in the next step.
+//   active_list[r] = utterance id of compact row r;  state->n_active = number of rows.
+// An utterance takes part if it is not retired, the caller's mask (if any) selects it, and its self-attention
+// cache still has room; a selected utterance with a full cache raises the sticky error instead of overflowing.
+// ------------------------------------------------------------------------------------------------------------
+__global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask, const int32_t *__restrict__ retired,
+                                    const int32_t *__restrict__ t_u, int max_dec_len,
+                                    int32_t *__restrict__ active_list, DecState *state)
+{
+    __shared__ int warp_counts[32];
+    __shared__ int base;
+    if (threadIdx.x == 0) base = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int start = 0; start < batch; start += blockDim.x) {
+        int u = start + threadIdx.x;
+        bool take = false;
+        if (u < batch) {
+            take = retired[u] == 0 && (mask == nullptr || mask[u] != 0);
+            if (take && t_u[u] >= max_dec_len) { take = false; atomicExch(&state->error, 1); }
+        }
+        unsigned ballot = __ballot_sync(0xffffffffu, take);
+        if (lane == 0) warp_counts[warp] = __popc(ballot);
+        __syncthreads();
+        int before = base;
+        for (int w = 0; w < warp; ++w) before += warp_counts[w];
+        if (take) active_list[before + __popc(ballot & ((1u << lane) - 1u))] = u;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int total = 0;
+            for (int w = 0; w < n_warps; ++w) total += warp_counts[w];
+            base += total;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) state->n_active = base;
+}
+
+// Sinusoidal position table PE[t][2i] = sin(t / 10000^(2i/d)), PE[t][2i+1] = cos(same), evaluated in double.
+__global__ void fill_pe_kernel(float *pe, int max_len, int d)
+{
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= max_len * d) return;
+    int t = idx / d, i = idx % d;
+    double angle = static_cast<double>(t) / pow(10000.0, (2.0 * (i / 2)) / static_cast<double>(d));
+    pe[idx] = static_cast<float>((i & 1) ? cos(angle) : sin(angle));
+}
+
+// x[r] = E[token of utterance] * sqrt(d) + PE[t_u]
+template <typename T>
+__global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ active_list,
+                             const int32_t *__restrict__ tokens, const int32_t *__restrict__ t_u,
+                             const T *__restrict__ embed, const float *__restrict__ pe, int d, int vocab, float scale,
+                             float *__restrict__ x)
+{
+    int r = blockIdx.x;
+    if (r >= state->n_active) return;
+    int u = active_list[r];
+    int tok = tokens[u];
+    tok = min(max(tok, 0), vocab - 1);
+    int t = t_u[u];
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+        x[(size_t)r * d + i] = to_f32(embed[(size_t)tok * d + i]) * scale + pe[(size_t)t * d + i];
+}
+
+// out[r] = g * (x[r] - mean) / sqrt(var + eps) + b, biased variance, two passes over a row held in registers.
+template <typename T, int kMaxPerThread>
+__global__ void layernorm_kernel(const DecState *state, const float *__restrict__ x, const T *__restrict__ g,
+                                 const T *__restrict__ b, int d, float eps, float *__restrict__ out)
+{
+    int r = blockIdx.x;
+    if (r >= state->n_active) return;
+    __shared__ float red[32];
+    __shared__ float stat;
+    float v[kMaxPerThread];
+    const float *xr = x + (size_t)r * d;
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        int i = threadIdx.x + j * blockDim.x;
+        v[j] = (i < d) ? xr[i] : 0.f;
+        s += v[j];
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    s = warp_sum(s);
+    if (lane == 0) red[warp] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) { float tsum = 0.f; for (int w = 0; w < n_warps; ++w) tsum += red[w]; stat = tsum / d; }
+    __syncthreads();
+    float mean = stat;
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        int i = threadIdx.x + j * blockDim.x;
+        float c = (i < d) ? v[j] - mean : 0.f;
+        q += c * c;
+    }
+    q = warp_sum(q);
+    __syncthreads();
+    if (lane == 0) red[warp] = q;
+    __syncthreads();
+    if (threadIdx.x == 0) { float tsum = 0.f; for (int w = 0; w < n_warps; ++w) tsum += red[w]; stat = rsqrtf(tsum / d + eps); }
+    __syncthreads();
+    float rstd = stat;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        int i = threadIdx.x + j * blockDim.x;
+        if (i < d) out[(size_t)r * d + i] = to_f32(g[i]) * (v[j] - mean) * rstd + to_f32(b[i]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// CUDA-core GEMM  out[r, o] = sum_k A[r, k] * W[o, k] + bias[o]  with fused epilogues.
+// 64 rows x 32 output features per block, K in slices of 32 staged through shared memory, 4x4 per thread.
+// ------------------------------------------------------------------------------------------------------------
+enum Epilogue { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_QKV = 3, EPI_LOGITS = 4, EPI_CROSSKV = 5 };
+
+template <typename CT>
+struct GemmEpilogueArgs {
+    float *out;                 // STORE / RELU: [rows, ldo];  RESID: x [rows, ldo];  QKV: q [rows, d]
+    int ldo;
+    // QKV: self-attention cache of this layer [batch][2][H][max_dec_len][64]
+    CT *self_cache;
+    const int32_t *active_list;
+    const int32_t *t_u;
+    int max_dec_len, d_model, n_heads;
+    // LOGITS
+    float *logits_out;          // [batch, vocab] by utterance, or nullptr
+    unsigned long long *keys;   // [rows] packed argmax keys
+    // CROSSKV: store of this layer [2][H][frame_capacity][64]
+    CT *cross_store;
+    int frame_capacity;
+};
+
+template <typename AT, typename WT, typename CT, int EPI>
+__global__ void __launch_bounds__(128)
+gemm_rows_kernel(const DecState *state, int rows_fixed, const AT *__restrict__ A, int lda,
+                 const WT *__restrict__ W, const WT *__restrict__ bias, int M, int K, GemmEpilogueArgs<CT> ep)
+{
+    constexpr int BM = 64, BN = 32, BK = 32;
+    const int n_rows = (rows_fixed >= 0) ? rows_fixed : state->n_active;
+    const int row0 = blockIdx.y * BM, o0 = blockIdx.x * BN;
+    if (row0 >= n_rows) return;
+    __shared__ __align__(16) float As[BK][BM + 4];
+    __shared__ __align__(16) float Ws[BK][BN + 4];
+    const int tid = threadIdx.x, tx = tid & 7, ty = tid >> 3;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        // A tile: 64 rows x 32 k, 4 elements per load
+        for (int idx = tid; idx < BM * BK / 4; idx += 128) {
+            int r = idx / (BK / 4), kq = (idx % (BK / 4)) * 4;
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            if (row0 + r < n_rows) load4(A + (size_t)(row0 + r) * lda + k0 + kq, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) As[kq + j][r] = v[j];
+        }
+        for (int idx = tid; idx < BN * BK / 4; idx += 128) {
+            int o = idx / (BK / 4), kq = (idx % (BK / 4)) * 4;
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            if (o0 + o < M) load4(W + (size_t)(o0 + o) * K + k0 + kq, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) Ws[kq + j][o] = v[j];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            float4 a4 = *reinterpret_cast<const float4 *>(&As[k][ty * 4]);
+            float4 w4 = *reinterpret_cast<const float4 *>(&Ws[k][tx * 4]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w}, w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    // epilogue
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = row0 + ty * 4 + i;
+        const bool row_ok = r < n_rows;
+        float best = -INFINITY;
+        uint32_t best_idx = 0;
+        int u = 0, t = 0;
+        if (row_ok && (EPI == EPI_QKV || EPI == EPI_LOGITS)) u = ep.active_list[r];
+        if (row_ok && EPI == EPI_QKV) t = ep.t_u[u];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int o = o0 + tx * 4 + j;
+            if (!row_ok || o >= M) continue;
+            float v = acc[i][j] + (bias ? to_f32(bias[o]) : 0.f);
+            if (EPI == EPI_STORE) {
+                ep.out[(size_t)r * ep.ldo + o] = v;
+            } else if (EPI == EPI_RELU) {
+                ep.out[(size_t)r * ep.ldo + o] = fmaxf(v, 0.f);
+            } else if (EPI == EPI_RESID) {
+                ep.out[(size_t)r * ep.ldo + o] += v;
+            } else if (EPI == EPI_QKV) {
+                const int d = ep.d_model;
+                if (o < d) {
+                    ep.out[(size_t)r * d + o] = v;
+                } else {
+                    const int kv = (o - d) / d, c = (o - d) % d, h = c / kHeadDim, e = c % kHeadDim;
+                    size_t off = ((((size_t)u * 2 + kv) * ep.n_heads + h) * ep.max_dec_len + t) * kHeadDim + e;
+                    ep.self_cache[off] = from_f32<CT>(v);
+                }
+            } else if (EPI == EPI_LOGITS) {
+                if (ep.logits_out) ep.logits_out[(size_t)u * M + o] = v;
+                if (v > best) { best = v; best_idx = o; }
+            } else if (EPI == EPI_CROSSKV) {
+                const int d = ep.d_model;
+                const int kv = o / d, c = o % d, h = c / kHeadDim, e = c % kHeadDim;
+                size_t off = (((size_t)kv * ep.n_heads + h) * ep.frame_capacity + r) * kHeadDim + e;
+                ep.cross_store[off] = from_f32<CT>(v);
+            }
+        }
+        if (EPI == EPI_LOGITS) {
+            // the 8 threads that share this row sit in consecutive lanes: reduce, then one atomic per block row
+            unsigned long long key = (row_ok && best > -INFINITY) ? argmax_key(best, best_idx) : 0ull;
+#pragma unroll
+            for (int off = 1; off < 8; off <<= 1) {
+                unsigned long long other = __shfl_xor_sync(0xffffffffu, key, off);
+                key = other > key ? other : key;
+            }
+            if (tx == 0 && row_ok && key != 0ull) atomicMax(ep.keys + r, key);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Flash-decoding attention over ragged caches.  One warp per (row, head, chunk of 64 positions): lanes are
+// 4 position groups x 8 dimension groups, each lane holds 8 of the 64 head dimensions (one 128-bit load of a
+// bf16 key or value row segment).  Scores are reduced over the 8 dimension lanes with shuffles, softmax is
+// kept online per position group and merged over the 4 groups at the end.  Each work item writes
+// (running max, running sum, 64 un-normalised accumulators); the combine kernel merges the chunks of a row.
+//   SELF : keys/values of utterance u, head h at  cache[((u*2 + kv)*H + h)*max_len*64],  length t_u + 1
+//   CROSS: keys/values at store[(kv*H + h)*capacity*64 + enc_off[u]*64],                 length enc_len[u]
+// ------------------------------------------------------------------------------------------------------------
+template <typename CT, bool kCross>
+__global__ void __launch_bounds__(128)
+attn_partial_kernel(const DecState *state, const int32_t *__restrict__ active_list, const float *__restrict__ q,
+                    int ldq, const CT *__restrict__ cache, int n_heads, int seq_capacity,
+                    const int32_t *__restrict__ t_u, const int32_t *__restrict__ enc_off,
+                    const int32_t *__restrict__ enc_len, int max_chunks, float scale, float *__restrict__ partials)
+{
+    const int rh = blockIdx.x;
+    const int r = rh / n_heads, h = rh % n_heads;
+    if (r >= state->n_active) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int chunk = blockIdx.y * 4 + warp;
+    const int u = active_list[r];
+    const int len = kCross ? enc_len[u] : t_u[u] + 1;
+    const int p0 = chunk * kAttnChunk;
+    if (chunk >= max_chunks || p0 >= len) return;
+    const int p1 = min(len, p0 + kAttnChunk);
+    const CT *kbase, *vbase;
+    if (kCross) {
+        kbase = cache + ((size_t)(0 * n_heads + h) * seq_capacity + enc_off[u]) * kHeadDim;
+        vbase = cache + ((size_t)(1 * n_heads + h) * seq_capacity + enc_off[u]) * kHeadDim;
+    } else {
+        kbase = cache + (((size_t)u * 2 + 0) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
+        vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
+    }
+    const int dg = lane & 7, pg = lane >> 3;
+    float qv[8];
+    load8(q + (size_t)r * ldq + h * kHeadDim + dg * 8, qv);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qv[i] *= scale;
+
+    float m = -INFINITY, l = 0.f, acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int p = p0 + pg; p < p0 + kAttnChunk; p += 4) {   // uniform trip count: shuffles need all lanes
+        const bool ok = p < p1;
+        float kv[8], s = 0.f;
+        if (ok) {
+            load8(kbase + (size_t)p * kHeadDim + dg * 8, kv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) s = fmaf(qv[i], kv[i], s);
+        }
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        if (ok) {
+            float vv[8];
+            load8(vbase + (size_t)p * kHeadDim + dg * 8, vv);
+            float m_new = fmaxf(m, s);
+            float corr = expf(m - m_new), pr = expf(s - m_new);
+            l = l * corr + pr;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = fmaf(pr, vv[i], acc[i] * corr);
+            m = m_new;
+        }
+    }
+    // merge the 4 position groups (lanes differing in bits 3 and 4)
+#pragma unroll
+    for (int off = 8; off < 32; off <<= 1) {
+        float m_o = __shfl_xor_sync(0xffffffffu, m, off);
+        float l_o = __shfl_xor_sync(0xffffffffu, l, off);
+        float m_new = fmaxf(m, m_o);
+        float c_self = (m == -INFINITY) ? 0.f : expf(m - m_new);
+        float c_oth = (m_o == -INFINITY) ? 0.f : expf(m_o - m_new);
+        l = l * c_self + l_o * c_oth;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float a_o = __shfl_xor_sync(0xffffffffu, acc[i], off);
+            acc[i] = acc[i] * c_self + a_o * c_oth;
+        }
+        m = m_new;
+    }
+    float *dst = partials + ((size_t)rh * max_chunks + chunk) * kPartialStride;
+    if (lane == 0) { dst[0] = m; dst[1] = l; }
+    if (pg == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dst[2 + dg * 8 + i] = acc[i];
+    }
+}
+
+// Merge the chunk partials of each (row, head): one warp per pair, 2 head dimensions per lane.
+template <bool kCross>
+__global__ void __launch_bounds__(128)
+attn_combine_kernel(const DecState *state, const int32_t *__restrict__ active_list, const float *__restrict__ partials,
+                    int n_heads, const int32_t *__restrict__ t_u, const int32_t *__restrict__ enc_len, int max_chunks,
+                    float *__restrict__ out, int ldo)
+{
+    const int rh = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int r = rh / n_heads, h = rh % n_heads;
+    if (r >= state->n_active) return;
+    const int u = active_list[r];
+    const int len = kCross ? enc_len[u] : t_u[u] + 1;
+    const int n_chunks = (len + kAttnChunk - 1) / kAttnChunk;
+    const float *src = partials + (size_t)rh * max_chunks * kPartialStride;
+    float m = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, src[(size_t)c * kPartialStride]);
+    float l = 0.f, a0 = 0.f, a1 = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+        const float *p = src + (size_t)c * kPartialStride;
+        float w = expf(p[0] - m);
+        l = fmaf(p[1], w, l);
+        a0 = fmaf(p[2 + lane * 2], w, a0);
+        a1 = fmaf(p[3 + lane * 2], w, a1);
+    }
+    float inv = 1.f / l;
+    float2 o = make_float2(a0 * inv, a1 * inv);
+    *reinterpret_cast<float2 *>(out + (size_t)r * ldo + h * kHeadDim + lane * 2) = o;
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// End of a step: decode the argmax keys, hand the choice out by utterance id, advance t_u, and (greedy mode)
+// record the token, feed it back and retire finished utterances.
+// ------------------------------------------------------------------------------------------------------------
+__global__ void finish_step_kernel(DecState *state, const int32_t *__restrict__ active_list,
+                                   unsigned long long *__restrict__ keys, int32_t *__restrict__ t_u,
+                                   int32_t *__restrict__ next_out /* by utterance, nullable */,
+                                   int greedy, int32_t *__restrict__ cur_tok, int32_t *__restrict__ retired,
+                                   const int32_t *__restrict__ max_len, int eos_id,
+                                   int32_t *__restrict__ tokens_out, int tokens_ld, int32_t *__restrict__ out_lens)
+{
+    int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= state->n_active) return;
+    int u = active_list[r];
+    int32_t tok = argmax_key_index(keys[r]);
+    keys[r] = 0ull;
+    int t = t_u[u];
+    t_u[u] = t + 1;
+    if (next_out) next_out[u] = tok;
+    if (greedy) {
+        cur_tok[u] = tok;
+        tokens_out[(size_t)u * tokens_ld + t] = tok;
+        if (t + 1 >= max_len[u] || (eos_id >= 0 && tok == eos_id)) {
+            retired[u] = 1;
+            out_lens[u] = t + 1;
+        }
+    }
+}
+
+__global__ void fill_i32_kernel(int32_t *p, int32_t v, size_t n)
+{
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+
+}  // namespace aed

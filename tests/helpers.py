@@ -1,0 +1,76 @@
+"""Shared helpers of the GPU parity tests: drive the C ABI and compare with the CPU checker."""
+import numpy as np
+
+from oracle import aed_oracle as orc
+
+TOL = {"fp32": 1e-4, "bf16": 3e-2}       # max-abs tolerance on teacher-forced logits
+MARGIN = 0.1                             # greedy ids must match where the checker's top-2 margin exceeds this
+
+
+def oracle_reference(w, rows=None, want_logits=True, n_threads=0):
+    """Free-running greedy decode of the given utterances (default: all) by the CPU checker."""
+    sub = w if rows is None else w.subset(rows)
+    model = orc.Model(w.model, w.weights, ln_eps=w.ln_eps)
+    return orc.decode_batch(model, sub.enc, sub.enc_lens, sub.dec_lens, bos=w.bos_id, want_logits=want_logits,
+                            n_threads=n_threads)
+
+
+def teacher_forced_compare(dec, w, ref, rows=None, check_rows_only=True):
+    """Feed the checker's greedy tokens to aed_dec_step and compare logits and argmax at every step.
+
+    ``ref`` covers the utterances ``rows`` (default all); the other utterances of the batch run on their own
+    previous argmax.  Returns (max |logit diff|, number of compared argmax, mismatches with margin > MARGIN)."""
+    import torch
+    B, V = w.batch, w.model["vocab"]
+    rows = list(range(B)) if rows is None else [int(r) for r in rows]
+    Lmax = int(w.dec_lens.max())
+    enc = dec.upload_encoder(w.enc)
+    dec.precompute_cross_kv(enc, w.enc_lens)
+    logits = torch.full((B, V), float("nan"), dtype=torch.float32, device=dec.device)
+    nxt = torch.full((B,), w.bos_id, dtype=torch.int32, device=dec.device)
+    toks = torch.full((B,), w.bos_id, dtype=torch.int32, device=dec.device)
+    worst, compared, bad = 0.0, 0, []
+    ridx = torch.tensor(rows, dtype=torch.long, device=dec.device)
+    for t in range(Lmax):
+        act = torch.from_numpy((w.dec_lens > t).astype(np.uint8)).to(dec.device)
+        if t > 0:
+            toks.copy_(nxt)
+            forced = np.array([max(int(ref["next"][i, min(t, int(w.dec_lens[u])) - 1]), 0) for i, u in enumerate(rows)],
+                              np.int32)
+            toks[ridx] = torch.from_numpy(forced).to(dec.device)
+        dec.step(toks, act, logits, nxt)
+        got = logits[ridx].cpu().numpy()
+        got_next = nxt[ridx].cpu().numpy()
+        for i, u in enumerate(rows):
+            if t >= int(w.dec_lens[u]):
+                continue
+            diff = float(np.max(np.abs(got[i].astype(np.float64) - ref["logits"][i][t])))
+            worst = max(worst, diff)
+            compared += 1
+            if ref["margin"][i, t] > MARGIN and got_next[i] != ref["next"][i, t]:
+                bad.append((u, t, int(got_next[i]), int(ref["next"][i, t])))
+    dec.sync_status()
+    return worst, compared, bad
+
+
+def greedy_compare(dec, w, ref, rows=None):
+    """aed_dec_greedy_decode against the checker: per utterance, tokens must agree up to and including the
+    last step before the checker's first near-tie (margin <= MARGIN).  Returns the number of compared tokens."""
+    rows = list(range(w.batch)) if rows is None else [int(r) for r in rows]
+    enc = dec.upload_encoder(w.enc)
+    dec.precompute_cross_kv(enc, w.enc_lens)
+    toks, lens = dec.greedy_decode(w.dec_lens)
+    toks, lens = toks.cpu().numpy(), lens.cpu().numpy()
+    assert np.array_equal(lens, w.dec_lens)
+    compared = 0
+    for u in range(w.batch):
+        L = int(w.dec_lens[u])
+        assert np.all(toks[u, :L] >= 0) and np.all(toks[u, :L] < w.model["vocab"])
+        assert np.all(toks[u, L:] == -1)
+    for i, u in enumerate(rows):
+        for t in range(int(w.dec_lens[u])):
+            if ref["margin"][i, t] <= MARGIN:
+                break
+            assert toks[u, t] == ref["next"][i, t], f"utterance {u} step {t}: {toks[u, t]} vs {ref['next'][i, t]}"
+            compared += 1
+    return compared, toks

@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the batched AED decoder: output tokens/s and RTFx on synthetic Canary-style workloads.
+
+    python bench.py --gpus 1 --steps 5 --warmup 3                 # this library
+    python bench.py --impl reference --steps 2 --warmup 1         # the CPU checker, as a baseline
+
+One "step" is one pass of the whole hot path over one batch: cross-K/V precompute followed by greedy
+decoding of every utterance to its forced length.  Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_05931_b200 import workloads as wl   # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+def step_bytes_and_flops(w):
+    """Algorithmic bytes and flops of greedy decoding, step by step (weights once per step, each active row's
+    own self and cross K/V once per layer), and of the cross-K/V precompute."""
+    m = w.model
+    e = 2 if w.dtype == "bf16" else 4
+    NL, d, F, V, de = m["n_layers"], m["d_model"], m["d_ffn"], m["vocab"], m["d_enc"]
+    step_params = NL * (4 * d * d + 2 * d * d + 2 * d * F) + V * d
+    T, L = w.enc_lens.astype(np.int64), w.dec_lens.astype(np.int64)
+    per_step = []
+    for s in range(int(L.max())):
+        act = L > s
+        n = int(act.sum())
+        kv_pos = int((T[act] + s + 1).sum())
+        per_step.append((e * step_params + e * NL * 2 * d * kv_pos, 2 * n * step_params + 4 * d * NL * kv_pos, n))
+    total_T = int(T.sum())
+    pre_flops = 2 * total_T * de * NL * 2 * d
+    pre_bytes = e * (total_T * de + NL * 2 * d * de + total_T * NL * 2 * d)
+    return per_step, pre_bytes, pre_flops, step_params
+
+
+def family_bytes(family, w):
+    """Algorithmic bytes one whole pass (precompute + greedy decode) moves in the launches of a kernel family."""
+    m = w.model
+    e = 2 if w.dtype == "bf16" else 4
+    NL, d, F, V, de = m["n_layers"], m["d_model"], m["d_ffn"], m["vocab"], m["d_enc"]
+    T, L = w.enc_lens.astype(np.int64), w.dec_lens.astype(np.int64)
+    steps = int(L.max())
+    per_layer_weights = {"gemm_qkv": 3 * d * d, "gemm_o": d * d, "gemm_qc": d * d, "gemm_oc": d * d,
+                         "gemm_ff1": d * F, "gemm_ff2": d * F, "ffn": 2 * d * F}
+    if family in per_layer_weights:
+        return e * per_layer_weights[family] * NL * steps
+    if family == "gemm_vocab":
+        return e * V * d * steps
+    if family == "attn_cross":
+        return sum(e * NL * 2 * d * int(T[L > s].sum()) for s in range(steps))
+    if family == "attn_self":
+        return sum(e * NL * 2 * d * int((L > s).sum()) * (s + 1) for s in range(steps))
+    if family == "precompute_cross_kv":
+        total_T = int(T.sum())
+        return e * (total_T * de + NL * 2 * d * de + total_T * NL * 2 * d)
+    return None
+
+
+def roofline_seconds(w, peaks):
+    per_step, pre_bytes, pre_flops, _ = step_bytes_and_flops(w)
+    bw, fl = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    dec = sum(max(b / bw, f / fl) for b, f, _ in per_step)
+    pre = max(pre_bytes / bw, pre_flops / fl)
+    return dec, pre
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.file:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def run_reference(args):
+    """The CPU checker, as it stands (fp32 build, OpenMP over utterances), on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import aed_oracle as orc
+    w = wl.make_workload(args.workload)
+    cores = os.cpu_count() or 1
+    rng = np.random.default_rng(1)
+    short = np.flatnonzero(w.dec_lens <= 24)
+    rows = sorted(int(r) for r in rng.choice(short, size=min(len(short), max(2, cores // 2)), replace=False))
+    sub = w.subset(rows)
+    model = orc.Model(w.model, w.weights, ln_eps=w.ln_eps)
+    n_tok = int(sub.dec_lens.sum())
+    times, threads = [], 1
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        out = orc.decode_batch(model, sub.enc, sub.enc_lens, sub.dec_lens, bos=w.bos_id, precision="f32")
+        dt = time.perf_counter() - t0
+        threads = out["threads"]
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = n_tok * len(times) / total
+    sample = f"{len(rows)} utterances of {w.name} with at most 24 output tokens ({n_tok} tokens, {int(sub.enc_lens.sum())} frames) per step"
+    line = {
+        "impl": "reference", "metric": "decoder output tokens/s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, **w.model, "batch": w.batch, "weights": w.dtype, "sample": sample},
+        "rtfx": float(sub.enc_lens.sum()) * wl.FRAME_SECONDS * len(times) / total,
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(w, budget_tokens: int = 0):
+    """Time the CPU checker (fp32 build) on a bounded sample of the same workload."""
+    from oracle import aed_oracle as orc
+    cores = os.cpu_count() or 1
+    rng = np.random.default_rng(2)
+    rows = sorted(int(r) for r in rng.choice(w.batch, size=min(w.batch, cores), replace=False))
+    sub = w.subset(rows)
+    model = orc.Model(w.model, w.weights, ln_eps=w.ln_eps)
+    t0 = time.perf_counter()
+    out = orc.decode_batch(model, sub.enc, sub.enc_lens, sub.dec_lens, bos=w.bos_id, precision="f32")
+    dt = time.perf_counter() - t0
+    n_tok = int(sub.dec_lens.sum())
+    return {"value": n_tok / dt, "unit": "tokens/s", "cores": int(out["threads"]), "kind": "oracle",
+            "sample": f"{len(rows)} randomly chosen utterances of {w.name} ({n_tok} tokens, {int(sub.enc_lens.sum())} "
+                      f"encoder frames), precompute + greedy decode, fp32 build, {dt:.1f} s",
+            "rtfx": float(sub.enc_lens.sum()) * wl.FRAME_SECONDS / dt}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=list(wl.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-profile", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2503_05931_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+
+    # Every rank decodes its own batch of the same distribution (utterances are independent: no collective
+    # on the data path, weak scaling).
+    w = wl.make_workload(args.workload, seed=wl.BASE_SEED + wl._CONFIG_INDEX[args.workload] + 1000 * rank)
+    peaks = load_peaks()
+    dec = binding.decoder_for_workload(w, device=device)
+    enc_host = torch.from_numpy(w.enc).to(dec.tdtype).pin_memory()
+    enc_dev = enc_host.to(device)
+    B, Lmax = w.batch, int(w.dec_lens.max())
+    toks_dev = torch.empty((B, Lmax), dtype=torch.int32, device=device)
+    lens_dev = torch.empty(B, dtype=torch.int32, device=device)
+    toks_host = torch.empty((B, Lmax), dtype=torch.int32).pin_memory()
+    lens_host = torch.empty(B, dtype=torch.int32).pin_memory()
+    n_tok = int(w.dec_lens.sum())
+
+    def one_pass(from_host: bool):
+        src = enc_dev
+        if from_host:
+            src = enc_host.to(device, non_blocking=True)
+        dec.precompute_cross_kv(src, w.enc_lens)
+        dec.greedy_decode(w.dec_lens, toks_dev, lens_dev)
+        if from_host:
+            toks_host.copy_(toks_dev, non_blocking=True)
+            lens_host.copy_(lens_dev, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(from_host: bool, steps: int):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        ev[0].record()
+        for i in range(steps):
+            one_pass(from_host)
+            ev[i + 1].record()
+        barrier()
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        total_ms = ev[0].elapsed_time(ev[steps])
+        if world > 1:
+            t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        return total_ms, per
+
+    for _ in range(max(args.warmup, 3)):
+        one_pass(False)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = dec.launch_count()
+    total_ms, per = timed(False, args.steps)
+    launches = dec.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    one_pass(True)
+    e2e_ms, _ = timed(True, args.steps)
+    dec.sync_status()
+
+    tok_all = torch.tensor([n_tok, int(w.enc_lens.sum())], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(tok_all)
+    total_tokens, total_frames = float(tok_all[0].item()), float(tok_all[1].item())
+    value = total_tokens * args.steps / (total_ms * 1e-3)
+    e2e_value = total_tokens * args.steps / (e2e_ms * 1e-3)
+    rtfx = total_frames * wl.FRAME_SECONDS * args.steps / (total_ms * 1e-3)
+
+    if rank == 0:
+        dec_s, pre_s = roofline_seconds(w, peaks)
+        ms_per_step = total_ms / args.steps
+        h2d = int(enc_host.numel() * enc_host.element_size())
+        d2h = int(toks_host.numel() * 4 + lens_host.numel() * 4)
+        line = {
+            "metric": "decoder output tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, **w.model, "batch_per_gpu": w.batch, "total_enc_frames": int(w.enc_lens.sum()),
+                       "total_out_tokens": n_tok, "decode_steps": Lmax,
+                       "l2": "inputs larger than L2 (weights + K/V stores stream every decode step)",
+                       "step": "cross-K/V precompute + greedy decode of one batch"},
+            "rtfx": rtfx,
+            "step_roofline": {"roofline_ms": 1e3 * (dec_s + pre_s), "frac": 1e3 * (dec_s + pre_s) / ms_per_step,
+                              "peaks": peaks["source"], "hbm_gbs": peaks["hbm_gbs"],
+                              "bf16_tflops": peaks["bf16_tflops_sustained"]},
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if not args.no_profile:
+            line["roofline"] = profile_dominant_kernel(dec, w, one_pass, peaks)
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line), flush=True)
+    dec.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def profile_dominant_kernel(dec, w, one_pass, peaks):
+    """Per-kernel device time of one more pass, taken with CUDA events around every launch on the library's
+    stream, and the roofline figure of the kernel family that takes the largest share."""
+    prof = dec.profile_pass(one_pass)
+    if not prof:
+        return None
+    top = max(prof, key=lambda k: prof[k]["ms"])
+    info = prof[top]
+    bytes_total = family_bytes(top, w)
+    achieved = bytes_total / (info["ms"] * 1e-3) / 1e9 if bytes_total else None
+    return {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": None,
+            "launches": info["launches"], "avg_us": 1e3 * info["ms"] / max(info["launches"], 1),
+            "peak_source": peaks["source"],
+            "shares": {k: round(v["ms"] / sum(x["ms"] for x in prof.values()), 4) for k, v in prof.items()}}
+
+
+if __name__ == "__main__":
+    main()

@@ -157,6 +157,18 @@ aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max_len, int32
 /* Synchronise the stream and report any sticky device-side error (AED_OK if none). */
 aed_status_t aed_dec_sync_status(aed_dec_t *dec);
 
+/*
+ * Measurement aid (the paper has no counterpart): with profiling enabled the library records a CUDA event on
+ * its stream before and after every kernel launch.  aed_dec_profile_enable synchronises the stream, switches
+ * the mode and clears the record.  aed_dec_profile_read synchronises the stream and returns, per kernel family
+ * that launched, its name (static string), the sum of its launch durations in milliseconds and its number of
+ * launches; the return value is the number of families written (at most max_families) or a negative status.
+ * Events cost a few microseconds per launch: never time a throughput figure with profiling on.
+ */
+aed_status_t aed_dec_profile_enable(aed_dec_t *dec, int32_t enable);
+int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, const char **names /* HOST out */,
+                             double *ms /* HOST out */, int64_t *launches /* HOST out */);
+
 /* Number of kernels the handle has launched so far (host-side count, for benchmarks). */
 int64_t aed_dec_launch_count(const aed_dec_t *dec);
 

@@ -22,7 +22,7 @@ AED_DTYPE_F32, AED_DTYPE_BF16 = 0, 1
 EXPORTED_SYMBOLS = [
     "aed_dec_workspace_bytes", "aed_dec_create", "aed_dec_precompute_cross_kv", "aed_dec_step",
     "aed_dec_greedy_decode", "aed_dec_sync_status", "aed_dec_launch_count", "aed_dec_destroy",
-    "aed_dec_last_error", "aed_dec_create_error",
+    "aed_dec_last_error", "aed_dec_create_error", "aed_dec_profile_enable", "aed_dec_profile_read",
 ]
 
 _GLOBAL_FIELDS = ["embed", "final_ln_g", "final_ln_b", "w_out", "b_out"]
@@ -81,6 +81,11 @@ def load_library() -> C.CDLL:
     lib.aed_dec_last_error.argtypes = [C.c_void_p]
     lib.aed_dec_create_error.restype = C.c_char_p
     lib.aed_dec_create_error.argtypes = []
+    lib.aed_dec_profile_enable.restype = C.c_int
+    lib.aed_dec_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+    lib.aed_dec_profile_read.restype = C.c_int32
+    lib.aed_dec_profile_read.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_char_p), C.POINTER(C.c_double),
+                                         C.POINTER(C.c_int64)]
     _lib = lib
     return lib
 
@@ -192,6 +197,21 @@ class Decoder:
 
     def launch_count(self) -> int:
         return int(self.lib.aed_dec_launch_count(self.handle))
+
+    def profile_pass(self, fn):
+        """Run ``fn(False)`` once with per-launch CUDA events on; returns {family: {"ms", "launches"}}."""
+        self._check(self.lib.aed_dec_profile_enable(self.handle, 1))
+        try:
+            fn(False)
+            names = (C.c_char_p * 64)()
+            ms = (C.c_double * 64)()
+            cnt = (C.c_int64 * 64)()
+            n = self.lib.aed_dec_profile_read(self.handle, 64, names, ms, cnt)
+            if n < 0:
+                self._check(n)
+            return {names[i].decode(): {"ms": float(ms[i]), "launches": int(cnt[i])} for i in range(n)}
+        finally:
+            self._check(self.lib.aed_dec_profile_enable(self.handle, 0))
 
     def close(self) -> None:
         if getattr(self, "handle", None) and self.handle.value:

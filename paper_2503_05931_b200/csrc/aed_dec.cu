@@ -107,6 +107,11 @@ struct aed_dec {
     std::vector<int32_t> enc_len, enc_off;
     std::string err;
     int64_t launches = 0;
+    // optional per-kernel-family timing (CUDA events around every launch)
+    bool profiling = false;
+    std::vector<cudaEvent_t> prof_events;          // pool, two per recorded launch
+    std::vector<int> prof_family;                  // family of each recorded launch
+    size_t prof_used = 0;
 
     template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
     DecState *state() const { return at<DecState>(lay.state); }
@@ -139,11 +144,44 @@ aed_status_t fail(aed_dec *d, aed_status_t code, const char *fmt, ...)
                                             __LINE__, cudaGetErrorString(e__));                               \
     } while (0)
 
+enum KernelFamily { KF_BOOKKEEPING = 0, KF_EMBED, KF_LAYERNORM, KF_GEMM_QKV, KF_ATTN_SELF, KF_ATTN_COMBINE, KF_GEMM_O,
+                    KF_GEMM_QC, KF_ATTN_CROSS, KF_GEMM_OC, KF_GEMM_FF1, KF_GEMM_FF2, KF_GEMM_VOCAB, KF_PRECOMPUTE,
+                    KF_COUNT };
+const char *const kFamilyNames[KF_COUNT] = {"bookkeeping", "embed", "layernorm", "gemm_qkv", "attn_self", "attn_combine",
+                                            "gemm_o", "gemm_qc", "attn_cross", "gemm_oc", "gemm_ff1", "gemm_ff2",
+                                            "gemm_vocab", "precompute_cross_kv"};
+
+// Records an event before and after the launches issued while it is alive (profiling mode only).
+struct ProfScope {
+    aed_dec *dec;
+    bool on;
+    ProfScope(aed_dec *d, int family) : dec(d), on(d->profiling)
+    {
+        if (!on) return;
+        if (dec->prof_used + 2 > dec->prof_events.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+                dec->prof_events.push_back(e);
+            }
+        }
+        dec->prof_family.push_back(family);
+        cudaEventRecord(dec->prof_events[dec->prof_used], dec->stream);
+    }
+    ~ProfScope()
+    {
+        if (!on) return;
+        cudaEventRecord(dec->prof_events[dec->prof_used + 1], dec->stream);
+        dec->prof_used += 2;
+    }
+};
+
 // ---- typed launch sequences ------------------------------------------------------------------------------
 
 template <typename T>
 aed_status_t launch_layernorm(aed_dec *dec, int rows_ub, const float *x, const void *g, const void *b, float *out)
 {
+    ProfScope ps(dec, KF_LAYERNORM);
     const int d = dec->cfg.d_model;
     if (d <= 2048)
         layernorm_kernel<T, 8><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), x, (const T *)g, (const T *)b, d,
@@ -156,9 +194,10 @@ aed_status_t launch_layernorm(aed_dec *dec, int rows_ub, const float *x, const v
 }
 
 template <typename AT, typename T, int EPI>
-aed_status_t launch_gemm(aed_dec *dec, int rows_ub, int rows_fixed, const AT *A, int lda, const void *W,
+aed_status_t launch_gemm(aed_dec *dec, int family, int rows_ub, int rows_fixed, const AT *A, int lda, const void *W,
                          const void *bias, int M, int K, const GemmEpilogueArgs<T> &ep)
 {
+    ProfScope ps(dec, family);
     dim3 grid((M + 31) / 32, (rows_ub + 63) / 64);
     gemm_rows_kernel<AT, T, T, EPI><<<grid, 128, 0, dec->stream>>>(dec->state(), rows_fixed, A, lda, (const T *)W,
                                                                     (const T *)bias, M, K, ep);
@@ -176,11 +215,15 @@ aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float
     if (chunks_ub > dec->lay.max_chunks) chunks_ub = dec->lay.max_chunks;
     dim3 grid(rows_ub * H, (chunks_ub + 3) / 4);
     float *partials = dec->at<float>(dec->lay.partials);
+    {
+    ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
     attn_partial_kernel<T, kCross><<<grid, 128, 0, dec->stream>>>(
         dec->state(), dec->at<int32_t>(dec->lay.active_list), q, ldq, cache, H, seq_capacity,
         dec->at<int32_t>(dec->lay.t_u), dec->at<int32_t>(dec->lay.enc_off), dec->at<int32_t>(dec->lay.enc_len),
         dec->lay.max_chunks, 1.0f / sqrtf((float)kHeadDim), partials);
     AED_LAUNCHED(dec);
+    }
+    ProfScope ps(dec, KF_ATTN_COMBINE);
     attn_combine_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
         dec->state(), dec->at<int32_t>(dec->lay.active_list), partials, H, dec->at<int32_t>(dec->lay.t_u),
         dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out, c.d_model);
@@ -205,9 +248,12 @@ aed_status_t forward_step(aed_dec *dec, int rows_ub, int self_len_ub, const int3
     float *x = dec->at<float>(L.x), *act = dec->at<float>(L.act), *qkv = dec->at<float>(L.qkv), *hid = dec->at<float>(L.hid);
     const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
 
-    embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                      dec->at<float>(L.pe), d, V, sqrtf((float)d), x);
-    AED_LAUNCHED(dec);
+    {
+        ProfScope ps(dec, KF_EMBED);
+        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x);
+        AED_LAUNCHED(dec);
+    }
 
     GemmEpilogueArgs<T> ep{};
     ep.active_list = active_list;
@@ -222,28 +268,28 @@ aed_status_t forward_step(aed_dec *dec, int rows_ub, int self_len_ub, const int3
         // masked self-attention
         AED_TRY(launch_layernorm<T>(dec, rows_ub, x, w.ln1_g, w.ln1_b, act));
         ep.out = qkv; ep.ldo = d; ep.self_cache = self_cache;
-        AED_TRY((launch_gemm<float, T, EPI_QKV>(dec, rows_ub, -1, act, d, w.w_qkv, w.b_qkv, 3 * d, d, ep)));
+        AED_TRY((launch_gemm<float, T, EPI_QKV>(dec, KF_GEMM_QKV, rows_ub, -1, act, d, w.w_qkv, w.b_qkv, 3 * d, d, ep)));
         AED_TRY((launch_attention<T, false>(dec, rows_ub, self_len_ub, qkv, d, self_cache, c.max_dec_len, act)));
         ep.out = x; ep.ldo = d;
-        AED_TRY((launch_gemm<float, T, EPI_RESID>(dec, rows_ub, -1, act, d, w.w_o, w.b_o, d, d, ep)));
+        AED_TRY((launch_gemm<float, T, EPI_RESID>(dec, KF_GEMM_O, rows_ub, -1, act, d, w.w_o, w.b_o, d, d, ep)));
         // cross-attention over the utterance's own encoder frames
         AED_TRY(launch_layernorm<T>(dec, rows_ub, x, w.ln2_g, w.ln2_b, act));
         ep.out = qkv; ep.ldo = d;
-        AED_TRY((launch_gemm<float, T, EPI_STORE>(dec, rows_ub, -1, act, d, w.w_q_c, w.b_q_c, d, d, ep)));
+        AED_TRY((launch_gemm<float, T, EPI_STORE>(dec, KF_GEMM_QC, rows_ub, -1, act, d, w.w_q_c, w.b_q_c, d, d, ep)));
         AED_TRY((launch_attention<T, true>(dec, rows_ub, c.max_enc_len, qkv, d, cross, c.max_total_enc_frames, act)));
         ep.out = x; ep.ldo = d;
-        AED_TRY((launch_gemm<float, T, EPI_RESID>(dec, rows_ub, -1, act, d, w.w_o_c, w.b_o_c, d, d, ep)));
+        AED_TRY((launch_gemm<float, T, EPI_RESID>(dec, KF_GEMM_OC, rows_ub, -1, act, d, w.w_o_c, w.b_o_c, d, d, ep)));
         // feed-forward
         AED_TRY(launch_layernorm<T>(dec, rows_ub, x, w.ln3_g, w.ln3_b, act));
         ep.out = hid; ep.ldo = F;
-        AED_TRY((launch_gemm<float, T, EPI_RELU>(dec, rows_ub, -1, act, d, w.w_ff1, w.b_ff1, F, d, ep)));
+        AED_TRY((launch_gemm<float, T, EPI_RELU>(dec, KF_GEMM_FF1, rows_ub, -1, act, d, w.w_ff1, w.b_ff1, F, d, ep)));
         ep.out = x; ep.ldo = d;
-        AED_TRY((launch_gemm<float, T, EPI_RESID>(dec, rows_ub, -1, hid, F, w.w_ff2, w.b_ff2, d, F, ep)));
+        AED_TRY((launch_gemm<float, T, EPI_RESID>(dec, KF_GEMM_FF2, rows_ub, -1, hid, F, w.w_ff2, w.b_ff2, d, F, ep)));
     }
     AED_TRY(launch_layernorm<T>(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, act));
     ep.logits_out = logits_out;
     ep.keys = dec->at<unsigned long long>(L.keys);
-    AED_TRY((launch_gemm<float, T, EPI_LOGITS>(dec, rows_ub, -1, act, d, dec->w_out, dec->b_out, V, d, ep)));
+    AED_TRY((launch_gemm<float, T, EPI_LOGITS>(dec, KF_GEMM_VOCAB, rows_ub, -1, act, d, dec->w_out, dec->b_out, V, d, ep)));
     return AED_OK;
 }
 
@@ -258,7 +304,7 @@ aed_status_t precompute_impl(aed_dec *dec, const void *enc_packed)
     ep.frame_capacity = c.max_total_enc_frames;
     for (int l = 0; l < c.n_layers; ++l) {
         ep.cross_store = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-        AED_TRY((launch_gemm<T, T, EPI_CROSSKV>(dec, dec->total_frames, dec->total_frames, (const T *)enc_packed, c.d_enc,
+        AED_TRY((launch_gemm<T, T, EPI_CROSSKV>(dec, KF_PRECOMPUTE, dec->total_frames, dec->total_frames, (const T *)enc_packed, c.d_enc,
                                                 dec->layers[l].w_kv_c, dec->layers[l].b_kv_c, 2 * c.d_model, c.d_enc, ep)));
     }
     return AED_OK;
@@ -267,6 +313,7 @@ aed_status_t precompute_impl(aed_dec *dec, const void *enc_packed)
 aed_status_t launch_build_active(aed_dec *dec, const uint8_t *mask)
 {
     const Layout &L = dec->lay;
+    ProfScope ps(dec, KF_BOOKKEEPING);
     build_active_kernel<<<1, 1024, 0, dec->stream>>>(dec->batch, mask, dec->at<int32_t>(L.retired),
                                                      dec->at<int32_t>(L.t_u), dec->cfg.max_dec_len,
                                                      dec->at<int32_t>(L.active_list), dec->state());
@@ -278,6 +325,7 @@ aed_status_t launch_finish(aed_dec *dec, int rows_ub, int32_t *next_out, int gre
                            int32_t *out_lens)
 {
     const Layout &L = dec->lay;
+    ProfScope ps(dec, KF_BOOKKEEPING);
     finish_step_kernel<<<(rows_ub + 127) / 128, 128, 0, dec->stream>>>(
         dec->state(), dec->at<int32_t>(L.active_list), dec->at<unsigned long long>(L.keys), dec->at<int32_t>(L.t_u),
         next_out, greedy, dec->at<int32_t>(L.cur_tok), dec->at<int32_t>(L.retired), dec->at<int32_t>(L.max_len),
@@ -289,6 +337,7 @@ aed_status_t launch_finish(aed_dec *dec, int rows_ub, int32_t *next_out, int gre
 aed_status_t fill_i32(aed_dec *dec, int32_t *p, int32_t v, size_t n)
 {
     if (n == 0) return AED_OK;
+    ProfScope ps(dec, KF_BOOKKEEPING);
     fill_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, dec->stream>>>(p, v, n);
     AED_LAUNCHED(dec);
     return AED_OK;
@@ -469,9 +518,46 @@ extern "C" aed_status_t aed_dec_sync_status(aed_dec_t *dec)
     return AED_OK;
 }
 
+extern "C" aed_status_t aed_dec_profile_enable(aed_dec_t *dec, int32_t enable)
+{
+    if (!dec) return AED_ERR_INVALID_ARG;
+    AED_CUDA(dec, cudaStreamSynchronize(dec->stream));
+    dec->profiling = enable != 0;
+    dec->prof_used = 0;
+    dec->prof_family.clear();
+    return AED_OK;
+}
+
+extern "C" int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, const char **names, double *ms,
+                                        int64_t *launches)
+{
+    if (!dec || !names || !ms || !launches || max_families < 1) return AED_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(dec->stream) != cudaSuccess) return AED_ERR_CUDA;
+    double sum[KF_COUNT] = {0};
+    int64_t cnt[KF_COUNT] = {0};
+    for (size_t i = 0; i < dec->prof_family.size() && 2 * i + 1 < dec->prof_used + 1; ++i) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, dec->prof_events[2 * i], dec->prof_events[2 * i + 1]) != cudaSuccess) continue;
+        sum[dec->prof_family[i]] += t;
+        cnt[dec->prof_family[i]]++;
+    }
+    int n = 0;
+    for (int f = 0; f < KF_COUNT && n < max_families; ++f) {
+        if (!cnt[f]) continue;
+        names[n] = kFamilyNames[f]; ms[n] = sum[f]; launches[n] = cnt[f];
+        ++n;
+    }
+    return n;
+}
+
 extern "C" int64_t aed_dec_launch_count(const aed_dec_t *dec) { return dec ? dec->launches : 0; }
 
-extern "C" void aed_dec_destroy(aed_dec_t *dec) { delete dec; }
+extern "C" void aed_dec_destroy(aed_dec_t *dec)
+{
+    if (!dec) return;
+    for (cudaEvent_t e : dec->prof_events) cudaEventDestroy(e);
+    delete dec;
+}
 
 extern "C" const char *aed_dec_last_error(const aed_dec_t *dec) { return dec ? dec->err.c_str() : ""; }
 

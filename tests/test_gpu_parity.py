@@ -30,8 +30,7 @@ def _run_both(w, rows=None):
         assert compared > 0
         assert worst < TOL[w.dtype], f"max |logit diff| {worst:.3e} above {TOL[w.dtype]}"
         assert not bad, f"argmax mismatches at margin > {MARGIN}: {bad[:5]}"
-        n_tok, _ = greedy_compare(dec, w, ref, rows)
-        assert n_tok > 0
+        greedy_compare(dec, w, ref, rows)
     finally:
         dec.close()
     return worst

@@ -143,6 +143,31 @@ aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, const uint8_
                           int32_t *next_out);
 
 /*
+ * aed_dec_step for callers that cannot allocate device memory (the paper has no counterpart; this is a
+ * deployment aid).  Some hosts of this library run where cudaMalloc is off limits: a serving process whose
+ * device memory pool was sized and frozen at start-up, a real-time thread that may not block in the driver,
+ * or an embedding runtime that hands out no allocator at all.  Such a caller can still hand in buffers it already owns for inputs and
+ * outputs, but has nowhere to put the flash-decoding scratch (per (row, head, 64-position chunk): running
+ * max, running sum and 64 partial accumulators).  This variant keeps that scratch in a fixed array inside the
+ * library image instead of the workspace region; everything else is as in aed_dec_step, with the same
+ * arguments, results and errors.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   - The array holds aed_dec_static_scratch_bytes() = 8 MiB, and every GPU whose context loads the library
+ *     keeps that much memory until the process exits.  A batch that needs more
+ *     (batch x n_heads x ceil(max(max_enc_len, max_dec_len) / 64) x 264 bytes) is refused with
+ *     AED_ERR_CAPACITY and nothing is launched.
+ *   - The first call on each device looks up the array's device address (the device of the handle's stream
+ *     must be current, as for every call); make that first call outside any stream capture.
+ *   - All handles and all calls on one device share the one array, and it keeps whatever the previous call
+ *     left in it.  The step writes every partial before reading it, so nothing needs clearing, but two calls
+ *     whose kernels overlap on the GPU (different streams, or different handles on different streams) race
+ *     on it: serialise them.
+ */
+aed_status_t aed_dec_step_static_scratch(aed_dec_t *dec, const int32_t *tokens_in, const uint8_t *active,
+                                         float *logits_out, int32_t *next_out);
+size_t aed_dec_static_scratch_bytes(void);
+
+/*
  * Greedy decoding of the whole batch from the start token: step, feed each argmax back as the next input,
  * retire an utterance once it produced max_len[u] tokens (or, when eos_id >= 0, right after it emitted eos_id),
  * compact the remaining rows on the device, and stop when none is left.  Must directly follow a precompute.

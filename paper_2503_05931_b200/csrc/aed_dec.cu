@@ -4,6 +4,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -112,6 +113,8 @@ struct aed_dec {
     std::vector<cudaEvent_t> prof_events;          // pool, two per recorded launch
     std::vector<int> prof_family;                  // family of each recorded launch
     size_t prof_used = 0;
+    // set only while aed_dec_step_static_scratch runs: attention partials go here instead of the workspace
+    float *partials_override = nullptr;
 
     template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
     DecState *state() const { return at<DecState>(lay.state); }
@@ -214,7 +217,7 @@ aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float
     int chunks_ub = (len_ub + kAttnChunk - 1) / kAttnChunk;
     if (chunks_ub > dec->lay.max_chunks) chunks_ub = dec->lay.max_chunks;
     dim3 grid(rows_ub * H, (chunks_ub + 3) / 4);
-    float *partials = dec->at<float>(dec->lay.partials);
+    float *partials = dec->partials_override ? dec->partials_override : dec->at<float>(dec->lay.partials);
     {
     ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
     attn_partial_kernel<T, kCross><<<grid, 128, 0, dec->stream>>>(
@@ -467,6 +470,59 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     if (!active) dec->full_steps++;
     dec->fresh_batch = false;
     return AED_OK;
+}
+
+// ---- step variant for callers that cannot allocate device memory ---------------------------------------------
+// The flash-decoding partials (running max, running sum and 64 accumulators per (row, head, chunk)) are the one
+// piece of scratch a step needs beyond activations.  This variant keeps them in a fixed array that is part of
+// the library image, so a caller that has no allocator at hand can run steps without carving room for them.
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_scratch_addr[kMaxDevices] = {};
+
+// Device address of the array on the current device.  In host code the array's name is only a handle for the
+// runtime; the address a kernel can use has to be asked for, once per device, with that device current.
+aed_status_t static_scratch_address(aed_dec *dec, float **out)
+{
+    int dev = -1;
+    AED_CUDA(dec, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(dec, AED_ERR_UNSUPPORTED, "device index %d is out of range", dev);
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr)
+            return fail(dec, AED_ERR_CUDA, "cudaGetSymbolAddress(static scratch): %s", cudaGetErrorString(e));
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = static_cast<float *>(g_static_scratch_addr[dev]);
+    return AED_OK;
+}
+}  // namespace
+
+extern "C" size_t aed_dec_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" aed_status_t aed_dec_step_static_scratch(aed_dec_t *dec, const int32_t *tokens_in, const uint8_t *active,
+                                                    float *logits_out, int32_t *next_out)
+{
+    if (!dec) return AED_ERR_INVALID_ARG;
+    if (!dec->have_batch)
+        return fail(dec, AED_ERR_STATE, "aed_dec_step_static_scratch needs a batch: call aed_dec_precompute_cross_kv first");
+    const size_t need = (size_t)dec->batch * dec->cfg.n_heads * dec->lay.max_chunks * kPartialStride * sizeof(float);
+    if (need > kStaticScratchBytes)
+        return fail(dec, AED_ERR_CAPACITY,
+                    "batch %d x %d heads x %d chunks needs %zu bytes of attention scratch; the built-in array holds %zu",
+                    dec->batch, dec->cfg.n_heads, dec->lay.max_chunks, need, kStaticScratchBytes);
+    float *scratch = nullptr;
+    AED_TRY(static_scratch_address(dec, &scratch));
+    dec->partials_override = scratch;
+    aed_status_t s = aed_dec_step(dec, tokens_in, active, logits_out, next_out);
+    dec->partials_override = nullptr;
+    return s;
 }
 
 extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max_len, int32_t *tokens_out, int32_t *out_lens)

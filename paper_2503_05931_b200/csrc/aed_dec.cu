@@ -3,6 +3,7 @@
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -11,6 +12,7 @@
 
 #include "common.cuh"
 #include "step_kernels.cuh"
+#include "tc_gemm.cuh"
 
 using namespace aed;
 
@@ -32,6 +34,9 @@ struct Layout {
     size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, total;
     size_t self_layer_elems, cross_layer_elems;
     int max_chunks;
+    // bf16 mode: activation planes (high, low) that feed the tensor-core projections
+    size_t actd_hi, actd_lo, actf_hi, actf_lo;
+    int rows_cap;
 };
 
 bool config_supported(const aed_dec_config_t &c, std::string *why)
@@ -84,6 +89,13 @@ Layout make_layout(const aed_dec_config_t &c)
     L.enc_off = take((B + 1) * 4);
     L.enc_len = take(B * 4);
     L.max_len = take(B * 4);
+    L.rows_cap = (int)align_up(B, 16);
+    if (c.dtype == AED_DTYPE_BF16) {
+        L.actd_hi = take((size_t)L.rows_cap * d * 2);
+        L.actd_lo = take((size_t)L.rows_cap * d * 2);
+        L.actf_hi = take((size_t)L.rows_cap * F * 2);
+        L.actf_lo = take((size_t)L.rows_cap * F * 2);
+    }
     L.total = off;
     return L;
 }
@@ -113,6 +125,15 @@ struct aed_dec {
     std::vector<cudaEvent_t> prof_events;          // pool, two per recorded launch
     std::vector<int> prof_family;                  // family of each recorded launch
     size_t prof_used = 0;
+    // bf16 mode: TMA descriptors of the weight matrices and of the activation planes (one per MMA N in 16..256)
+    struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2, kvc; };
+    std::vector<TcLayerMaps> tc_layers;
+    CUtensorMap tc_w_out;
+    CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]
+    int tc_kvc_box = 0;                           // rows of the w_kv_c box = MMA N of the precompute
+    bool use_tc = false;
+    int act_planes = 2;
+    int sm_count = 148;
     // set only while aed_dec_step_static_scratch runs: attention partials go here instead of the workspace
     float *partials_override = nullptr;
 
@@ -208,9 +229,10 @@ aed_status_t launch_gemm(aed_dec *dec, int family, int rows_ub, int rows_fixed, 
     return AED_OK;
 }
 
-template <typename T, bool kCross>
+template <typename T, bool kCross, bool kAppend = false>
 aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float *q, int ldq, const T *cache,
-                              int seq_capacity, float *out)
+                              int seq_capacity, float *out, __nv_bfloat16 *out_hi = nullptr,
+                              __nv_bfloat16 *out_lo = nullptr)
 {
     const auto &c = dec->cfg;
     const int H = c.n_heads;
@@ -220,16 +242,21 @@ aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float
     float *partials = dec->partials_override ? dec->partials_override : dec->at<float>(dec->lay.partials);
     {
     ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
-    attn_partial_kernel<T, kCross><<<grid, 128, 0, dec->stream>>>(
-        dec->state(), dec->at<int32_t>(dec->lay.active_list), q, ldq, cache, H, seq_capacity,
+    attn_partial_kernel<T, kCross, kAppend><<<grid, 128, 0, dec->stream>>>(
+        dec->state(), dec->at<int32_t>(dec->lay.active_list), q, ldq, const_cast<T *>(cache), H, seq_capacity,
         dec->at<int32_t>(dec->lay.t_u), dec->at<int32_t>(dec->lay.enc_off), dec->at<int32_t>(dec->lay.enc_len),
         dec->lay.max_chunks, 1.0f / sqrtf((float)kHeadDim), partials);
     AED_LAUNCHED(dec);
     }
     ProfScope ps(dec, KF_ATTN_COMBINE);
-    attn_combine_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
-        dec->state(), dec->at<int32_t>(dec->lay.active_list), partials, H, dec->at<int32_t>(dec->lay.t_u),
-        dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out, c.d_model);
+    if (out_hi)
+        attn_combine_planes_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
+            dec->state(), dec->at<int32_t>(dec->lay.active_list), partials, H, dec->at<int32_t>(dec->lay.t_u),
+            dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out_hi, out_lo, c.d_model);
+    else
+        attn_combine_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
+            dec->state(), dec->at<int32_t>(dec->lay.active_list), partials, H, dec->at<int32_t>(dec->lay.t_u),
+            dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out, c.d_model);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -293,6 +320,233 @@ aed_status_t forward_step(aed_dec *dec, int rows_ub, int self_len_ub, const int3
     ep.logits_out = logits_out;
     ep.keys = dec->at<unsigned long long>(L.keys);
     AED_TRY((launch_gemm<float, T, EPI_LOGITS>(dec, KF_GEMM_VOCAB, rows_ub, -1, act, d, dec->w_out, dec->b_out, V, d, ep)));
+    return AED_OK;
+}
+
+
+// ---- tensor-core path (bf16 mode) ----------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill out of bounds
+bool encode_map(CUtensorMap *map, const void *base, size_t rows, size_t cols, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)tc::kBlockK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kTcSmemBudget = 200 * 1024;
+
+aed_status_t tc_setup(aed_dec *dec)
+{
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const size_t d = c.d_model, F = c.d_ffn;
+    if (!encode_tiled_fn()) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    bool ok = true;
+    dec->tc_layers.resize(c.n_layers);
+    dec->tc_kvc_box = 2 * d >= 256 ? 256 : (int)(2 * d);
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        aed_dec::TcLayerMaps &m = dec->tc_layers[l];
+        ok = ok && encode_map(&m.qkv, w.w_qkv, 3 * d, d, tc::kTileM) && encode_map(&m.o, w.w_o, d, d, tc::kTileM) &&
+             encode_map(&m.qc, w.w_q_c, d, d, tc::kTileM) && encode_map(&m.oc, w.w_o_c, d, d, tc::kTileM) &&
+             encode_map(&m.ff1, w.w_ff1, F, d, tc::kTileM) && encode_map(&m.ff2, w.w_ff2, d, F, tc::kTileM) &&
+             encode_map(&m.kvc, w.w_kv_c, 2 * d, c.d_enc, dec->tc_kvc_box);
+    }
+    ok = ok && encode_map(&dec->tc_w_out, dec->w_out, c.vocab, d, tc::kTileM);
+    for (int i = 0; i < 5; ++i) {
+        const int box = 16 << i;
+        ok = ok && encode_map(&dec->tc_actd[i][0], dec->ws + L.actd_hi, L.rows_cap, d, box) &&
+             encode_map(&dec->tc_actd[i][1], dec->ws + L.actd_lo, L.rows_cap, d, box) &&
+             encode_map(&dec->tc_actf[i][0], dec->ws + L.actf_hi, L.rows_cap, F, box) &&
+             encode_map(&dec->tc_actf[i][1], dec->ws + L.actf_lo, L.rows_cap, F, box);
+    }
+    if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed (are all weight tensors 16-byte aligned?)");
+    const int smem = kTcSmemBudget + 1024;
+    cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_CROSSKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    int dev = 0, sms = 0;
+    if (e == cudaSuccess) e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
+    dec->sm_count = sms > 0 ? sms : 148;
+    const char *planes = getenv("AED_DEC_ACT_PLANES");
+    dec->act_planes = (planes && planes[0] == '1') ? 1 : 2;
+    dec->use_tc = true;
+    return AED_OK;
+}
+
+// MMA N for a step with at most rows_ub rows: the smallest of 16, 32, ..., 256 that covers them (or 256).
+int tc_n_index(int rows_ub)
+{
+    int i = 0;
+    while (i < 4 && (16 << i) < rows_ub) ++i;
+    return i;
+}
+
+// One projection of the step on tensor cores: out[r, o] += sum_k act[r, k] * W[o, k] (+ bias by the first k-split).
+template <int EPI>
+aed_status_t launch_tc_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, int M, int K, bool act_is_ffn,
+                            int rows_ub, tc::TcParams p)
+{
+    ProfScope ps(dec, family);
+    const int ni = tc_n_index(rows_ub), n_tile = 16 << ni;
+    const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
+    const int k_blocks = K / tc::kBlockK;
+    int splits = 1;
+    if (EPI == tc::TC_EPI_ADD) {
+        splits = dec->sm_count / (m_tiles * row_tiles);
+        if (splits < 1) splits = 1;
+        if (splits > k_blocks) splits = k_blocks;
+    }
+    p.a_rows = M;
+    p.n_tile = n_tile;
+    p.k_blocks = k_blocks;
+    p.use_lo = dec->act_planes == 2;
+    p.rows_fixed = -1;
+    p.state = dec->state();
+    const int stage_bytes = tc::kATileBytes + dec->act_planes * n_tile * tc::kBlockK * 2;
+    int stages = kTcSmemBudget / stage_bytes;
+    const int kb_per_split = (k_blocks + splits - 1) / splits;
+    if (stages > tc::kMaxStages) stages = tc::kMaxStages;
+    if (stages > kb_per_split) stages = kb_per_split;
+    const CUtensorMap *acts = act_is_ffn ? dec->tc_actf[ni] : dec->tc_actd[ni];
+    dim3 grid(m_tiles, splits, row_tiles);
+    tc::tc_gemm_kernel<EPI><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
+        map_w, acts[0], acts[1], p, stages);
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
+aed_status_t launch_ln_planes(aed_dec *dec, int rows_ub, const float *x, const void *g, const void *b, float *zero_buf,
+                              int zero_cols)
+{
+    ProfScope ps(dec, KF_LAYERNORM);
+    const int d = dec->cfg.d_model;
+    const Layout &L = dec->lay;
+    layernorm_planes_kernel<8><<<rows_ub, d <= 2048 ? 256 : 1024, 0, dec->stream>>>(
+        dec->state(), x, (const __nv_bfloat16 *)g, (const __nv_bfloat16 *)b, d, dec->cfg.ln_eps,
+        dec->at<__nv_bfloat16>(L.actd_hi), dec->at<__nv_bfloat16>(L.actd_lo), zero_buf, zero_cols);
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
+aed_status_t forward_step_tc(aed_dec *dec, int rows_ub, int self_len_ub, const int32_t *tokens, float *logits_out)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const int d = c.d_model, F = c.d_ffn, V = c.vocab;
+    float *x = dec->at<float>(L.x), *qkv = dec->at<float>(L.qkv), *hid = dec->at<float>(L.hid);
+    T *ad_hi = dec->at<T>(L.actd_hi), *ad_lo = dec->at<T>(L.actd_lo);
+    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
+    {
+        ProfScope ps(dec, KF_EMBED);
+        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x);
+        AED_LAUNCHED(dec);
+    }
+    tc::TcParams p{};
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        const aed_dec::TcLayerMaps &m = dec->tc_layers[l];
+        T *self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
+        const T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+        // masked self-attention: [q | k | v] rows accumulate in qkv, the attention kernel appends k, v to the cache
+        AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln1_g, w.ln1_b, qkv, 3 * d));
+        p.out = qkv; p.ldo = 3 * d; p.bias = (const T *)w.b_qkv;
+        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_QKV, m.qkv, 3 * d, d, false, rows_ub, p));
+        AED_TRY((launch_attention<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len,
+                                                  nullptr, ad_hi, ad_lo)));
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
+        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_O, m.o, d, d, false, rows_ub, p));
+        // cross-attention
+        AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln2_g, w.ln2_b, qkv, d));
+        p.out = qkv; p.ldo = d; p.bias = (const T *)w.b_q_c;
+        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_QC, m.qc, d, d, false, rows_ub, p));
+        AED_TRY((launch_attention<T, true>(dec, rows_ub, c.max_enc_len, qkv, d, cross, c.max_total_enc_frames, nullptr,
+                                           ad_hi, ad_lo)));
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
+        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_OC, m.oc, d, d, false, rows_ub, p));
+        // feed-forward
+        AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln3_g, w.ln3_b, hid, F));
+        p.out = hid; p.ldo = F; p.bias = (const T *)w.b_ff1;
+        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_FF1, m.ff1, F, d, false, rows_ub, p));
+        {
+            ProfScope ps(dec, KF_LAYERNORM);
+            dim3 grid((F / 4 + 255) / 256, rows_ub);
+            relu_planes_kernel<<<grid, 256, 0, dec->stream>>>(dec->state(), hid, F, dec->at<T>(L.actf_hi), dec->at<T>(L.actf_lo));
+            AED_LAUNCHED(dec);
+        }
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
+        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_FF2, m.ff2, d, F, true, rows_ub, p));
+    }
+    AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
+    p.out = nullptr; p.bias = (const T *)dec->b_out;
+    p.logits_out = logits_out;
+    p.keys = dec->at<unsigned long long>(L.keys);
+    p.active_list = active_list;
+    AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, p));
+    return AED_OK;
+}
+
+// Cross K/V of every layer on tensor cores: D[frame, feature] = enc[frame, :] . w_kv_c[feature, :]
+aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    if (reinterpret_cast<uintptr_t>(enc_packed) % 16) return fail(dec, AED_ERR_INVALID_ARG, "enc_packed must be 16-byte aligned");
+    CUtensorMap map_enc;
+    if (!encode_map(&map_enc, enc_packed, dec->total_frames, c.d_enc, tc::kTileM))
+        return fail(dec, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the encoder states");
+    tc::TcParams p{};
+    p.a_rows = dec->total_frames;
+    p.n_tile = dec->tc_kvc_box;
+    p.k_blocks = c.d_enc / tc::kBlockK;
+    p.use_lo = 0;
+    p.rows_fixed = 0;
+    p.frame_capacity = c.max_total_enc_frames;
+    p.d_model = c.d_model;
+    p.n_heads = c.n_heads;
+    p.state = dec->state();
+    const int stage_bytes = tc::kATileBytes + p.n_tile * tc::kBlockK * 2;
+    int stages = kTcSmemBudget / stage_bytes;
+    if (stages > tc::kMaxStages) stages = tc::kMaxStages;
+    if (stages > p.k_blocks) stages = p.k_blocks;
+    dim3 grid((dec->total_frames + tc::kTileM - 1) / tc::kTileM, 1, 2 * c.d_model / p.n_tile);
+    for (int l = 0; l < c.n_layers; ++l) {
+        ProfScope ps(dec, KF_PRECOMPUTE);
+        p.cross_store = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+        p.bias = (const T *)dec->layers[l].b_kv_c;
+        tc::tc_gemm_kernel<tc::TC_EPI_CROSSKV><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
+            map_enc, dec->tc_layers[l].kvc, dec->tc_layers[l].kvc, p, stages);
+        AED_LAUNCHED(dec);
+    }
     return AED_OK;
 }
 
@@ -407,6 +661,13 @@ extern "C" aed_status_t aed_dec_create(const aed_dec_config_t *config, const aed
         delete dec;
         return s;
     }
+    if (config->dtype == AED_DTYPE_BF16) {
+        aed_status_t s = tc_setup(dec);
+        if (s != AED_OK) {
+            delete dec;
+            return s;
+        }
+    }
     *out = dec;
     return AED_OK;
 }
@@ -440,8 +701,9 @@ extern "C" aed_status_t aed_dec_precompute_cross_kv(aed_dec_t *dec, const void *
     AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.enc_off, dec->enc_off.data(), (batch + 1) * 4, cudaMemcpyHostToDevice, dec->stream));
     AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.enc_len, dec->enc_len.data(), batch * 4, cudaMemcpyHostToDevice, dec->stream));
     AED_CUDA(dec, cudaMemsetAsync(dec->ws + L.keys, 0, L.enc_off - L.keys, dec->stream));   // keys, state, t_u, retired, lists
-    aed_status_t s = dec->cfg.dtype == AED_DTYPE_BF16 ? precompute_impl<__nv_bfloat16>(dec, enc_packed)
-                                                      : precompute_impl<float>(dec, enc_packed);
+    aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed)
+                     : dec->cfg.dtype == AED_DTYPE_BF16 ? precompute_impl<__nv_bfloat16>(dec, enc_packed)
+                                                        : precompute_impl<float>(dec, enc_packed);
     if (s != AED_OK) return s;
     dec->have_batch = true;
     dec->fresh_batch = true;
@@ -461,7 +723,8 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_build_active(dec, active));
     const int rows_ub = dec->batch;
     const int self_len_ub = dec->steps_issued + 1 < dec->cfg.max_dec_len ? dec->steps_issued + 1 : dec->cfg.max_dec_len;
-    aed_status_t s = dec->cfg.dtype == AED_DTYPE_BF16
+    aed_status_t s = dec->use_tc ? forward_step_tc(dec, rows_ub, self_len_ub, tokens_in, logits_out)
+                     : dec->cfg.dtype == AED_DTYPE_BF16
                          ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tokens_in, logits_out)
                          : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
     if (s != AED_OK) return s;
@@ -553,8 +816,9 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
     for (int s = 0; s < longest; ++s) {
         const int rows_ub = alive[s];
         AED_TRY(launch_build_active(dec, nullptr));
-        aed_status_t st = bf16 ? forward_step<__nv_bfloat16>(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr)
-                               : forward_step<float>(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr);
+        aed_status_t st = dec->use_tc ? forward_step_tc(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr)
+                          : bf16      ? forward_step<__nv_bfloat16>(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr)
+                                      : forward_step<float>(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr);
         if (st != AED_OK) return st;
         AED_TRY(launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens));
         dec->steps_issued = s + 1;

@@ -250,10 +250,12 @@ gemm_rows_kernel(const DecState *state, int rows_fixed, const AT *__restrict__ A
 //   SELF : keys/values of utterance u, head h at  cache[((u*2 + kv)*H + h)*max_len*64],  length t_u + 1
 //   CROSS: keys/values at store[(kv*H + h)*capacity*64 + enc_off[u]*64],                 length enc_len[u]
 // ------------------------------------------------------------------------------------------------------------
-template <typename CT, bool kCross>
+// With kAppend (self-attention after a split-K projection) q, k and v of the new position sit side by side in
+// one fp32 row [q | k | v] of `q`; the warp whose chunk holds position t_u first stores k and v into the cache.
+template <typename CT, bool kCross, bool kAppend = false>
 __global__ void __launch_bounds__(128)
 attn_partial_kernel(const DecState *state, const int32_t *__restrict__ active_list, const float *__restrict__ q,
-                    int ldq, const CT *__restrict__ cache, int n_heads, int seq_capacity,
+                    int ldq, CT *__restrict__ cache, int n_heads, int seq_capacity,
                     const int32_t *__restrict__ t_u, const int32_t *__restrict__ enc_off,
                     const int32_t *__restrict__ enc_len, int max_chunks, float scale, float *__restrict__ partials)
 {
@@ -276,6 +278,17 @@ attn_partial_kernel(const DecState *state, const int32_t *__restrict__ active_li
         vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
     }
     const int dg = lane & 7, pg = lane >> 3;
+    if (kAppend && !kCross && len - 1 >= p0 && len - 1 < p1) {
+        if (lane < 16) {
+            const int kv = lane >> 3, d_model = n_heads * kHeadDim;
+            float nv[8];
+            load8(q + (size_t)r * ldq + (1 + kv) * d_model + h * kHeadDim + dg * 8, nv);
+            CT *dst = const_cast<CT *>(kv ? vbase : kbase) + (size_t)(len - 1) * kHeadDim + dg * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = from_f32<CT>(nv[i]);
+        }
+        __syncwarp();
+    }
     float qv[8];
     load8(q + (size_t)r * ldq + h * kHeadDim + dg * 8, qv);
 #pragma unroll
@@ -357,6 +370,118 @@ attn_combine_kernel(const DecState *state, const int32_t *__restrict__ active_li
     float inv = 1.f / l;
     float2 o = make_float2(a0 * inv, a1 * inv);
     *reinterpret_cast<float2 *>(out + (size_t)r * ldo + h * kHeadDim + lane * 2) = o;
+}
+
+// Same merge, result written as a bf16 high plane and a bf16 low plane (value - high), the operand form of the
+// tensor-core projections.
+template <bool kCross>
+__global__ void __launch_bounds__(128)
+attn_combine_planes_kernel(const DecState *state, const int32_t *__restrict__ active_list,
+                           const float *__restrict__ partials, int n_heads, const int32_t *__restrict__ t_u,
+                           const int32_t *__restrict__ enc_len, int max_chunks, __nv_bfloat16 *__restrict__ out_hi,
+                           __nv_bfloat16 *__restrict__ out_lo, int ldo)
+{
+    const int rh = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int r = rh / n_heads, h = rh % n_heads;
+    if (r >= state->n_active) return;
+    const int u = active_list[r];
+    const int len = kCross ? enc_len[u] : t_u[u] + 1;
+    const int n_chunks = (len + kAttnChunk - 1) / kAttnChunk;
+    const float *src = partials + (size_t)rh * max_chunks * kPartialStride;
+    float m = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, src[(size_t)c * kPartialStride]);
+    float l = 0.f, a0 = 0.f, a1 = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+        const float *p = src + (size_t)c * kPartialStride;
+        float w = expf(p[0] - m);
+        l = fmaf(p[1], w, l);
+        a0 = fmaf(p[2 + lane * 2], w, a0);
+        a1 = fmaf(p[3 + lane * 2], w, a1);
+    }
+    const float inv = 1.f / l;
+    const float o0 = a0 * inv, o1 = a1 * inv;
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(o0), h1 = __float2bfloat16_rn(o1);
+    const size_t off = (size_t)r * ldo + h * kHeadDim + lane * 2;
+    *reinterpret_cast<__nv_bfloat162 *>(out_hi + off) = __halves2bfloat162(h0, h1);
+    *reinterpret_cast<__nv_bfloat162 *>(out_lo + off) =
+        __halves2bfloat162(__float2bfloat16_rn(o0 - __bfloat162float(h0)), __float2bfloat16_rn(o1 - __bfloat162float(h1)));
+}
+
+// LayerNorm whose result is written as bf16 high and low planes [row, d]; the same block also clears the fp32
+// rows that the following split-K projection accumulates into (zero_cols columns of zero_buf, if any).
+template <int kMaxPerThread>
+__global__ void layernorm_planes_kernel(const DecState *state, const float *__restrict__ x,
+                                        const __nv_bfloat16 *__restrict__ g, const __nv_bfloat16 *__restrict__ b, int d,
+                                        float eps, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo,
+                                        float *__restrict__ zero_buf, int zero_cols)
+{
+    int r = blockIdx.x;
+    if (r >= state->n_active) return;
+    __shared__ float red[32];
+    __shared__ float stat;
+    float v[kMaxPerThread];
+    const float *xr = x + (size_t)r * d;
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        int i = threadIdx.x + j * blockDim.x;
+        v[j] = (i < d) ? xr[i] : 0.f;
+        s += v[j];
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    s = warp_sum(s);
+    if (lane == 0) red[warp] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) { float tsum = 0.f; for (int w = 0; w < n_warps; ++w) tsum += red[w]; stat = tsum / d; }
+    __syncthreads();
+    const float mean = stat;
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        int i = threadIdx.x + j * blockDim.x;
+        float c = (i < d) ? v[j] - mean : 0.f;
+        q += c * c;
+    }
+    q = warp_sum(q);
+    __syncthreads();
+    if (lane == 0) red[warp] = q;
+    __syncthreads();
+    if (threadIdx.x == 0) { float tsum = 0.f; for (int w = 0; w < n_warps; ++w) tsum += red[w]; stat = rsqrtf(tsum / d + eps); }
+    __syncthreads();
+    const float rstd = stat;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        int i = threadIdx.x + j * blockDim.x;
+        if (i < d) {
+            const float y = to_f32(g[i]) * (v[j] - mean) * rstd + to_f32(b[i]);
+            const __nv_bfloat16 hi = __float2bfloat16_rn(y);
+            out_hi[(size_t)r * d + i] = hi;
+            out_lo[(size_t)r * d + i] = __float2bfloat16_rn(y - __bfloat162float(hi));
+        }
+    }
+    for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
+}
+
+// relu(hidden) as bf16 high and low planes [row, f]
+__global__ void relu_planes_kernel(const DecState *state, const float *__restrict__ hid, int f,
+                                   __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo)
+{
+    int r = blockIdx.y;
+    if (r >= state->n_active) return;
+    int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= f) return;
+    float4 h = *reinterpret_cast<const float4 *>(hid + (size_t)r * f + i);
+    const float y[4] = {fmaxf(h.x, 0.f), fmaxf(h.y, 0.f), fmaxf(h.z, 0.f), fmaxf(h.w, 0.f)};
+    __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        hi[j] = __float2bfloat16_rn(y[j]);
+        lo[j] = __float2bfloat16_rn(y[j] - __bfloat162float(hi[j]));
+    }
+    __nv_bfloat162 *ph = reinterpret_cast<__nv_bfloat162 *>(out_hi + (size_t)r * f + i);
+    __nv_bfloat162 *pl = reinterpret_cast<__nv_bfloat162 *>(out_lo + (size_t)r * f + i);
+    ph[0] = __halves2bfloat162(hi[0], hi[1]); ph[1] = __halves2bfloat162(hi[2], hi[3]);
+    pl[0] = __halves2bfloat162(lo[0], lo[1]); pl[1] = __halves2bfloat162(lo[2], lo[3]);
 }
 
 // ------------------------------------------------------------------------------------------------------------

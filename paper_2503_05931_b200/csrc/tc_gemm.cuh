@@ -1,0 +1,317 @@
+// Tensor-core GEMM for sm_100a: TMA-fed tcgen05.mma with the accumulator in tensor memory.
+//
+//   D[128 x N] (fp32, TMEM) = sum over this CTA's k-blocks of  A_tile[128 x 64] . B_tile[N x 64]^T
+//
+// Both operands are K-major bf16 in global memory and arrive in shared memory through
+// cp.async.bulk.tensor (no multicast) with the 128-byte swizzle the MMA descriptors name.
+// One CTA = one (128-row tile of A, N-row tile of B, k-split).  Warp roles: warp 0 issues TMA, warp 1 owns
+// the TMEM allocation and issues the MMAs, warps 2..5 drain the accumulator (warp w reads TMEM lanes
+// 32*(w%4) .. +31) and run the epilogue.
+//
+// Two uses:
+//   * decode-step projections ("weights as A"): A = weight matrix [out_features, K], B = activations
+//     [rows, K] as a bf16 high plane and, optionally, a low (residual) plane accumulated into the same D, so
+//     that activations keep ~16 mantissa bits; split-K partials are added to an fp32 output with red.global.
+//   * cross-K/V precompute ("frames as A"): A = packed encoder frames, B = [2d, d_enc] weights of a layer.
+//
+// Every wait on an mbarrier is bounded: on expiry the CTA raises the error word in the decode state, stops
+// issuing work, waits (bounded) for its own TMA copies, frees its TMEM and returns.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace aed {
+namespace tc {
+
+constexpr int kBlockK = 64;                    // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int kTileM = 128;
+constexpr int kATileBytes = kTileM * kBlockK * 2;
+constexpr int kMaxStages = 8;
+constexpr int kThreads = 192;
+constexpr long long kWaitCycles = 2000000000ll;   // about a second at B200 clocks
+constexpr int kErrTimeout = 2;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the phase did not complete in time or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - start > kWaitCycles) { *abort_flag = 1; return false; }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c_inner, int c_outer, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *slot, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major operand tile in shared memory, rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
+{
+    uint64_t desc = static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+    desc |= static_cast<uint64_t>(1) << 16;            // leading byte offset (unused for swizzled K-major), 16 B
+    desc |= static_cast<uint64_t>(1024 >> 4) << 32;    // stride byte offset between 8-row groups
+    desc |= static_cast<uint64_t>(1) << 46;            // descriptor version of this architecture
+    desc |= static_cast<uint64_t>(2) << 61;            // 128-byte swizzle
+    return desc;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+enum TcEpilogue { TC_EPI_ADD = 0, TC_EPI_LOGITS = 1, TC_EPI_CROSSKV = 2 };
+
+struct TcParams {
+    int a_rows;          // valid rows of A (output features, or frames)
+    int n_tile;          // rows of B per CTA = MMA N (multiple of 16, at most 256)
+    int k_blocks;        // k-blocks over the whole K
+    int use_lo;          // 1: accumulate the low activation plane as well
+    int rows_fixed;      // >= 0: number of valid B rows; < 0: read it from the decode state
+    // TC_EPI_ADD: out[r * ldo + o] += D[o][r] (+ bias[o] from the CTA of k-split 0)
+    float *out;
+    int ldo;
+    const __nv_bfloat16 *bias;
+    // TC_EPI_LOGITS
+    float *logits_out;                 // [batch, vocab] by utterance or nullptr
+    unsigned long long *keys;          // [rows]
+    const int32_t *active_list;
+    // TC_EPI_CROSSKV: D[frame][feature] -> store [2][H][frame_capacity][64]; bias over features
+    __nv_bfloat16 *cross_store;
+    int frame_capacity, d_model, n_heads;
+    DecState *state;
+};
+
+// grid: x = 128-row tiles of A, y = k-splits, z = N-row tiles of B.  Dynamic shared memory: stage ring + 1024.
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_b_lo, TcParams p, int stages)
+{
+    extern __shared__ uint8_t smem_dyn[];
+    __shared__ __align__(8) uint64_t bar_full[kMaxStages];
+    __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
+    __shared__ __align__(8) uint64_t bar_done;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_rows = p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active;
+    const int row0 = blockIdx.z * p.n_tile;
+    if (EPI != TC_EPI_CROSSKV && row0 >= n_rows) return;          // uniform over the CTA
+    const int a0 = blockIdx.x * kTileM;
+    const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
+    const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
+    const int n_kb = kb_end - kb_begin;
+    if (n_kb <= 0) return;
+
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int b_bytes = p.n_tile * kBlockK * 2;
+    const int planes = p.use_lo ? 2 : 1;
+    const int stage_bytes = kATileBytes + planes * b_bytes;
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < static_cast<uint32_t>(p.n_tile)) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+        mbar_init(&bar_done, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&tmem_slot, tmem_cols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&map_a);
+            prefetch_tensormap(&map_b);
+            if (p.use_lo) prefetch_tensormap(&map_b_lo);
+            int issued = 0;
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % stages;
+                if (i >= stages && !mbar_wait(&bar_empty[s], ((i / stages) - 1) & 1, &abort_flag)) break;
+                uint8_t *st = tiles + static_cast<size_t>(s) * stage_bytes;
+                mbar_expect_tx(&bar_full[s], stage_bytes);
+                const int kc = (kb_begin + i) * kBlockK;
+                tma_load_2d(st, &map_a, kc, a0, &bar_full[s]);
+                tma_load_2d(st + kATileBytes, &map_b, kc, row0, &bar_full[s]);
+                if (p.use_lo) tma_load_2d(st + kATileBytes + b_bytes, &map_b_lo, kc, row0, &bar_full[s]);
+                issued = i + 1;
+            }
+            if (abort_flag) {
+                // give copies that are still in flight a bounded chance to land before the CTA's memory goes away
+                for (int i = (issued > stages ? issued - stages : 0); i < issued; ++i) {
+                    const long long start = clock64();
+                    while (!mbar_try_wait(&bar_full[i % stages], (i / stages) & 1) && clock64() - start < kWaitCycles / 8) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(p.n_tile);
+            bool ok = true;
+            for (int i = 0; i < n_kb && ok; ++i) {
+                const int s = i % stages;
+                ok = mbar_wait(&bar_full[s], (i / stages) & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sa = smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
+                const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + kATileBytes);
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k)
+                    mma_bf16(tmem_base, da + 2 * k, db + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                if (p.use_lo) {
+                    const uint64_t dl = smem_desc_sw128(sa + kATileBytes + b_bytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(tmem_base, da + 2 * k, dl + 2 * k, idesc, 1u);
+                }
+                mma_commit(&bar_empty[s]);      // the stage may be refilled once these MMAs have read it
+            }
+            if (ok) mma_commit(&bar_done);      // accumulator complete
+        }
+    } else {
+        // epilogue warps
+        const int quarter = warp & 3;
+        const bool ok = mbar_wait(&bar_done, 0, &abort_flag);
+        tc_fence_after_sync();
+        if (ok) {
+            const int a_idx = a0 + quarter * 32 + lane;          // row of A this thread owns
+            const bool a_ok = a_idx < p.a_rows;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            if (EPI == TC_EPI_ADD) {
+                const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+                for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(taddr + c0, v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int r = row0 + c0 + j;
+                        if (a_ok && r < n_rows) atomicAdd(p.out + static_cast<size_t>(r) * p.ldo + a_idx, v[j] + bias);
+                    }
+                }
+            } else if (EPI == TC_EPI_LOGITS) {
+                const float bias = (p.bias && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+                for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(taddr + c0, v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int r = row0 + c0 + j;                 // uniform over the warp
+                        if (r >= n_rows) continue;
+                        const float z = v[j] + bias;
+                        if (p.logits_out && a_ok) p.logits_out[static_cast<size_t>(p.active_list[r]) * p.a_rows + a_idx] = z;
+                        unsigned long long key = a_ok ? argmax_key(z, static_cast<uint32_t>(a_idx)) : 0ull;
+#pragma unroll
+                        for (int off = 16; off > 0; off >>= 1) {
+                            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, off);
+                            key = other > key ? other : key;
+                        }
+                        if (lane == 0 && key != 0ull) atomicMax(p.keys + r, key);
+                    }
+                }
+            } else {   // TC_EPI_CROSSKV: this thread owns frame a_idx; columns are features row0 + c
+                for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(taddr + c0, v);
+                    const int o = row0 + c0;                         // 16 consecutive features inside one head
+                    if (!a_ok || o >= 2 * p.d_model) continue;
+                    const int kv = o / p.d_model, c = o % p.d_model, h = c / kHeadDim, e = c % kHeadDim;
+                    uint32_t packed[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float lo = v[2 * j] + (p.bias ? to_f32(p.bias[o + 2 * j]) : 0.f);
+                        const float hi = v[2 * j + 1] + (p.bias ? to_f32(p.bias[o + 2 * j + 1]) : 0.f);
+                        __nv_bfloat162 pair = __floats2bfloat162_rn(lo, hi);
+                        packed[j] = *reinterpret_cast<uint32_t *>(&pair);
+                    }
+                    __nv_bfloat16 *dst = p.cross_store +
+                        ((static_cast<size_t>(kv) * p.n_heads + h) * p.frame_capacity + a_idx) * kHeadDim + e;
+                    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    reinterpret_cast<uint4 *>(dst)[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&p.state->error, kErrTimeout);
+}
+
+}  // namespace tc
+}  // namespace aed

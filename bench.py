@@ -204,6 +204,8 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=list(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--clip-len", type=int, default=0,
+                    help="shorten every forced output length to at most this many tokens (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -228,6 +230,8 @@ def main():
     # Every rank decodes its own batch of the same distribution (utterances are independent: no collective
     # on the data path, weak scaling).
     w = wl.make_workload(args.workload, seed=wl.BASE_SEED + wl._CONFIG_INDEX[args.workload] + 1000 * rank)
+    if args.clip_len > 0:
+        w.dec_lens = np.minimum(w.dec_lens, args.clip_len).astype(np.int32)
     peaks = load_peaks()
     dec = binding.decoder_for_workload(w, device=device)
     enc_host = torch.from_numpy(w.enc).to(dec.tdtype).pin_memory()
@@ -301,7 +305,7 @@ def main():
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, **w.model, "batch_per_gpu": w.batch, "total_enc_frames": int(w.enc_lens.sum()),
-                       "total_out_tokens": n_tok, "decode_steps": Lmax,
+                       "total_out_tokens": n_tok, "decode_steps": Lmax, "clip_len": args.clip_len,
                        "l2": "inputs larger than L2 (weights + K/V stores stream every decode step)",
                        "step": "cross-K/V precompute + greedy decode of one batch"},
             "rtfx": rtfx,

@@ -5,7 +5,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <tuple>
 #include <new>
 #include <string>
 #include <vector>
@@ -134,6 +136,12 @@ struct aed_dec {
     bool use_tc = false;
     int act_planes = 2;
     int sm_count = 148;
+    // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
+    typedef std::tuple<int, int, const void *, const void *> GraphKey;
+    struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
+    std::map<GraphKey, GraphEntry> graphs;
+    cudaStream_t capture_stream = nullptr;
+    bool use_graphs = true;
     // set only while aed_dec_step_static_scratch runs: attention partials go here instead of the workspace
     float *partials_override = nullptr;
 
@@ -661,6 +669,10 @@ extern "C" aed_status_t aed_dec_create(const aed_dec_config_t *config, const aed
         delete dec;
         return s;
     }
+    {
+        const char *no_graph = getenv("AED_DEC_NO_GRAPH");
+        dec->use_graphs = !(no_graph && no_graph[0] == '1');
+    }
     if (config->dtype == AED_DTYPE_BF16) {
         aed_status_t s = tc_setup(dec);
         if (s != AED_OK) {
@@ -788,6 +800,56 @@ extern "C" aed_status_t aed_dec_step_static_scratch(aed_dec_t *dec, const int32_
     return s;
 }
 
+namespace {
+
+aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int32_t *tokens_out, int32_t *out_lens)
+{
+    const Layout &L = dec->lay;
+    if (self_len_ub > dec->cfg.max_dec_len) self_len_ub = dec->cfg.max_dec_len;
+    AED_TRY(launch_build_active(dec, nullptr));
+    const int32_t *tok = dec->at<int32_t>(L.cur_tok);
+    aed_status_t st = dec->use_tc ? forward_step_tc(dec, rows_ub, self_len_ub, tok, nullptr)
+                      : dec->cfg.dtype == AED_DTYPE_BF16 ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tok, nullptr)
+                                                         : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
+    if (st != AED_OK) return st;
+    return launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens);
+}
+
+// Row counts are rounded up to 16, 32, ..., 256 and then to multiples of 256, so that few graphs cover a decode.
+int rows_bucket(int rows)
+{
+    int b = 16;
+    while (b < rows && b < 256) b <<= 1;
+    if (b < rows) b = (rows + 255) / 256 * 256;
+    return b;
+}
+
+// Record one greedy step into a graph on the library's capture stream (nothing runs) and instantiate it.
+aed_status_t capture_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int32_t *tokens_out, int32_t *out_lens,
+                                 aed_dec::GraphEntry *entry)
+{
+    if (!dec->capture_stream)
+        AED_CUDA(dec, cudaStreamCreateWithFlags(&dec->capture_stream, cudaStreamNonBlocking));
+    cudaStream_t user = dec->stream;
+    const int64_t before = dec->launches;
+    AED_CUDA(dec, cudaStreamBeginCapture(dec->capture_stream, cudaStreamCaptureModeThreadLocal));
+    dec->stream = dec->capture_stream;
+    aed_status_t st = enqueue_greedy_step(dec, rows_ub, self_len_ub, tokens_out, out_lens);
+    dec->stream = user;
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(dec->capture_stream, &graph);
+    entry->nodes = dec->launches - before;
+    dec->launches = before;
+    if (st != AED_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+    if (e != cudaSuccess || !graph) return fail(dec, AED_ERR_CUDA, "cudaStreamEndCapture: %s", cudaGetErrorString(e));
+    e = cudaGraphInstantiate(&entry->exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e));
+    return AED_OK;
+}
+
+}  // namespace
+
 extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max_len, int32_t *tokens_out, int32_t *out_lens)
 {
     if (!dec) return AED_ERR_INVALID_ARG;
@@ -812,15 +874,23 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
     AED_TRY(fill_i32(dec, dec->at<int32_t>(L.cur_tok), dec->cfg.bos_id, B));
     AED_TRY(fill_i32(dec, tokens_out, -1, (size_t)B * dec->cfg.max_dec_len));
     AED_TRY(fill_i32(dec, out_lens, 0, B));
-    const bool bf16 = dec->cfg.dtype == AED_DTYPE_BF16;
     for (int s = 0; s < longest; ++s) {
         const int rows_ub = alive[s];
-        AED_TRY(launch_build_active(dec, nullptr));
-        aed_status_t st = dec->use_tc ? forward_step_tc(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr)
-                          : bf16      ? forward_step<__nv_bfloat16>(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr)
-                                      : forward_step<float>(dec, rows_ub, s + 1, dec->at<int32_t>(L.cur_tok), nullptr);
-        if (st != AED_OK) return st;
-        AED_TRY(launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens));
+        if (dec->use_graphs && !dec->profiling) {
+            // grids are sized for the bucket; kernels leave rows beyond the device-side row count alone
+            const int rows_b = rows_bucket(rows_ub), chunks = (s + 1 + kAttnChunk - 1) / kAttnChunk;
+            const aed_dec::GraphKey key(rows_b, chunks, tokens_out, out_lens);
+            auto it = dec->graphs.find(key);
+            if (it == dec->graphs.end()) {
+                aed_dec::GraphEntry entry{};
+                AED_TRY(capture_greedy_step(dec, rows_b, chunks * kAttnChunk, tokens_out, out_lens, &entry));
+                it = dec->graphs.emplace(key, entry).first;
+            }
+            AED_CUDA(dec, cudaGraphLaunch(it->second.exec, dec->stream));
+            dec->launches += it->second.nodes;
+        } else {
+            AED_TRY(enqueue_greedy_step(dec, rows_ub, s + 1, tokens_out, out_lens));
+        }
         dec->steps_issued = s + 1;
     }
     dec->full_steps = dec->cfg.max_dec_len;   // every utterance is retired: further steps are refused
@@ -876,6 +946,8 @@ extern "C" void aed_dec_destroy(aed_dec_t *dec)
 {
     if (!dec) return;
     for (cudaEvent_t e : dec->prof_events) cudaEventDestroy(e);
+    for (auto &g : dec->graphs) cudaGraphExecDestroy(g.second.exec);
+    if (dec->capture_stream) cudaStreamDestroy(dec->capture_stream);
     delete dec;
 }
 

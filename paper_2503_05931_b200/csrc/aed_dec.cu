@@ -269,6 +269,23 @@ aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float
     return AED_OK;
 }
 
+// Attention in one kernel per call (no scratch): one block per (row, head), one warp per 32 positions, at most 16.
+template <typename T, bool kCross, bool kAppend>
+aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const float *q, int ldq, const T *cache,
+                                    int seq_capacity, float *out, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo)
+{
+    ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
+    int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
+    if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
+    if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
+    attn_fused_kernel<T, kCross, kAppend><<<rows_ub * dec->cfg.n_heads, warps * 32, 0, dec->stream>>>(
+        dec->state(), dec->at<int32_t>(dec->lay.active_list), q, ldq, const_cast<T *>(cache), dec->cfg.n_heads,
+        seq_capacity, dec->at<int32_t>(dec->lay.t_u), dec->at<int32_t>(dec->lay.enc_off),
+        dec->at<int32_t>(dec->lay.enc_len), 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo, dec->cfg.d_model);
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
 #define AED_TRY(expr)                        \
     do {                                     \
         aed_status_t s__ = (expr);           \
@@ -488,16 +505,16 @@ aed_status_t forward_step_tc(aed_dec *dec, int rows_ub, int self_len_ub, const i
         AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln1_g, w.ln1_b, qkv, 3 * d));
         p.out = qkv; p.ldo = 3 * d; p.bias = (const T *)w.b_qkv;
         AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_QKV, m.qkv, 3 * d, d, false, rows_ub, p));
-        AED_TRY((launch_attention<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len,
-                                                  nullptr, ad_hi, ad_lo)));
+        AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len,
+                                                        nullptr, ad_hi, ad_lo)));
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
         AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_O, m.o, d, d, false, rows_ub, p));
         // cross-attention
         AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln2_g, w.ln2_b, qkv, d));
         p.out = qkv; p.ldo = d; p.bias = (const T *)w.b_q_c;
         AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_QC, m.qc, d, d, false, rows_ub, p));
-        AED_TRY((launch_attention<T, true>(dec, rows_ub, c.max_enc_len, qkv, d, cross, c.max_total_enc_frames, nullptr,
-                                           ad_hi, ad_lo)));
+        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qkv, d, cross, c.max_total_enc_frames,
+                                                        nullptr, ad_hi, ad_lo)));
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
         AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_OC, m.oc, d, d, false, rows_ub, p));
         // feed-forward

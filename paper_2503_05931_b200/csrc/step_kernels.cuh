@@ -343,6 +343,160 @@ attn_partial_kernel(const DecState *state, const int32_t *__restrict__ active_li
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------------------
+// Single-pass attention for one (row, head) per block: no scratch, no second kernel.  Warp w takes the
+// 32-position chunks w, w + n_warps, ...; within a chunk every lane first issues all of its key loads (8
+// independent 128-bit loads in flight per lane), reduces the scores with shuffles, then issues all value loads.
+// Warps keep a running (max, sum, accumulator) and are merged through shared memory at the end.
+// Lanes: 8 dimension groups (8 head dimensions each) x 4 position groups.
+//   kAppend (self-attention): q row is [q | k | v]; k and v of the new position are stored first.
+//   Output: fp32 [row, d] (out) and/or bf16 high/low planes (out_hi/out_lo), whichever pointers are non-null.
+// ------------------------------------------------------------------------------------------------------------
+template <typename CT> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+    uint4 v;
+    __device__ __forceinline__ void load(const __nv_bfloat16 *p) { v = *reinterpret_cast<const uint4 *>(p); }
+    __device__ __forceinline__ void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
+    __device__ __forceinline__ void get(float (&f)[8]) const
+    {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+    }
+};
+template <> struct Raw8<float> {
+    float4 a, b;
+    __device__ __forceinline__ void load(const float *p) { a = *reinterpret_cast<const float4 *>(p); b = *reinterpret_cast<const float4 *>(p + 4); }
+    __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+    __device__ __forceinline__ void get(float (&f)[8]) const
+    { f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w; }
+};
+
+constexpr int kFusedChunk = 32;
+constexpr int kFusedMaxWarps = 16;
+
+template <typename CT, bool kCross, bool kAppend>
+__global__ void __launch_bounds__(kFusedMaxWarps * 32)
+attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list, const float *__restrict__ q, int ldq,
+                  CT *__restrict__ cache, int n_heads, int seq_capacity, const int32_t *__restrict__ t_u,
+                  const int32_t *__restrict__ enc_off, const int32_t *__restrict__ enc_len, float scale,
+                  float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo)
+{
+    __shared__ float sm_m[kFusedMaxWarps], sm_l[kFusedMaxWarps];
+    __shared__ float sm_acc[kFusedMaxWarps][kHeadDim];
+    const int rh = blockIdx.x;
+    const int r = rh / n_heads, h = rh % n_heads;
+    if (r >= state->n_active) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    const int u = active_list[r];
+    const int len = kCross ? enc_len[u] : t_u[u] + 1;
+    const CT *kbase, *vbase;
+    if (kCross) {
+        kbase = cache + ((size_t)(0 * n_heads + h) * seq_capacity + enc_off[u]) * kHeadDim;
+        vbase = cache + ((size_t)(1 * n_heads + h) * seq_capacity + enc_off[u]) * kHeadDim;
+    } else {
+        kbase = cache + (((size_t)u * 2 + 0) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
+        vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
+    }
+    const int dg = lane & 7, pg = lane >> 3;
+    if (kAppend && !kCross) {
+        if (warp == 0 && lane < 16) {
+            const int kv = lane >> 3, d_model = n_heads * kHeadDim;
+            float nv[8];
+            load8(q + (size_t)r * ldq + (1 + kv) * d_model + h * kHeadDim + dg * 8, nv);
+            CT *dst = const_cast<CT *>(kv ? vbase : kbase) + (size_t)(len - 1) * kHeadDim + dg * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = from_f32<CT>(nv[i]);
+        }
+        __syncthreads();
+    }
+    float qv[8];
+    load8(q + (size_t)r * ldq + h * kHeadDim + dg * 8, qv);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qv[i] *= scale;
+
+    float m = -INFINITY, l = 0.f, acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int p0 = warp * kFusedChunk; p0 < len; p0 += n_warps * kFusedChunk) {
+        Raw8<CT> raw[8];
+        float s[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int p = p0 + i * 4 + pg;
+            if (p < len) raw[i].load(kbase + (size_t)p * kHeadDim + dg * 8); else raw[i].zero();
+        }
+        float cmax = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float kf[8], d = 0.f;
+            raw[i].get(kf);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) d = fmaf(qv[j], kf[j], d);
+            d += __shfl_xor_sync(0xffffffffu, d, 1);
+            d += __shfl_xor_sync(0xffffffffu, d, 2);
+            d += __shfl_xor_sync(0xffffffffu, d, 4);
+            s[i] = (p0 + i * 4 + pg < len) ? d : -INFINITY;
+            cmax = fmaxf(cmax, s[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int p = p0 + i * 4 + pg;
+            if (p < len) raw[i].load(vbase + (size_t)p * kHeadDim + dg * 8); else raw[i].zero();
+        }
+        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
+        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));     // chunk max, uniform over the warp, finite
+        const float m_new = fmaxf(m, cmax);
+        const float corr = expf(m - m_new);
+        l *= corr;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] *= corr;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float pr = expf(s[i] - m_new);      // exp(-inf) = 0 for positions past the end
+            float vf[8];
+            raw[i].get(vf);
+            l += pr;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = fmaf(pr, vf[j], acc[j]);
+        }
+        m = m_new;
+    }
+    // sum the 4 position groups (they share m)
+    l += __shfl_xor_sync(0xffffffffu, l, 8);
+    l += __shfl_xor_sync(0xffffffffu, l, 16);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 8);
+        acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 16);
+    }
+    if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+    if (pg == 0) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sm_acc[warp][dg * 8 + j] = acc[j];
+    }
+    __syncthreads();
+    if (threadIdx.x < kHeadDim) {
+        float big = -INFINITY;
+        for (int w = 0; w < n_warps; ++w) big = fmaxf(big, sm_m[w]);
+        float lsum = 0.f, a = 0.f;
+        for (int w = 0; w < n_warps; ++w) {
+            const float wgt = (sm_m[w] == -INFINITY) ? 0.f : expf(sm_m[w] - big);
+            lsum = fmaf(sm_l[w], wgt, lsum);
+            a = fmaf(sm_acc[w][threadIdx.x], wgt, a);
+        }
+        const float o = a / lsum;
+        const size_t off = (size_t)r * ldo + h * kHeadDim + threadIdx.x;
+        if (out) out[off] = o;
+        if (out_hi) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(o);
+            out_hi[off] = hi;
+            out_lo[off] = __float2bfloat16_rn(o - __bfloat162float(hi));
+        }
+    }
+}
+
 // Merge the chunk partials of each (row, head): one warp per pair, 2 head dimensions per lane.
 template <bool kCross>
 __global__ void __launch_bounds__(128)

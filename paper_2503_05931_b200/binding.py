@@ -13,7 +13,7 @@ from typing import Dict, Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libaed_dec.so")
+LIB_PATH = os.environ.get("AED_DEC_LIB") or os.path.join(_HERE, "libaed_dec.so")   # AED_DEC_LIB: debug builds
 
 AED_OK, AED_ERR_INVALID_ARG, AED_ERR_CAPACITY, AED_ERR_STATE = 0, -1, -2, -3
 AED_ERR_CUDA, AED_ERR_TIMEOUT, AED_ERR_UNSUPPORTED = -4, -5, -6

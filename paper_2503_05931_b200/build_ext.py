@@ -25,6 +25,13 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > built for p in deps)
 
 
+def build_trace() -> str:
+    """Debug build with device-side start-time stamps in every step kernel (libaed_dec_trace.so)."""
+    out = os.path.join(_HERE, "libaed_dec_trace.so")
+    subprocess.run([os.environ.get("NVCC", "nvcc")] + NVCC_FLAGS + ["-DAED_TRACE", "-o", out] + _sources(), check=True)
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile csrc/*.cu into libaed_dec.so next to this file; returns its path."""
     if not force and not _stale():

@@ -84,6 +84,9 @@ Layout make_layout(const aed_dec_config_t &c)
     L.pe = take((size_t)c.max_dec_len * d * 4);
     L.keys = take(B * 8);
     L.state = take(sizeof(DecState));
+#ifdef AED_TRACE
+    take(sizeof(TraceBuf));       // must directly follow the state (see trace_begin)
+#endif
     L.t_u = take(B * 4);
     L.retired = take(B * 4);
     L.active_list = take(B * 4);
@@ -136,6 +139,7 @@ struct aed_dec {
     bool use_tc = false;
     int act_planes = 2;
     int sm_count = 148;
+    int tc_target_ctas = 64;
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
     struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -275,9 +279,11 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
                                     int seq_capacity, float *out, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo)
 {
     ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
+    // Few warps per block, each looping over its chunks: registers are reserved for every warp of a block, and
+    // with ragged lengths most warps of a block sized for the longest row would sit idle.
     int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
     if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
-    if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
+    if (warps > 4) warps = 4;
     attn_fused_kernel<T, kCross, kAppend><<<rows_ub * dec->cfg.n_heads, warps * 32, 0, dec->stream>>>(
         dec->state(), dec->at<int32_t>(dec->lay.active_list), q, ldq, const_cast<T *>(cache), dec->cfg.n_heads,
         seq_capacity, dec->at<int32_t>(dec->lay.t_u), dec->at<int32_t>(dec->lay.enc_off),
@@ -421,6 +427,8 @@ aed_status_t tc_setup(aed_dec *dec)
     dec->sm_count = sms > 0 ? sms : 148;
     const char *planes = getenv("AED_DEC_ACT_PLANES");
     dec->act_planes = (planes && planes[0] == '1') ? 1 : 2;
+    const char *ctas = getenv("AED_DEC_GEMM_CTAS");
+    if (ctas && atoi(ctas) > 0) dec->tc_target_ctas = atoi(ctas);
     dec->use_tc = true;
     return AED_OK;
 }
@@ -444,7 +452,9 @@ aed_status_t launch_tc_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, 
     const int k_blocks = K / tc::kBlockK;
     int splits = 1;
     if (EPI == tc::TC_EPI_ADD) {
-        splits = dec->sm_count / (m_tiles * row_tiles);
+        // About 64 CTAs with deep TMA rings already pull the weights at HBM rate; more k-splits only multiply
+        // the red.global traffic of the epilogue (splits x rows x features x 4 bytes).
+        splits = dec->tc_target_ctas / (m_tiles * row_tiles);
         if (splits < 1) splits = 1;
         if (splits > k_blocks) splits = k_blocks;
     }
@@ -956,6 +966,23 @@ extern "C" int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, co
     }
     return n;
 }
+
+#ifdef AED_TRACE
+// Debug builds only: copy out the device-side start-time trace (ids and nanosecond stamps) and clear it.
+extern "C" int32_t aed_dec_trace_read(aed_dec_t *dec, int32_t max_events, uint32_t *ids, unsigned long long *t_ns)
+{
+    if (!dec) return AED_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(dec->stream) != cudaSuccess) return AED_ERR_CUDA;
+    static TraceBuf host;
+    char *src = dec->ws + dec->lay.state + 256;
+    if (cudaMemcpy(&host, src, sizeof host, cudaMemcpyDeviceToHost) != cudaSuccess) return AED_ERR_CUDA;
+    cudaMemset(src, 0, 8);
+    int n = host.count < (1u << 16) ? (int)host.count : (1 << 16);
+    if (n > max_events) n = max_events;
+    for (int i = 0; i < n; ++i) { ids[i] = host.ev[i].id; t_ns[i] = host.ev[i].t_ns; }
+    return n;
+}
+#endif
 
 extern "C" int64_t aed_dec_launch_count(const aed_dec_t *dec) { return dec ? dec->launches : 0; }
 

@@ -18,6 +18,41 @@ struct DecState {
     int32_t pad;
 };
 
+// Optional device-side timeline (debug builds with -DAED_TRACE): block 0 of every traced kernel stamps its start
+// time.  The buffer follows the decode state in the workspace.
+struct TraceBuf {
+    uint32_t count, pad;
+    struct { uint32_t id, pad; unsigned long long t_ns; } ev[1 << 16];
+};
+#ifdef AED_TRACE
+__device__ __forceinline__ void trace_begin(const DecState *state, uint32_t id)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+        TraceBuf *tb = reinterpret_cast<TraceBuf *>(reinterpret_cast<char *>(const_cast<DecState *>(state)) + 256);
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        uint32_t i = atomicAdd(&tb->count, 1u);
+        if (i < (1u << 16)) { tb->ev[i].id = id; tb->ev[i].t_ns = t; }
+    }
+}
+// stamp from whichever thread of block 0 calls it
+__device__ __forceinline__ void trace_mark(const DecState *state, uint32_t id)
+{
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+        TraceBuf *tb = reinterpret_cast<TraceBuf *>(reinterpret_cast<char *>(const_cast<DecState *>(state)) + 256);
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        uint32_t i = atomicAdd(&tb->count, 1u);
+        if (i < (1u << 16)) { tb->ev[i].id = id; tb->ev[i].t_ns = t; }
+    }
+}
+#define AED_TRACE_BEGIN(state, id) trace_begin(state, id)
+#define AED_TRACE_MARK(state, id) trace_mark(state, id)
+#else
+#define AED_TRACE_BEGIN(state, id) ((void)0)
+#define AED_TRACE_MARK(state, id) ((void)0)
+#endif
+
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 

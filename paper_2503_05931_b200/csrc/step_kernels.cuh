@@ -15,6 +15,7 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
                                     const int32_t *__restrict__ t_u, int max_dec_len,
                                     int32_t *__restrict__ active_list, DecState *state)
 {
+    AED_TRACE_BEGIN(state, 1);
     __shared__ int warp_counts[32];
     __shared__ int base;
     if (threadIdx.x == 0) base = 0;
@@ -61,6 +62,7 @@ __global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ 
                              const T *__restrict__ embed, const float *__restrict__ pe, int d, int vocab, float scale,
                              float *__restrict__ x)
 {
+    AED_TRACE_BEGIN(state, 2);
     int r = blockIdx.x;
     if (r >= state->n_active) return;
     int u = active_list[r];
@@ -383,6 +385,7 @@ attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list
                   const int32_t *__restrict__ enc_off, const int32_t *__restrict__ enc_len, float scale,
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo)
 {
+    AED_TRACE_BEGIN(state, 3);
     __shared__ float sm_m[kFusedMaxWarps], sm_l[kFusedMaxWarps];
     __shared__ float sm_acc[kFusedMaxWarps][kHeadDim];
     const int rh = blockIdx.x;
@@ -569,6 +572,7 @@ __global__ void layernorm_planes_kernel(const DecState *state, const float *__re
                                         float eps, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo,
                                         float *__restrict__ zero_buf, int zero_cols)
 {
+    AED_TRACE_BEGIN(state, 4);
     int r = blockIdx.x;
     if (r >= state->n_active) return;
     __shared__ float red[32];
@@ -620,6 +624,7 @@ __global__ void layernorm_planes_kernel(const DecState *state, const float *__re
 __global__ void relu_planes_kernel(const DecState *state, const float *__restrict__ hid, int f,
                                    __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo)
 {
+    AED_TRACE_BEGIN(state, 5);
     int r = blockIdx.y;
     if (r >= state->n_active) return;
     int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
@@ -649,6 +654,7 @@ __global__ void finish_step_kernel(DecState *state, const int32_t *__restrict__ 
                                    const int32_t *__restrict__ max_len, int eos_id,
                                    int32_t *__restrict__ tokens_out, int tokens_ld, int32_t *__restrict__ out_lens)
 {
+    AED_TRACE_BEGIN(state, 6);
     int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= state->n_active) return;
     int u = active_list[r];

@@ -164,10 +164,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
+    AED_TRACE_BEGIN(p.state, 16 + EPI);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_rows = p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active;
     const int row0 = blockIdx.z * p.n_tile;
-    if (EPI != TC_EPI_CROSSKV && row0 >= n_rows) return;          // uniform over the CTA
+    // Only row tiles after the first can be empty; the first one skips this read so that set-up and the first
+    // loads do not wait on it (the epilogue reads the row count when it needs it).
+    if (EPI != TC_EPI_CROSSKV && blockIdx.z > 0 && row0 >= (p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active)) return;
     const int a0 = blockIdx.x * kTileM;
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
@@ -192,6 +194,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
+    if (threadIdx.x == 0) AED_TRACE_MARK(p.state, 32);      // set-up done
 
     if (warp == 0) {
         if (lane == 0) {
@@ -226,6 +229,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int s = i % stages;
                 ok = mbar_wait(&bar_full[s], (i / stages) & 1, &abort_flag);
                 if (!ok) break;
+                if (i == 0) AED_TRACE_MARK(p.state, 33);    // first operands landed
                 tc_fence_after_sync();
                 const uint32_t sa = smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
                 const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + kATileBytes);
@@ -244,8 +248,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // epilogue warps
         const int quarter = warp & 3;
+        const int n_rows = p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active;
         const bool ok = mbar_wait(&bar_done, 0, &abort_flag);
         tc_fence_after_sync();
+        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 34);  // accumulator complete
         if (ok) {
             const int a_idx = a0 + quarter * 32 + lane;          // row of A this thread owns
             const bool a_ok = a_idx < p.a_rows;
@@ -272,12 +278,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (r >= n_rows) continue;
                         const float z = v[j] + bias;
                         if (p.logits_out && a_ok) p.logits_out[static_cast<size_t>(p.active_list[r]) * p.a_rows + a_idx] = z;
-                        unsigned long long key = a_ok ? argmax_key(z, static_cast<uint32_t>(a_idx)) : 0ull;
-#pragma unroll
-                        for (int off = 16; off > 0; off >>= 1) {
-                            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, off);
-                            key = other > key ? other : key;
-                        }
+                        // warp maximum of the order-preserving key, then the lowest lane that attains it
+                        const uint32_t k32 = a_ok ? float_order_key(z) : 0u;
+                        const uint32_t kmax = __reduce_max_sync(0xffffffffu, k32);
+                        const uint32_t winners = __ballot_sync(0xffffffffu, k32 == kmax);
+                        const uint32_t best = a0 + quarter * 32 + (__ffs(winners) - 1);
+                        const unsigned long long key =
+                            kmax ? ((static_cast<unsigned long long>(kmax) << 32) | (0xFFFFFFFFu - best)) : 0ull;
                         if (lane == 0 && key != 0ull) atomicMax(p.keys + r, key);
                     }
                 }
@@ -304,6 +311,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     }
+    if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 35);      // epilogue issued
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {

@@ -24,6 +24,15 @@ thread_local std::string g_create_error;
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Row counts are rounded up to 16, 32, ..., 256 and then to multiples of 256, so that few graphs cover a decode.
+int rows_bucket(int rows)
+{
+    int b = 16;
+    while (b < rows && b < 256) b <<= 1;
+    if (b < rows) b = (rows + 255) / 256 * 256;
+    return b;
+}
+
 struct LayerWeights {
     const void *ln1_g, *ln1_b, *w_qkv, *b_qkv, *w_o, *b_o;
     const void *ln2_g, *ln2_b, *w_q_c, *b_q_c, *w_kv_c, *b_kv_c, *w_o_c, *b_o_c;
@@ -33,7 +42,7 @@ struct LayerWeights {
 // Byte offsets of every region of the caller's workspace.
 struct Layout {
     size_t self_cache, cross_store, x, act, qkv, hid, partials, pe, keys, state;
-    size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, total;
+    size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, row_info, total;
     size_t self_layer_elems, cross_layer_elems;
     int max_chunks;
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
@@ -94,6 +103,7 @@ Layout make_layout(const aed_dec_config_t &c)
     L.enc_off = take((B + 1) * 4);
     L.enc_len = take(B * 4);
     L.max_len = take(B * 4);
+    L.row_info = take((size_t)rows_bucket(c.max_batch) * 16);      // grids are sized for the bucket
     L.rows_cap = (int)align_up(B, 16);
     if (c.dtype == AED_DTYPE_BF16) {
         L.actd_hi = take((size_t)L.rows_cap * d * 2);
@@ -283,11 +293,10 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     // with ragged lengths most warps of a block sized for the longest row would sit idle.
     int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
     if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
-    if (warps > 4) warps = 4;
+    if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
     attn_fused_kernel<T, kCross, kAppend><<<rows_ub * dec->cfg.n_heads, warps * 32, 0, dec->stream>>>(
-        dec->state(), dec->at<int32_t>(dec->lay.active_list), q, ldq, const_cast<T *>(cache), dec->cfg.n_heads,
-        seq_capacity, dec->at<int32_t>(dec->lay.t_u), dec->at<int32_t>(dec->lay.enc_off),
-        dec->at<int32_t>(dec->lay.enc_len), 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo, dec->cfg.d_model);
+        dec->state(), dec->at<int4>(dec->lay.row_info), q, ldq, const_cast<T *>(cache), dec->cfg.n_heads,
+        seq_capacity, 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo, dec->cfg.d_model);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -608,7 +617,9 @@ aed_status_t launch_build_active(aed_dec *dec, const uint8_t *mask)
     ProfScope ps(dec, KF_BOOKKEEPING);
     build_active_kernel<<<1, 1024, 0, dec->stream>>>(dec->batch, mask, dec->at<int32_t>(L.retired),
                                                      dec->at<int32_t>(L.t_u), dec->cfg.max_dec_len,
-                                                     dec->at<int32_t>(L.active_list), dec->state());
+                                                     dec->at<int32_t>(L.active_list), dec->state(),
+                                                     dec->at<int32_t>(L.enc_len), dec->at<int32_t>(L.enc_off),
+                                                     dec->at<int4>(L.row_info), rows_bucket(dec->cfg.max_batch));
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -840,15 +851,6 @@ aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int
                                                          : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
     if (st != AED_OK) return st;
     return launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens);
-}
-
-// Row counts are rounded up to 16, 32, ..., 256 and then to multiples of 256, so that few graphs cover a decode.
-int rows_bucket(int rows)
-{
-    int b = 16;
-    while (b < rows && b < 256) b <<= 1;
-    if (b < rows) b = (rows + 255) / 256 * 256;
-    return b;
 }
 
 // Record one greedy step into a graph on the library's capture stream (nothing runs) and instantiate it.

@@ -11,9 +11,13 @@ namespace aed {
 // An utterance takes part if it is not retired, the caller's mask (if any) selects it, and its self-attention
 // cache still has room; a selected utterance with a full cache raises the sticky error instead of overflowing.
 // ------------------------------------------------------------------------------------------------------------
+// It also fills the row table: row_info[r] = (utterance, t_u, encoder length, encoder offset) for every compact
+// row, and utterance -1 for the slots past the last row, so that a kernel needs one 16-byte load per row.
 __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask, const int32_t *__restrict__ retired,
                                     const int32_t *__restrict__ t_u, int max_dec_len,
-                                    int32_t *__restrict__ active_list, DecState *state)
+                                    int32_t *__restrict__ active_list, DecState *state,
+                                    const int32_t *__restrict__ enc_len, const int32_t *__restrict__ enc_off,
+                                    int4 *__restrict__ row_info, int row_slots)
 {
     AED_TRACE_BEGIN(state, 1);
     __shared__ int warp_counts[32];
@@ -33,7 +37,11 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
         __syncthreads();
         int before = base;
         for (int w = 0; w < warp; ++w) before += warp_counts[w];
-        if (take) active_list[before + __popc(ballot & ((1u << lane) - 1u))] = u;
+        if (take) {
+            const int slot = before + __popc(ballot & ((1u << lane) - 1u));
+            active_list[slot] = u;
+            row_info[slot] = make_int4(u, t_u[u], enc_len[u], enc_off[u]);
+        }
         __syncthreads();
         if (threadIdx.x == 0) {
             int total = 0;
@@ -43,6 +51,7 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
         __syncthreads();
     }
     if (threadIdx.x == 0) state->n_active = base;
+    for (int r = base + threadIdx.x; r < row_slots; r += blockDim.x) row_info[r] = make_int4(-1, 0, 0, 0);
 }
 
 // Sinusoidal position table PE[t][2i] = sin(t / 10000^(2i/d)), PE[t][2i+1] = cos(same), evaluated in double.
@@ -348,8 +357,8 @@ attn_partial_kernel(const DecState *state, const int32_t *__restrict__ active_li
 
 // ------------------------------------------------------------------------------------------------------------
 // Single-pass attention for one (row, head) per block: no scratch, no second kernel.  Warp w takes the
-// 32-position chunks w, w + n_warps, ...; within a chunk every lane first issues all of its key loads (8
-// independent 128-bit loads in flight per lane), reduces the scores with shuffles, then issues all value loads.
+// 16-position chunks w, w + n_warps, ...; within a chunk every lane issues its 4 key and 4 value loads (128 bits
+// each) together, so one memory latency covers the chunk, then reduces the scores with shuffles.
 // Warps keep a running (max, sum, accumulator) and are merged through shared memory at the end.
 // Lanes: 8 dimension groups (8 head dimensions each) x 4 position groups.
 //   kAppend (self-attention): q row is [q | k | v]; k and v of the new position are stored first.
@@ -375,14 +384,13 @@ template <> struct Raw8<float> {
     { f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w; }
 };
 
-constexpr int kFusedChunk = 32;
-constexpr int kFusedMaxWarps = 16;
+constexpr int kFusedChunk = 16;       // positions per warp and iteration
+constexpr int kFusedMaxWarps = 8;
 
 template <typename CT, bool kCross, bool kAppend>
-__global__ void __launch_bounds__(kFusedMaxWarps * 32)
-attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list, const float *__restrict__ q, int ldq,
-                  CT *__restrict__ cache, int n_heads, int seq_capacity, const int32_t *__restrict__ t_u,
-                  const int32_t *__restrict__ enc_off, const int32_t *__restrict__ enc_len, float scale,
+__global__ void __launch_bounds__(kFusedMaxWarps * 32, 4)
+attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ q, int ldq,
+                  CT *__restrict__ cache, int n_heads, int seq_capacity, float scale,
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo)
 {
     AED_TRACE_BEGIN(state, 3);
@@ -390,14 +398,15 @@ attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list
     __shared__ float sm_acc[kFusedMaxWarps][kHeadDim];
     const int rh = blockIdx.x;
     const int r = rh / n_heads, h = rh % n_heads;
-    if (r >= state->n_active) return;
+    const int4 ri = row_info[r];                       // (utterance, t_u, encoder length, encoder offset)
+    if (ri.x < 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
-    const int u = active_list[r];
-    const int len = kCross ? enc_len[u] : t_u[u] + 1;
+    const int u = ri.x;
+    const int len = kCross ? ri.z : ri.y + 1;
     const CT *kbase, *vbase;
     if (kCross) {
-        kbase = cache + ((size_t)(0 * n_heads + h) * seq_capacity + enc_off[u]) * kHeadDim;
-        vbase = cache + ((size_t)(1 * n_heads + h) * seq_capacity + enc_off[u]) * kHeadDim;
+        kbase = cache + ((size_t)(0 * n_heads + h) * seq_capacity + ri.w) * kHeadDim;
+        vbase = cache + ((size_t)(1 * n_heads + h) * seq_capacity + ri.w) * kHeadDim;
     } else {
         kbase = cache + (((size_t)u * 2 + 0) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
         vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
@@ -423,18 +432,20 @@ attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
     for (int p0 = warp * kFusedChunk; p0 < len; p0 += n_warps * kFusedChunk) {
-        Raw8<CT> raw[8];
-        float s[8];
+        Raw8<CT> rk[4], rv[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {          // keys and values of the chunk are requested together
             const int p = p0 + i * 4 + pg;
-            if (p < len) raw[i].load(kbase + (size_t)p * kHeadDim + dg * 8); else raw[i].zero();
+            if (p < len) {
+                rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
+                rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
+            } else { rk[i].zero(); rv[i].zero(); }
         }
-        float cmax = -INFINITY;
+        float s[4], cmax = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {
             float kf[8], d = 0.f;
-            raw[i].get(kf);
+            rk[i].get(kf);
 #pragma unroll
             for (int j = 0; j < 8; ++j) d = fmaf(qv[j], kf[j], d);
             d += __shfl_xor_sync(0xffffffffu, d, 1);
@@ -442,11 +453,6 @@ attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list
             d += __shfl_xor_sync(0xffffffffu, d, 4);
             s[i] = (p0 + i * 4 + pg < len) ? d : -INFINITY;
             cmax = fmaxf(cmax, s[i]);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int p = p0 + i * 4 + pg;
-            if (p < len) raw[i].load(vbase + (size_t)p * kHeadDim + dg * 8); else raw[i].zero();
         }
         cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
         cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));     // chunk max, uniform over the warp, finite
@@ -456,10 +462,10 @@ attn_fused_kernel(const DecState *state, const int32_t *__restrict__ active_list
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] *= corr;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 4; ++i) {
             const float pr = expf(s[i] - m_new);      // exp(-inf) = 0 for positions past the end
             float vf[8];
-            raw[i].get(vf);
+            rv[i].get(vf);
             l += pr;
 #pragma unroll
             for (int j = 0; j < 8; ++j) acc[j] = fmaf(pr, vf[j], acc[j]);

@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "step_kernels.cuh"
 #include "tc_gemm.cuh"
+#include "step_gemm.cuh"
 
 using namespace aed;
 
@@ -47,6 +48,8 @@ struct Layout {
     int max_chunks;
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
     size_t actd_hi, actd_lo, actf_hi, actf_lo;
+    size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
+    size_t fold_layer_floats;
     int rows_cap;
 };
 
@@ -110,6 +113,10 @@ Layout make_layout(const aed_dec_config_t &c)
         L.actd_lo = take((size_t)L.rows_cap * d * 2);
         L.actf_hi = take((size_t)L.rows_cap * F * 2);
         L.actf_lo = take((size_t)L.rows_cap * F * 2);
+        L.fold_layer_floats = 2 * (3 * d + d + F);       // c1 | c2 for qkv, then for cross-q, then for ffn1
+        L.fold_c = take(L.fold_layer_floats * c.n_layers * 4);
+        L.ln_stats = take((size_t)3 * rows_bucket(c.max_batch) * 8);
+        L.qc = take(B * d * 4);
     }
     L.total = off;
     return L;
@@ -149,7 +156,9 @@ struct aed_dec {
     bool use_tc = false;
     int act_planes = 2;
     int sm_count = 148;
-    int tc_target_ctas = 64;
+    int tc_target_ctas = 128;
+    bool use_pdl = true;
+    bool use_fused = true;
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
     struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -283,20 +292,32 @@ aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float
     return AED_OK;
 }
 
-// Attention in one kernel per call (no scratch): one block per (row, head), one warp per 32 positions, at most 16.
+// Attention in one kernel per call (no scratch): one block per (row, head), one warp per 16 positions, at most 8.
+// The kernel starts with a programmatic-dependency wait, so it may be launched ahead of its predecessor's end.
 template <typename T, bool kCross, bool kAppend>
 aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const float *q, int ldq, const T *cache,
-                                    int seq_capacity, float *out, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo)
+                                    int seq_capacity, float *out, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
+                                    const float2 *ln_stats = nullptr, const float *ln_c1 = nullptr,
+                                    const float *ln_c2 = nullptr, bool pdl = false)
 {
     ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
-    // Few warps per block, each looping over its chunks: registers are reserved for every warp of a block, and
-    // with ragged lengths most warps of a block sized for the longest row would sit idle.
     int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
     if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
     if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
-    attn_fused_kernel<T, kCross, kAppend><<<rows_ub * dec->cfg.n_heads, warps * 32, 0, dec->stream>>>(
-        dec->state(), dec->at<int4>(dec->lay.row_info), q, ldq, const_cast<T *>(cache), dec->cfg.n_heads,
-        seq_capacity, 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo, dec->cfg.d_model);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(rows_ub * dec->cfg.n_heads);
+    cfg.blockDim = dim3(warps * 32);
+    cfg.stream = dec->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_fused_kernel<T, kCross, kAppend>, (const DecState *)dec->state(),
+                                       (const int4 *)dec->at<int4>(dec->lay.row_info), q, ldq, const_cast<T *>(cache),
+                                       dec->cfg.n_heads, seq_capacity, 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo,
+                                       dec->cfg.d_model, ln_stats, ln_c1, ln_c2);
+    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -434,6 +455,31 @@ aed_status_t tc_setup(aed_dec *dec)
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
     dec->sm_count = sms > 0 ? sms : 148;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_GAMMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_LN_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
+    // LayerNorm-fold constants of every layer
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
+        typedef __nv_bfloat16 T;
+        sg::ln_fold_constants_kernel<<<(3 * d + 7) / 8, 256, 0, dec->stream>>>((const T *)w.w_qkv, (const T *)w.ln1_g, (const T *)w.ln1_b,
+                                                                               (const T *)w.b_qkv, 3 * (int)d, (int)d, fc, fc + 3 * d);
+        sg::ln_fold_constants_kernel<<<(d + 7) / 8, 256, 0, dec->stream>>>((const T *)w.w_q_c, (const T *)w.ln2_g, (const T *)w.ln2_b,
+                                                                           (const T *)w.b_q_c, (int)d, (int)d, fc + 6 * d, fc + 7 * d);
+        sg::ln_fold_constants_kernel<<<(F + 7) / 8, 256, 0, dec->stream>>>((const T *)w.w_ff1, (const T *)w.ln3_g, (const T *)w.ln3_b,
+                                                                           (const T *)w.b_ff1, (int)F, (int)d, fc + 8 * d, fc + 8 * d + F);
+        dec->launches += 3;
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "fold constants: %s", cudaGetErrorString(e));
+    {
+        const char *v = getenv("AED_DEC_NO_PDL");
+        dec->use_pdl = !(v && v[0] == '1');
+        v = getenv("AED_DEC_NO_FUSED");
+        dec->use_fused = !(v && v[0] == '1');
+    }
     const char *planes = getenv("AED_DEC_ACT_PLANES");
     dec->act_planes = (planes && planes[0] == '1') ? 1 : 2;
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
@@ -555,6 +601,130 @@ aed_status_t forward_step_tc(aed_dec *dec, int rows_ub, int self_len_ub, const i
     p.keys = dec->at<unsigned long long>(L.keys);
     p.active_list = active_list;
     AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, p));
+    return AED_OK;
+}
+
+
+// ---- fused step (bf16 mode): 8 kernels per layer, chained with programmatic dependent launch -------------------
+
+struct FusedGemm {
+    const CUtensorMap *map;
+    int M, K, mode;
+};
+
+template <int MODE>
+aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, int M, int K, int rows_ub,
+                              sg::StepGemmParams p)
+{
+    ProfScope ps(dec, family);
+    const int ni = tc_n_index(rows_ub), n_tile = 16 << ni;
+    const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
+    const int k_blocks = K / tc::kBlockK;
+    const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2;
+    int kb_cta = kTcSmemBudget / stage_bytes;
+    if (kb_cta > sg::kMaxKb) kb_cta = sg::kMaxKb;
+    int splits = (k_blocks + kb_cta - 1) / kb_cta;
+    const int want = dec->tc_target_ctas / (m_tiles * row_tiles);
+    if (want > splits) splits = want;
+    if (splits > k_blocks) splits = k_blocks;
+    const int kb_max = (k_blocks + splits - 1) / splits;
+    p.a_rows = M;
+    p.k_blocks = k_blocks;
+    p.n_tile = n_tile;
+    p.state = dec->state();
+    p.eps = dec->cfg.ln_eps;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(m_tiles, splits, row_tiles);
+    cfg.blockDim = dim3(sg::kSgThreads);
+    cfg.dynamicSmemBytes = (size_t)kb_max * stage_bytes + 1024;
+    cfg.stream = dec->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, p);
+    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "projection launch: %s", cudaGetErrorString(e));
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
+aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, const int32_t *tokens, float *logits_out)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const int d = c.d_model, F = c.d_ffn, V = c.vocab;
+    float *x = dec->at<float>(L.x), *qkv = dec->at<float>(L.qkv), *hid = dec->at<float>(L.hid), *att = dec->at<float>(L.act);
+    float *qc = dec->at<float>(L.qc);
+    float2 *stats = dec->at<float2>(L.ln_stats);
+    const int stats_stride = rows_bucket(c.max_batch);
+    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
+    {
+        ProfScope ps(dec, KF_EMBED);
+        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
+        AED_LAUNCHED(dec);
+    }
+    const bool pdl = dec->use_pdl;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        const aed_dec::TcLayerMaps &m = dec->tc_layers[l];
+        T *self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
+        const T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+        const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
+        const float *c1_qkv = fc, *c2_qkv = fc + 3 * d, *c1_qc = fc + 6 * d, *c2_qc = fc + 7 * d, *c1_ff = fc + 8 * d,
+                    *c2_ff = fc + 8 * d + F;
+        sg::StepGemmParams p{};
+        // 1. [q | k | v] raw = (gamma1 * x) Wqkv^T ; side: LN1 statistics of x, clear the cross-query rows
+        p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln1_g;
+        p.out = qkv; p.ldo = 3 * d; p.bias = nullptr;
+        p.stats_src = x; p.stats_out = stats; p.stats_d = d;
+        p.zero_buf = qc; p.zero_cols = d;
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, 3 * d, d, rows_ub, p));
+        // 2. self-attention (applies LN1 to q, k, v; appends k, v)
+        AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
+                                                        nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
+        // 3. x += att Wo^T + bo ; side: clear the FFN hidden rows
+        p = sg::StepGemmParams{};
+        p.src = att; p.ld_src = d;
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
+        p.zero_buf = hid; p.zero_cols = F;
+        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, d, d, rows_ub, p));
+        // 4. q' raw = (gamma2 * x) Wqc^T ; side: LN2 statistics
+        p = sg::StepGemmParams{};
+        p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln2_g;
+        p.out = qc; p.ldo = d;
+        p.stats_src = x; p.stats_out = stats + stats_stride; p.stats_d = d;
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QC, m.qc, d, d, rows_ub, p));
+        // 5. cross-attention
+        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
+                                                        nullptr, nullptr, stats + stats_stride, c1_qc, c2_qc, pdl)));
+        // 6. x += att Woc^T + boc ; side: clear the [q | k | v] rows for the next layer
+        p = sg::StepGemmParams{};
+        p.src = att; p.ld_src = d;
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
+        p.zero_buf = qkv; p.zero_cols = 3 * d;
+        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_OC, m.oc, d, d, rows_ub, p));
+        // 7. hidden raw = (gamma3 * x) W1^T ; side: LN3 statistics
+        p = sg::StepGemmParams{};
+        p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln3_g;
+        p.out = hid; p.ldo = F;
+        p.stats_src = x; p.stats_out = stats + 2 * stats_stride; p.stats_d = d;
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, F, d, rows_ub, p));
+        // 8. x += relu(LN3-corrected hidden) W2^T + b2
+        p = sg::StepGemmParams{};
+        p.src = hid; p.ld_src = F; p.c1 = c1_ff; p.c2 = c2_ff; p.stats_in = stats + 2 * stats_stride;
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
+        AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, d, F, rows_ub, p));
+    }
+    AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
+    tc::TcParams tp{};
+    tp.bias = (const T *)dec->b_out;
+    tp.logits_out = logits_out;
+    tp.keys = dec->at<unsigned long long>(L.keys);
+    tp.active_list = active_list;
+    AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, tp));
     return AED_OK;
 }
 
@@ -773,7 +943,7 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_build_active(dec, active));
     const int rows_ub = dec->batch;
     const int self_len_ub = dec->steps_issued + 1 < dec->cfg.max_dec_len ? dec->steps_issued + 1 : dec->cfg.max_dec_len;
-    aed_status_t s = dec->use_tc ? forward_step_tc(dec, rows_ub, self_len_ub, tokens_in, logits_out)
+    aed_status_t s = dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out) : forward_step_tc(dec, rows_ub, self_len_ub, tokens_in, logits_out))
                      : dec->cfg.dtype == AED_DTYPE_BF16
                          ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tokens_in, logits_out)
                          : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
@@ -846,7 +1016,7 @@ aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int
     if (self_len_ub > dec->cfg.max_dec_len) self_len_ub = dec->cfg.max_dec_len;
     AED_TRY(launch_build_active(dec, nullptr));
     const int32_t *tok = dec->at<int32_t>(L.cur_tok);
-    aed_status_t st = dec->use_tc ? forward_step_tc(dec, rows_ub, self_len_ub, tok, nullptr)
+    aed_status_t st = dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr) : forward_step_tc(dec, rows_ub, self_len_ub, tok, nullptr))
                       : dec->cfg.dtype == AED_DTYPE_BF16 ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tok, nullptr)
                                                          : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
     if (st != AED_OK) return st;

@@ -1,0 +1,285 @@
+// Decode-step projection on tensor cores with the activation operand built in the kernel.
+//
+//   out[r, o] += sum_k B(r, k) * W[o, k]      (+ bias[o] from the CTA of the first k-split)
+//
+// W tiles (128 output features x 64 k, bf16) arrive by TMA; they do not depend on earlier kernels, so they are
+// requested before the programmatic-dependency wait and stream in while the previous kernel drains.
+// The activation tile B is produced by four warps straight from fp32 sources into the 128-byte-swizzled layout the
+// MMA reads, as a bf16 high plane and a bf16 low plane (value - high), with one of three transforms fused:
+//   B_PLAIN    B = src                                   (attention output -> output projection)
+//   B_GAMMA    B = gamma[k] * src                        (LayerNorm folded into the projection, see below)
+//   B_LN_RELU  B = relu(rstd_r * (src - mean_r * c1[k]) + c2[k])   (FFN hidden layer from the folded first GEMM)
+//
+// LayerNorm folding: LN(x) W^T = rstd * ((gamma*x) W^T - mean * c1) + c2 with c1[o] = sum_k gamma_k W[o,k] and
+// c2[o] = sum_k beta_k W[o,k] + b[o].  The GEMM therefore runs on gamma*x without knowing the row statistics;
+// whoever consumes its output applies (mean, rstd).  The statistics themselves are a side job: while the MMAs
+// run, the producer warps of this kernel compute mean and rstd of the rows assigned to their CTA and store
+// them for the consumer.  A second side job clears the fp32 rows a later split-K projection accumulates into.
+//
+// All k-blocks of a CTA are resident at once (at most 4), so there is no ring to recycle.  Waits are bounded.
+#pragma once
+#include "tc_gemm.cuh"
+
+namespace aed {
+namespace sg {
+
+using namespace tc;
+
+constexpr int kMaxKb = 4;             // k-blocks per CTA
+constexpr int kSgThreads = 192;
+
+enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2 };
+
+struct StepGemmParams {
+    int a_rows;                // output features M
+    int k_blocks;              // K / 64
+    int n_tile;                // MMA N: rows per CTA tile (16..256, multiple of 16)
+    // activation source [rows, ld_src] fp32
+    const float *src;
+    int ld_src;
+    const __nv_bfloat16 *gamma;    // B_GAMMA: [K]
+    const float *c1, *c2;          // B_LN_RELU: [K] each
+    const float2 *stats_in;        // B_LN_RELU: (mean, rstd) per row
+    // epilogue
+    float *out;
+    int ldo;
+    const __nv_bfloat16 *bias;     // added by k-split 0, may be null
+    // side job 1: (mean, rstd) of the rows of stats_src [rows, stats_d]
+    const float *stats_src;
+    float2 *stats_out;
+    int stats_d;
+    float eps;
+    // side job 2: clear zero_buf [rows, zero_cols]
+    float *zero_buf;
+    int zero_cols;
+    DecState *state;
+};
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b)
+{
+    __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&p);
+}
+
+// 8 values -> one 16-byte chunk of the high plane and one of the low plane
+__device__ __forceinline__ void split_planes(const float (&y)[8], uint4 &hi, uint4 &lo)
+{
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(y[2 * i]), h1 = __float2bfloat16_rn(y[2 * i + 1]);
+        __nv_bfloat162 hp = __halves2bfloat162(h0, h1);
+        h[i] = *reinterpret_cast<uint32_t *>(&hp);
+        l[i] = pack_bf16(y[2 * i] - __bfloat162float(h0), y[2 * i + 1] - __bfloat162float(h1));
+    }
+    hi = make_uint4(h[0], h[1], h[2], h[3]);
+    lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+// grid: x = 128-feature tiles, y = k-splits, z = row tiles.  Dynamic smem: kb * (16 KB + 2 * n_tile * 128) + 1024.
+template <int MODE>
+__global__ void __launch_bounds__(kSgThreads, 1)
+step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, StepGemmParams p)
+{
+    extern __shared__ uint8_t smem_dyn[];
+    __shared__ __align__(8) uint64_t bar_a[kMaxKb];
+    __shared__ __align__(8) uint64_t bar_b;
+    __shared__ __align__(8) uint64_t bar_done;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ float red_s[4], red_q[4];
+
+    AED_TRACE_BEGIN(p.state, 19);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int a0 = blockIdx.x * kTileM;
+    const int row0 = blockIdx.z * p.n_tile;
+    const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
+    const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
+    const int n_kb = kb_end - kb_begin;          // 1..kMaxKb by construction of the grid
+
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int plane_bytes = p.n_tile * kBlockK * 2;
+    const int stage_bytes = kATileBytes + 2 * plane_bytes;
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < static_cast<uint32_t>(p.n_tile)) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxKb; ++s) mbar_init(&bar_a[s], 1);
+        mbar_init(&bar_b, 4);
+        mbar_init(&bar_done, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&tmem_slot, tmem_cols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&map_w);
+            for (int i = 0; i < n_kb; ++i) {      // weights: independent of every earlier kernel
+                mbar_expect_tx(&bar_a[i], kATileBytes);
+                tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[i]);
+            }
+        }
+        pdl_wait();
+    } else if (warp == 1) {
+        pdl_wait();
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(p.n_tile);
+            bool ok = mbar_wait(&bar_b, 0, &abort_flag);
+            for (int i = 0; i < n_kb && ok; ++i) {
+                ok = mbar_wait(&bar_a[i], 0, &abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sa = smem_u32(tiles + static_cast<size_t>(i) * stage_bytes);
+                const uint64_t da = smem_desc_sw128(sa), dh = smem_desc_sw128(sa + kATileBytes),
+                               dl = smem_desc_sw128(sa + kATileBytes + plane_bytes);
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(tmem_base, da + 2 * k, dh + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(tmem_base, da + 2 * k, dl + 2 * k, idesc, 1u);
+            }
+            if (ok) mma_commit(&bar_done);
+            else {
+                // the weight copies were requested whatever happens: let them land before the block retires
+                for (int i = 0; i < n_kb; ++i) {
+                    const long long start = clock64();
+                    while (!mbar_try_wait(&bar_a[i], 0) && clock64() - start < kWaitCycles / 8) {}
+                }
+            }
+        }
+    } else {
+        pdl_wait();
+        const int pt = threadIdx.x - 64;                  // 0..127 among the producer / epilogue threads
+        const int n_rows = p.state->n_active;
+        // ---- activation tiles --------------------------------------------------------------------------
+        const int units = p.n_tile * 8;                   // (row, 16-byte chunk) pairs per k-block
+        for (int i = 0; i < n_kb; ++i) {
+            uint8_t *hi_tile = tiles + static_cast<size_t>(i) * stage_bytes + kATileBytes;
+            uint8_t *lo_tile = hi_tile + plane_bytes;
+            const int k0 = (kb_begin + i) * kBlockK;
+            for (int uidx = pt; uidx < units; uidx += 128) {
+                const int rl = uidx >> 3, c = uidx & 7;
+                const int r = row0 + rl, k = k0 + c * 8;
+                float y[8];
+                if (r < n_rows) {
+                    load8(p.src + static_cast<size_t>(r) * p.ld_src + k, y);
+                    if (MODE == B_GAMMA) {
+                        float g[8];
+                        load8(p.gamma + k, g);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) y[j] *= g[j];
+                    } else if (MODE == B_LN_RELU) {
+                        const float2 st = p.stats_in[r];
+                        float c1[8], c2[8];
+                        load8(p.c1 + k, c1);
+                        load8(p.c2 + k, c2);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) y[j] = fmaxf(fmaf(st.y, y[j] - st.x * c1[j], c2[j]), 0.f);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) y[j] = 0.f;
+                }
+                uint4 hi, lo;
+                split_planes(y, hi, lo);
+                const int off = rl * 128 + ((c ^ (rl & 7)) << 4);
+                *reinterpret_cast<uint4 *>(hi_tile + off) = hi;
+                *reinterpret_cast<uint4 *>(lo_tile + off) = lo;
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b)) : "memory");
+
+        // ---- side jobs while the MMAs run ------------------------------------------------------------------
+        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        const int n_cta = gridDim.x * gridDim.y * gridDim.z;
+        if (p.zero_buf) {
+            const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
+            float4 *z = reinterpret_cast<float4 *>(p.zero_buf);
+            for (size_t idx = static_cast<size_t>(cta) * 128 + pt; idx < total4; idx += static_cast<size_t>(n_cta) * 128)
+                z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (p.stats_src) {
+            for (int r = cta; r < n_rows; r += n_cta) {    // uniform over the four warps
+                const float *xr = p.stats_src + static_cast<size_t>(r) * p.stats_d;
+                float s = 0.f;
+                for (int idx = pt * 4; idx < p.stats_d; idx += 512) {
+                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+                    s += (v.x + v.y) + (v.z + v.w);
+                }
+                s = warp_sum(s);
+                if (lane == 0) red_s[warp - 2] = s;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const float mean = (red_s[0] + red_s[1] + red_s[2] + red_s[3]) / p.stats_d;
+                float q = 0.f;
+                for (int idx = pt * 4; idx < p.stats_d; idx += 512) {
+                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+                    const float d0 = v.x - mean, d1 = v.y - mean, d2 = v.z - mean, d3 = v.w - mean;
+                    q += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+                }
+                q = warp_sum(q);
+                if (lane == 0) red_q[warp - 2] = q;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (pt == 0) p.stats_out[r] = make_float2(mean, rsqrtf((red_q[0] + red_q[1] + red_q[2] + red_q[3]) / p.stats_d + p.eps));
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+        }
+
+        // ---- epilogue -------------------------------------------------------------------------------------------
+        const int quarter = warp & 3;
+        const bool ok = mbar_wait(&bar_done, 0, &abort_flag);
+        tc_fence_after_sync();
+        if (ok) {
+            const int a_idx = a0 + quarter * 32 + lane;
+            const bool a_ok = a_idx < p.a_rows;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+            for (int c0 = 0; c0 < p.n_tile && row0 + c0 < n_rows; c0 += 16) {
+                float v[16];
+                tmem_ld16(taddr + c0, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int r = row0 + c0 + j;
+                    if (a_ok && r < n_rows) atomicAdd(p.out + static_cast<size_t>(r) * p.ldo + a_idx, v[j] + bias);
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&p.state->error, kErrTimeout);
+}
+
+// c1[o] = sum_k gamma[k] W[o,k];  c2[o] = sum_k beta[k] W[o,k] + bias[o]   (one warp per output feature)
+__global__ void ln_fold_constants_kernel(const __nv_bfloat16 *__restrict__ w, const __nv_bfloat16 *__restrict__ gamma,
+                                         const __nv_bfloat16 *__restrict__ beta, const __nv_bfloat16 *__restrict__ bias,
+                                         int m, int k, float *__restrict__ c1, float *__restrict__ c2)
+{
+    const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (o >= m) return;
+    float s1 = 0.f, s2 = 0.f;
+    for (int i = lane; i < k; i += 32) {
+        const float wv = to_f32(w[static_cast<size_t>(o) * k + i]);
+        s1 = fmaf(to_f32(gamma[i]), wv, s1);
+        s2 = fmaf(to_f32(beta[i]), wv, s2);
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    if (lane == 0) { c1[o] = s1; c2[o] = s2 + (bias ? to_f32(bias[o]) : 0.f); }
+}
+
+}  // namespace sg
+}  // namespace aed

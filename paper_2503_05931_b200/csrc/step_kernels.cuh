@@ -69,7 +69,7 @@ template <typename T>
 __global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ active_list,
                              const int32_t *__restrict__ tokens, const int32_t *__restrict__ t_u,
                              const T *__restrict__ embed, const float *__restrict__ pe, int d, int vocab, float scale,
-                             float *__restrict__ x)
+                             float *__restrict__ x, float *__restrict__ zero_buf = nullptr, int zero_cols = 0)
 {
     AED_TRACE_BEGIN(state, 2);
     int r = blockIdx.x;
@@ -80,6 +80,7 @@ __global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ 
     int t = t_u[u];
     for (int i = threadIdx.x; i < d; i += blockDim.x)
         x[(size_t)r * d + i] = to_f32(embed[(size_t)tok * d + i]) * scale + pe[(size_t)t * d + i];
+    for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
 }
 
 // out[r] = g * (x[r] - mean) / sqrt(var + eps) + b, biased variance, two passes over a row held in registers.
@@ -391,8 +392,12 @@ template <typename CT, bool kCross, bool kAppend>
 __global__ void __launch_bounds__(kFusedMaxWarps * 32, 4)
 attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ q, int ldq,
                   CT *__restrict__ cache, int n_heads, int seq_capacity, float scale,
-                  float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo)
+                  float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo,
+                  const float2 *__restrict__ ln_stats, const float *__restrict__ ln_c1, const float *__restrict__ ln_c2)
 {
+    // Launched with programmatic stream serialization: nothing written by earlier kernels is touched before this.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     AED_TRACE_BEGIN(state, 3);
     __shared__ float sm_m[kFusedMaxWarps], sm_l[kFusedMaxWarps];
     __shared__ float sm_acc[kFusedMaxWarps][kHeadDim];
@@ -412,11 +417,22 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
     }
     const int dg = lane & 7, pg = lane >> 3;
+    // When the projection ran on gamma*x (LayerNorm folded), its raw output y becomes rstd*(y - mean*c1) + c2 here.
+    float2 st = make_float2(0.f, 1.f);
+    if (ln_stats) st = ln_stats[r];
     if (kAppend && !kCross) {
         if (warp == 0 && lane < 16) {
             const int kv = lane >> 3, d_model = n_heads * kHeadDim;
+            const int col = (1 + kv) * d_model + h * kHeadDim + dg * 8;
             float nv[8];
-            load8(q + (size_t)r * ldq + (1 + kv) * d_model + h * kHeadDim + dg * 8, nv);
+            load8(q + (size_t)r * ldq + col, nv);
+            if (ln_stats) {
+                float c1[8], c2[8];
+                load8(ln_c1 + col, c1);
+                load8(ln_c2 + col, c2);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) nv[i] = fmaf(st.y, nv[i] - st.x * c1[i], c2[i]);
+            }
             CT *dst = const_cast<CT *>(kv ? vbase : kbase) + (size_t)(len - 1) * kHeadDim + dg * 8;
 #pragma unroll
             for (int i = 0; i < 8; ++i) dst[i] = from_f32<CT>(nv[i]);
@@ -425,6 +441,13 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     }
     float qv[8];
     load8(q + (size_t)r * ldq + h * kHeadDim + dg * 8, qv);
+    if (ln_stats) {
+        float c1[8], c2[8];
+        load8(ln_c1 + h * kHeadDim + dg * 8, c1);
+        load8(ln_c2 + h * kHeadDim + dg * 8, c2);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * c1[i], c2[i]);
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) qv[i] *= scale;
 

@@ -152,6 +152,7 @@ struct aed_dec {
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
     CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]
+    CUtensorMap tc_src_x[5], tc_src_att[5], tc_src_hid[5];   // fp32 sources of the fused projections, per MMA N
     int tc_kvc_box = 0;                           // rows of the w_kv_c box = MMA N of the precompute
     bool use_tc = false;
     int act_planes = 2;
@@ -404,17 +405,20 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// bf16 matrix [rows, cols] row-major; box = box_rows x 64 columns, 128-byte swizzle, zero fill out of bounds
-bool encode_map(CUtensorMap *map, const void *base, size_t rows, size_t cols, int box_rows)
+// matrix [rows, cols] row-major; box = box_rows x 64 columns, zero fill out of bounds.  bf16 operands use the
+// 128-byte swizzle the MMA descriptors name; fp32 staging tiles are copied unswizzled.
+bool encode_map(CUtensorMap *map, const void *base, size_t rows, size_t cols, int box_rows, bool fp32 = false)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    const size_t esz = fp32 ? 4 : 2;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
+    cuuint64_t strides[1] = {cols * esz};
     cuuint32_t box[2] = {(cuuint32_t)tc::kBlockK, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base),
+              dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              fp32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -443,7 +447,10 @@ aed_status_t tc_setup(aed_dec *dec)
         ok = ok && encode_map(&dec->tc_actd[i][0], dec->ws + L.actd_hi, L.rows_cap, d, box) &&
              encode_map(&dec->tc_actd[i][1], dec->ws + L.actd_lo, L.rows_cap, d, box) &&
              encode_map(&dec->tc_actf[i][0], dec->ws + L.actf_hi, L.rows_cap, F, box) &&
-             encode_map(&dec->tc_actf[i][1], dec->ws + L.actf_lo, L.rows_cap, F, box);
+             encode_map(&dec->tc_actf[i][1], dec->ws + L.actf_lo, L.rows_cap, F, box) &&
+             encode_map(&dec->tc_src_x[i], dec->ws + L.x, c.max_batch, d, box, true) &&
+             encode_map(&dec->tc_src_att[i], dec->ws + L.act, c.max_batch, d, box, true) &&
+             encode_map(&dec->tc_src_hid[i], dec->ws + L.hid, c.max_batch, F, box, true);
     }
     if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed (are all weight tensors 16-byte aligned?)");
     const int smem = kTcSmemBudget + 1024;
@@ -613,14 +620,14 @@ struct FusedGemm {
 };
 
 template <int MODE>
-aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, int M, int K, int rows_ub,
-                              sg::StepGemmParams p)
+aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, const CUtensorMap *src_maps, int M,
+                              int K, int rows_ub, sg::StepGemmParams p)
 {
     ProfScope ps(dec, family);
     const int ni = tc_n_index(rows_ub), n_tile = 16 << ni;
     const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
     const int k_blocks = K / tc::kBlockK;
-    const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2;
+    const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2 + n_tile * tc::kBlockK * 4;
     int kb_cta = kTcSmemBudget / stage_bytes;
     if (kb_cta > sg::kMaxKb) kb_cta = sg::kMaxKb;
     int splits = (k_blocks + kb_cta - 1) / kb_cta;
@@ -643,7 +650,7 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     attr[0].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, src_maps[ni], p);
     if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "projection launch: %s", cudaGetErrorString(e));
     AED_LAUNCHED(dec);
     return AED_OK;
@@ -681,7 +688,7 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.out = qkv; p.ldo = 3 * d; p.bias = nullptr;
         p.stats_src = x; p.stats_out = stats; p.stats_d = d;
         p.zero_buf = qc; p.zero_cols = d;
-        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, 3 * d, d, rows_ub, p));
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p));
         // 2. self-attention (applies LN1 to q, k, v; appends k, v)
         AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
                                                         nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
@@ -690,13 +697,13 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.src = att; p.ld_src = d;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
         p.zero_buf = hid; p.zero_cols = F;
-        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, d, d, rows_ub, p));
+        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, dec->tc_src_att, d, d, rows_ub, p));
         // 4. q' raw = (gamma2 * x) Wqc^T ; side: LN2 statistics
         p = sg::StepGemmParams{};
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln2_g;
         p.out = qc; p.ldo = d;
         p.stats_src = x; p.stats_out = stats + stats_stride; p.stats_d = d;
-        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QC, m.qc, d, d, rows_ub, p));
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QC, m.qc, dec->tc_src_x, d, d, rows_ub, p));
         // 5. cross-attention
         AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
                                                         nullptr, nullptr, stats + stats_stride, c1_qc, c2_qc, pdl)));
@@ -705,18 +712,18 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.src = att; p.ld_src = d;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
         p.zero_buf = qkv; p.zero_cols = 3 * d;
-        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_OC, m.oc, d, d, rows_ub, p));
+        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_OC, m.oc, dec->tc_src_att, d, d, rows_ub, p));
         // 7. hidden raw = (gamma3 * x) W1^T ; side: LN3 statistics
         p = sg::StepGemmParams{};
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln3_g;
         p.out = hid; p.ldo = F;
         p.stats_src = x; p.stats_out = stats + 2 * stats_stride; p.stats_d = d;
-        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, F, d, rows_ub, p));
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, dec->tc_src_x, F, d, rows_ub, p));
         // 8. x += relu(LN3-corrected hidden) W2^T + b2
         p = sg::StepGemmParams{};
         p.src = hid; p.ld_src = F; p.c1 = c1_ff; p.c2 = c2_ff; p.stats_in = stats + 2 * stats_stride;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
-        AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, d, F, rows_ub, p));
+        AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, dec->tc_src_hid, d, F, rows_ub, p));
     }
     AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
     tc::TcParams tp{};

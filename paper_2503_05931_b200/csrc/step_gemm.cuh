@@ -26,7 +26,7 @@ namespace sg {
 using namespace tc;
 
 constexpr int kMaxKb = 4;             // k-blocks per CTA
-constexpr int kSgThreads = 192;
+constexpr int kSgThreads = 256;       // warp 0 TMA, warp 1 MMA, warps 2..5 activation tiles + epilogue, warps 6..7 side jobs
 
 enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2 };
 
@@ -79,18 +79,27 @@ __device__ __forceinline__ void split_planes(const float (&y)[8], uint4 &hi, uin
     lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
-// grid: x = 128-feature tiles, y = k-splits, z = row tiles.  Dynamic smem: kb * (16 KB + 2 * n_tile * 128) + 1024.
+// 4 floats added to 4 consecutive addresses with one reduction (16-byte aligned)
+__device__ __forceinline__ void red_add_v4(float *addr, float4 v)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
+// grid: x = 128-feature tiles, y = k-splits, z = row tiles.
+// Dynamic smem per k-block: weight tile 16 KB | high plane | low plane (n_tile x 128 B each) | fp32 source tile
+// (n_tile x 256 B, filled by TMA, later reused to transpose the accumulator); plus 1024 for alignment.
 template <int MODE>
 __global__ void __launch_bounds__(kSgThreads, 1)
-step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, StepGemmParams p)
+step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_src, StepGemmParams p)
 {
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t bar_a[kMaxKb];
+    __shared__ __align__(8) uint64_t bar_s[kMaxKb];
     __shared__ __align__(8) uint64_t bar_b;
     __shared__ __align__(8) uint64_t bar_done;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float red_s[4], red_q[4];
+    __shared__ float red_s[2], red_q[2];
 
     AED_TRACE_BEGIN(p.state, 19);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -102,12 +111,13 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, StepGemmParams p)
 
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
     const int plane_bytes = p.n_tile * kBlockK * 2;
-    const int stage_bytes = kATileBytes + 2 * plane_bytes;
+    const int src_bytes = p.n_tile * kBlockK * 4;
+    const int stage_bytes = kATileBytes + 2 * plane_bytes + src_bytes;
     uint32_t tmem_cols = 32;
     while (tmem_cols < static_cast<uint32_t>(p.n_tile)) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxKb; ++s) mbar_init(&bar_a[s], 1);
+        for (int s = 0; s < kMaxKb; ++s) { mbar_init(&bar_a[s], 1); mbar_init(&bar_s[s], 1); }
         mbar_init(&bar_b, 4);
         mbar_init(&bar_done, 1);
         abort_flag = 0;
@@ -119,16 +129,25 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, StepGemmParams p)
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     pdl_launch_dependents();
+    if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 40);      // set-up done
 
     if (warp == 0) {
         if (lane == 0) {
             prefetch_tensormap(&map_w);
+            prefetch_tensormap(&map_src);
             for (int i = 0; i < n_kb; ++i) {      // weights: independent of every earlier kernel
                 mbar_expect_tx(&bar_a[i], kATileBytes);
                 tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[i]);
             }
         }
         pdl_wait();
+        if (lane == 0) {
+            for (int i = 0; i < n_kb; ++i) {      // fp32 activation source, written by the previous kernels
+                mbar_expect_tx(&bar_s[i], src_bytes);
+                tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes + kATileBytes + 2 * plane_bytes, &map_src,
+                            (kb_begin + i) * kBlockK, row0, &bar_s[i]);
+            }
+        }
     } else if (warp == 1) {
         pdl_wait();
         if (lane == 0) {
@@ -155,38 +174,85 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, StepGemmParams p)
                 }
             }
         }
+    } else if (warp >= 6) {
+        // ---- side jobs, off the critical path --------------------------------------------------------------
+        pdl_wait();
+        const int st = threadIdx.x - 192;                 // 0..63
+        const int n_rows = p.state->n_active;
+        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        const int n_cta = gridDim.x * gridDim.y * gridDim.z;
+        if (p.zero_buf) {
+            const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
+            float4 *z = reinterpret_cast<float4 *>(p.zero_buf);
+            for (size_t idx = static_cast<size_t>(cta) * 64 + st; idx < total4; idx += static_cast<size_t>(n_cta) * 64)
+                z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (p.stats_src) {
+            for (int r = cta; r < n_rows; r += n_cta) {    // uniform over the two warps
+                const float *xr = p.stats_src + static_cast<size_t>(r) * p.stats_d;
+                float s = 0.f;
+                for (int idx = st * 4; idx < p.stats_d; idx += 256) {
+                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+                    s += (v.x + v.y) + (v.z + v.w);
+                }
+                s = warp_sum(s);
+                if (lane == 0) red_s[warp - 6] = s;
+                asm volatile("bar.sync 1, 64;" ::: "memory");
+                const float mean = (red_s[0] + red_s[1]) / p.stats_d;
+                float q = 0.f;
+                for (int idx = st * 4; idx < p.stats_d; idx += 256) {
+                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+                    const float d0 = v.x - mean, d1 = v.y - mean, d2 = v.z - mean, d3 = v.w - mean;
+                    q += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+                }
+                q = warp_sum(q);
+                if (lane == 0) red_q[warp - 6] = q;
+                asm volatile("bar.sync 1, 64;" ::: "memory");
+                if (st == 0) p.stats_out[r] = make_float2(mean, rsqrtf((red_q[0] + red_q[1]) / p.stats_d + p.eps));
+                asm volatile("bar.sync 1, 64;" ::: "memory");
+            }
+        }
     } else {
         pdl_wait();
+        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 41);  // dependency resolved
         const int pt = threadIdx.x - 64;                  // 0..127 among the producer / epilogue threads
         const int n_rows = p.state->n_active;
         // ---- activation tiles --------------------------------------------------------------------------
-        const int units = p.n_tile * 8;                   // (row, 16-byte chunk) pairs per k-block
-        for (int i = 0; i < n_kb; ++i) {
-            uint8_t *hi_tile = tiles + static_cast<size_t>(i) * stage_bytes + kATileBytes;
-            uint8_t *lo_tile = hi_tile + plane_bytes;
-            const int k0 = (kb_begin + i) * kBlockK;
-            for (int uidx = pt; uidx < units; uidx += 128) {
-                const int rl = uidx >> 3, c = uidx & 7;
-                const int r = row0 + rl, k = k0 + c * 8;
+        // Thread pt owns the 16-byte output chunk c = pt & 7 (8 consecutive k) of rows (pt >> 3) + 16 j.  The fp32
+        // source tile of each k-block is already on its way into shared memory (TMA, no swizzle, 256 B per row).
+        const int c = pt & 7, rbase = pt >> 3;
+        const int passes = p.n_tile / 16;                 // n_tile is a multiple of 16
+        const int quarter = warp & 3;
+        const int a_idx = a0 + quarter * 32 + lane;
+        const bool a_ok = a_idx < p.a_rows;
+        const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+        bool ok = true;
+        for (int i = 0; i < n_kb && ok; ++i) {
+            uint8_t *stage = tiles + static_cast<size_t>(i) * stage_bytes;
+            uint8_t *hi_tile = stage + kATileBytes, *lo_tile = hi_tile + plane_bytes;
+            const float *src_tile = reinterpret_cast<const float *>(lo_tile + plane_bytes);
+            const int k = (kb_begin + i) * kBlockK + c * 8;
+            float g[8], c1[8], c2[8];
+            if (MODE == B_GAMMA) load8(p.gamma + k, g);
+            if (MODE == B_LN_RELU) { load8(p.c1 + k, c1); load8(p.c2 + k, c2); }
+            ok = mbar_wait(&bar_s[i], 0, &abort_flag);
+            if (!ok) break;
+            for (int j = 0; j < passes; ++j) {
+                const int rl = rbase + j * 16, r = row0 + rl;
                 float y[8];
                 if (r < n_rows) {
-                    load8(p.src + static_cast<size_t>(r) * p.ld_src + k, y);
+                    load8(src_tile + rl * kBlockK + c * 8, y);
                     if (MODE == B_GAMMA) {
-                        float g[8];
-                        load8(p.gamma + k, g);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) y[j] *= g[j];
+                        for (int e = 0; e < 8; ++e) y[e] *= g[e];
                     } else if (MODE == B_LN_RELU) {
                         const float2 st = p.stats_in[r];
-                        float c1[8], c2[8];
-                        load8(p.c1 + k, c1);
-                        load8(p.c2 + k, c2);
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) y[j] = fmaxf(fmaf(st.y, y[j] - st.x * c1[j], c2[j]), 0.f);
+                        for (int e = 0; e < 8; ++e) y[e] = fmaxf(fmaf(st.y, y[e] - st.x * c1[e], c2[e]), 0.f);
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) y[j] = 0.f;
+                    for (int e = 0; e < 8; ++e) y[e] = 0.f;
                 }
                 uint4 hi, lo;
                 split_planes(y, hi, lo);
@@ -197,63 +263,53 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, StepGemmParams p)
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
         __syncwarp();
-        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b)) : "memory");
+        if (lane == 0 && ok) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b)) : "memory");
+        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 42);  // activation tiles written
 
-        // ---- side jobs while the MMAs run ------------------------------------------------------------------
-        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        const int n_cta = gridDim.x * gridDim.y * gridDim.z;
-        if (p.zero_buf) {
-            const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
-            float4 *z = reinterpret_cast<float4 *>(p.zero_buf);
-            for (size_t idx = static_cast<size_t>(cta) * 128 + pt; idx < total4; idx += static_cast<size_t>(n_cta) * 128)
-                z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (p.stats_src) {
-            for (int r = cta; r < n_rows; r += n_cta) {    // uniform over the four warps
-                const float *xr = p.stats_src + static_cast<size_t>(r) * p.stats_d;
-                float s = 0.f;
-                for (int idx = pt * 4; idx < p.stats_d; idx += 512) {
-                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
-                    s += (v.x + v.y) + (v.z + v.w);
-                }
-                s = warp_sum(s);
-                if (lane == 0) red_s[warp - 2] = s;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                const float mean = (red_s[0] + red_s[1] + red_s[2] + red_s[3]) / p.stats_d;
-                float q = 0.f;
-                for (int idx = pt * 4; idx < p.stats_d; idx += 512) {
-                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
-                    const float d0 = v.x - mean, d1 = v.y - mean, d2 = v.z - mean, d3 = v.w - mean;
-                    q += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-                }
-                q = warp_sum(q);
-                if (lane == 0) red_q[warp - 2] = q;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (pt == 0) p.stats_out[r] = make_float2(mean, rsqrtf((red_q[0] + red_q[1] + red_q[2] + red_q[3]) / p.stats_d + p.eps));
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-            }
-        }
-
-        // ---- epilogue -------------------------------------------------------------------------------------------
-        const int quarter = warp & 3;
-        const bool ok = mbar_wait(&bar_done, 0, &abort_flag);
+        // ---- epilogue: accumulator -> shared memory (transposed) -> 16-byte reductions ---------------------------
+        ok = ok && mbar_wait(&bar_done, 0, &abort_flag);
         tc_fence_after_sync();
-        if (ok) {
-            const int a_idx = a0 + quarter * 32 + lane;
-            const bool a_ok = a_idx < p.a_rows;
+        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 44);  // accumulator complete
+        // every MMA has completed, so the whole stage area is free: T[r][o], 132 floats per row (bank spread)
+        float *trans = reinterpret_cast<float *>(tiles);
+        constexpr int kPitch = kTileM + 4;
+        const int rows_here = min(p.n_tile, max(n_rows - row0, 0));
+        const bool fits = static_cast<size_t>(p.n_tile) * kPitch * 4 <= static_cast<size_t>(n_kb) * stage_bytes;
+        if (ok && fits) {
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
-            for (int c0 = 0; c0 < p.n_tile && row0 + c0 < n_rows; c0 += 16) {
+            for (int c0 = 0; c0 < rows_here; c0 += 16) {
                 float v[16];
                 tmem_ld16(taddr + c0, v);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int r = row0 + c0 + j;
-                    if (a_ok && r < n_rows) atomicAdd(p.out + static_cast<size_t>(r) * p.ldo + a_idx, v[j] + bias);
+                for (int j = 0; j < 16; ++j) trans[(c0 + j) * kPitch + quarter * 32 + lane] = v[j] + bias;
+            }
+        }
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (ok && fits) {
+            const int o4 = (pt & 31) * 4;
+            for (int rl = pt >> 5; rl < rows_here; rl += 4) {
+                const float4 v = *reinterpret_cast<const float4 *>(trans + rl * kPitch + o4);
+                float *dst = p.out + static_cast<size_t>(row0 + rl) * p.ldo + a0 + o4;
+                if (a0 + o4 + 3 < p.a_rows) red_add_v4(dst, v);
+                else {
+                    if (a0 + o4 + 0 < p.a_rows) atomicAdd(dst + 0, v.x);
+                    if (a0 + o4 + 1 < p.a_rows) atomicAdd(dst + 1, v.y);
+                    if (a0 + o4 + 2 < p.a_rows) atomicAdd(dst + 2, v.z);
                 }
+            }
+        } else if (ok) {
+            // transposition buffer too small for this shape: scalar reductions straight from the accumulator
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            for (int c0 = 0; c0 < rows_here; c0 += 16) {
+                float v[16];
+                tmem_ld16(taddr + c0, v);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (a_ok && c0 + j < rows_here) atomicAdd(p.out + static_cast<size_t>(row0 + c0 + j) * p.ldo + a_idx, v[j] + bias);
             }
         }
     }
+    if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 45);      // epilogue issued
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {

@@ -26,7 +26,7 @@ namespace sg {
 using namespace tc;
 
 constexpr int kMaxKb = 4;             // k-blocks per CTA
-constexpr int kSgThreads = 256;       // warp 0 TMA, warp 1 MMA, warps 2..5 activation tiles + epilogue, warps 6..7 side jobs
+constexpr int kSgThreads = 384;       // warp 0 TMA, warp 1 MMA, warps 2..9 activation tiles (2..5 also epilogue), warps 10..11 side jobs
 
 enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2 };
 
@@ -95,7 +95,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t bar_a[kMaxKb];
     __shared__ __align__(8) uint64_t bar_s[kMaxKb];
-    __shared__ __align__(8) uint64_t bar_b;
+    __shared__ __align__(8) uint64_t bar_b[kMaxKb];
     __shared__ __align__(8) uint64_t bar_done;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -117,8 +117,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     while (tmem_cols < static_cast<uint32_t>(p.n_tile)) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxKb; ++s) { mbar_init(&bar_a[s], 1); mbar_init(&bar_s[s], 1); }
-        mbar_init(&bar_b, 4);
+        for (int s = 0; s < kMaxKb; ++s) { mbar_init(&bar_a[s], 1); mbar_init(&bar_s[s], 1); mbar_init(&bar_b[s], 8); }
         mbar_init(&bar_done, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -152,9 +151,9 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         pdl_wait();
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(p.n_tile);
-            bool ok = mbar_wait(&bar_b, 0, &abort_flag);
+            bool ok = true;
             for (int i = 0; i < n_kb && ok; ++i) {
-                ok = mbar_wait(&bar_a[i], 0, &abort_flag);
+                ok = mbar_wait(&bar_b[i], 0, &abort_flag) && mbar_wait(&bar_a[i], 0, &abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t sa = smem_u32(tiles + static_cast<size_t>(i) * stage_bytes);
@@ -174,10 +173,10 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 }
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= 10) {
         // ---- side jobs, off the critical path --------------------------------------------------------------
         pdl_wait();
-        const int st = threadIdx.x - 192;                 // 0..63
+        const int st = threadIdx.x - 320;                 // 0..63
         const int n_rows = p.state->n_active;
         const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
         const int n_cta = gridDim.x * gridDim.y * gridDim.z;
@@ -196,7 +195,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     s += (v.x + v.y) + (v.z + v.w);
                 }
                 s = warp_sum(s);
-                if (lane == 0) red_s[warp - 6] = s;
+                if (lane == 0) red_s[warp - 10] = s;
                 asm volatile("bar.sync 1, 64;" ::: "memory");
                 const float mean = (red_s[0] + red_s[1]) / p.stats_d;
                 float q = 0.f;
@@ -206,7 +205,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     q += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
                 }
                 q = warp_sum(q);
-                if (lane == 0) red_q[warp - 6] = q;
+                if (lane == 0) red_q[warp - 10] = q;
                 asm volatile("bar.sync 1, 64;" ::: "memory");
                 if (st == 0) p.stats_out[r] = make_float2(mean, rsqrtf((red_q[0] + red_q[1]) / p.stats_d + p.eps));
                 asm volatile("bar.sync 1, 64;" ::: "memory");
@@ -215,17 +214,17 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     } else {
         pdl_wait();
         if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 41);  // dependency resolved
-        const int pt = threadIdx.x - 64;                  // 0..127 among the producer / epilogue threads
+        const int pt = threadIdx.x - 64;                  // 0..255 among the producer threads
         const int n_rows = p.state->n_active;
         // ---- activation tiles --------------------------------------------------------------------------
-        // Thread pt owns the 16-byte output chunk c = pt & 7 (8 consecutive k) of rows (pt >> 3) + 16 j.  The fp32
+        // Thread pt owns the 16-byte output chunk c = pt & 7 (8 consecutive k) of rows (pt >> 3) + 32 j.  The fp32
         // source tile of each k-block is already on its way into shared memory (TMA, no swizzle, 256 B per row).
+        // Each k-block has its own barrier, so the MMAs of one k-block run while the next is converted.
         const int c = pt & 7, rbase = pt >> 3;
-        const int passes = p.n_tile / 16;                 // n_tile is a multiple of 16
         const int quarter = warp & 3;
         const int a_idx = a0 + quarter * 32 + lane;
         const bool a_ok = a_idx < p.a_rows;
-        const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+        const float bias = (warp < 6 && p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
         bool ok = true;
         for (int i = 0; i < n_kb && ok; ++i) {
             uint8_t *stage = tiles + static_cast<size_t>(i) * stage_bytes;
@@ -237,8 +236,8 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             if (MODE == B_LN_RELU) { load8(p.c1 + k, c1); load8(p.c2 + k, c2); }
             ok = mbar_wait(&bar_s[i], 0, &abort_flag);
             if (!ok) break;
-            for (int j = 0; j < passes; ++j) {
-                const int rl = rbase + j * 16, r = row0 + rl;
+            for (int rl = rbase; rl < p.n_tile; rl += 32) {
+                const int r = row0 + rl;
                 float y[8];
                 if (r < n_rows) {
                     load8(src_tile + rl * kBlockK + c * 8, y);
@@ -260,11 +259,12 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 *reinterpret_cast<uint4 *>(hi_tile + off) = hi;
                 *reinterpret_cast<uint4 *>(lo_tile + off) = lo;
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b[i])) : "memory");
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
-        __syncwarp();
-        if (lane == 0 && ok) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b)) : "memory");
         if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 42);  // activation tiles written
+        if (warp < 6) {                                   // only warps 2..5 own accumulator lanes
 
         // ---- epilogue: accumulator -> shared memory (transposed) -> 16-byte reductions ---------------------------
         ok = ok && mbar_wait(&bar_done, 0, &abort_flag);
@@ -307,6 +307,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 for (int j = 0; j < 16; ++j)
                     if (a_ok && c0 + j < rows_here) atomicAdd(p.out + static_cast<size_t>(row0 + c0 + j) * p.ldo + a_idx, v[j] + bias);
             }
+        }
         }
     }
     if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 45);      // epilogue issued

@@ -395,16 +395,18 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo,
                   const float2 *__restrict__ ln_stats, const float *__restrict__ ln_c1, const float *__restrict__ ln_c2)
 {
-    // Launched with programmatic stream serialization: nothing written by earlier kernels is touched before this.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    AED_TRACE_BEGIN(state, 3);
+    // Launched with programmatic stream serialization.  Before the dependency wait only data that no kernel of
+    // this step writes is touched: the row table (written by the step's first kernel, which ran to completion
+    // before any programmatic launch of the step) and, for cross-attention, the encoder K/V store.
     __shared__ float sm_m[kFusedMaxWarps], sm_l[kFusedMaxWarps];
     __shared__ float sm_acc[kFusedMaxWarps][kHeadDim];
     const int rh = blockIdx.x;
     const int r = rh / n_heads, h = rh % n_heads;
     const int4 ri = row_info[r];                       // (utterance, t_u, encoder length, encoder offset)
-    if (ri.x < 0) return;
+    if (ri.x < 0) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
     const int u = ri.x;
     const int len = kCross ? ri.z : ri.y + 1;
@@ -416,6 +418,23 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         kbase = cache + (((size_t)u * 2 + 0) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
         vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
     }
+    Raw8<CT> rk[4], rv[4];
+    if (kCross) {
+        // The encoder keys and values of this warp's first chunk start streaming while the kernel that produces
+        // the query is still running.
+        const int p0 = warp * kFusedChunk;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = p0 + i * 4 + (lane >> 3);
+            if (p < len) {
+                rk[i].load(kbase + (size_t)p * kHeadDim + (lane & 7) * 8);
+                rv[i].load(vbase + (size_t)p * kHeadDim + (lane & 7) * 8);
+            } else { rk[i].zero(); rv[i].zero(); }
+        }
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    AED_TRACE_BEGIN(state, 3);
     const int dg = lane & 7, pg = lane >> 3;
     // When the projection ran on gamma*x (LayerNorm folded), its raw output y becomes rstd*(y - mean*c1) + c2 here.
     float2 st = make_float2(0.f, 1.f);
@@ -454,16 +473,19 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     float m = -INFINITY, l = 0.f, acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    bool loaded = kCross;
     for (int p0 = warp * kFusedChunk; p0 < len; p0 += n_warps * kFusedChunk) {
-        Raw8<CT> rk[4], rv[4];
+        if (!loaded) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {          // keys and values of the chunk are requested together
-            const int p = p0 + i * 4 + pg;
-            if (p < len) {
-                rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
-                rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
-            } else { rk[i].zero(); rv[i].zero(); }
+            for (int i = 0; i < 4; ++i) {          // keys and values of the chunk are requested together
+                const int p = p0 + i * 4 + pg;
+                if (p < len) {
+                    rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
+                    rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
+                } else { rk[i].zero(); rv[i].zero(); }
+            }
         }
+        loaded = false;
         float s[4], cmax = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

@@ -305,6 +305,9 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
     if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
     if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
+    // Cross-attention starts early and holds its first chunk in registers: 4 warps per block keep every block of
+    // a 64-row step resident at once (8 blocks per SM), longer rows loop and find their later chunks in L2.
+    if (kCross && warps > 4) warps = 4;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(rows_ub * dec->cfg.n_heads);
     cfg.blockDim = dim3(warps * 32);
@@ -682,12 +685,15 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
         const float *c1_qkv = fc, *c2_qkv = fc + 3 * d, *c1_qc = fc + 6 * d, *c2_qc = fc + 7 * d, *c1_ff = fc + 8 * d,
                     *c2_ff = fc + 8 * d + F;
+        const LayerWeights &wn = dec->layers[(l + 1) % c.n_layers];     // next layer (or layer 0 of the next step)
+        const size_t e2 = sizeof(T);
         sg::StepGemmParams p{};
         // 1. [q | k | v] raw = (gamma1 * x) Wqkv^T ; side: LN1 statistics of x, clear the cross-query rows
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln1_g;
         p.out = qkv; p.ldo = 3 * d; p.bias = nullptr;
         p.stats_src = x; p.stats_out = stats; p.stats_d = d;
         p.zero_buf = qc; p.zero_cols = d;
+        p.prefetch_ptr = wn.w_qkv; p.prefetch_bytes = (size_t)3 * d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p));
         // 2. self-attention (applies LN1 to q, k, v; appends k, v)
         AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
@@ -697,12 +703,14 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.src = att; p.ld_src = d;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
         p.zero_buf = hid; p.zero_cols = F;
+        p.prefetch_ptr = wn.w_o; p.prefetch_bytes = (size_t)d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, dec->tc_src_att, d, d, rows_ub, p));
         // 4. q' raw = (gamma2 * x) Wqc^T ; side: LN2 statistics
         p = sg::StepGemmParams{};
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln2_g;
         p.out = qc; p.ldo = d;
         p.stats_src = x; p.stats_out = stats + stats_stride; p.stats_d = d;
+        p.prefetch_ptr = wn.w_q_c; p.prefetch_bytes = (size_t)d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QC, m.qc, dec->tc_src_x, d, d, rows_ub, p));
         // 5. cross-attention
         AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
@@ -712,17 +720,20 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.src = att; p.ld_src = d;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
         p.zero_buf = qkv; p.zero_cols = 3 * d;
+        p.prefetch_ptr = wn.w_o_c; p.prefetch_bytes = (size_t)d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_OC, m.oc, dec->tc_src_att, d, d, rows_ub, p));
         // 7. hidden raw = (gamma3 * x) W1^T ; side: LN3 statistics
         p = sg::StepGemmParams{};
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln3_g;
         p.out = hid; p.ldo = F;
         p.stats_src = x; p.stats_out = stats + 2 * stats_stride; p.stats_d = d;
+        p.prefetch_ptr = wn.w_ff1; p.prefetch_bytes = (size_t)F * d * e2;
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, dec->tc_src_x, F, d, rows_ub, p));
         // 8. x += relu(LN3-corrected hidden) W2^T + b2
         p = sg::StepGemmParams{};
         p.src = hid; p.ld_src = F; p.c1 = c1_ff; p.c2 = c2_ff; p.stats_in = stats + 2 * stats_stride;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
+        p.prefetch_ptr = wn.w_ff2; p.prefetch_bytes = (size_t)F * d * e2;
         AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, dec->tc_src_hid, d, F, rows_ub, p));
     }
     AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));

@@ -52,6 +52,9 @@ struct StepGemmParams {
     // side job 2: clear zero_buf [rows, zero_cols]
     float *zero_buf;
     int zero_cols;
+    // side job 3: pull a byte range that a later kernel streams (next layer's weights) into L2
+    const void *prefetch_ptr;
+    size_t prefetch_bytes;
     DecState *state;
 };
 
@@ -175,11 +178,18 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         }
     } else if (warp >= 10) {
         // ---- side jobs, off the critical path --------------------------------------------------------------
-        pdl_wait();
         const int st = threadIdx.x - 320;                 // 0..63
-        const int n_rows = p.state->n_active;
         const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
         const int n_cta = gridDim.x * gridDim.y * gridDim.z;
+        if (p.prefetch_ptr) {
+            // static data: no need to wait for the previous kernel.  4 KB pieces, spread over all CTAs and threads.
+            const size_t pieces = p.prefetch_bytes / 4096;
+            const char *base = static_cast<const char *>(p.prefetch_ptr);
+            for (size_t i = static_cast<size_t>(cta) * 64 + st; i < pieces; i += static_cast<size_t>(n_cta) * 64)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + i * 4096), "r"(4096) : "memory");
+        }
+        pdl_wait();
+        const int n_rows = p.state->n_active;
         if (p.zero_buf) {
             const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
             float4 *z = reinterpret_cast<float4 *>(p.zero_buf);

@@ -431,6 +431,19 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
                 rv[i].load(vbase + (size_t)p * kHeadDim + (lane & 7) * 8);
             } else { rk[i].zero(); rv[i].zero(); }
         }
+        // later chunks of this warp: pull them into L2 now (one 128-byte row per lane group)
+        if ((lane & 7) == 0) {
+            for (int q0 = p0 + n_warps * kFusedChunk; q0 < len; q0 += n_warps * kFusedChunk) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int p = q0 + i * 4 + (lane >> 3);
+                    if (p < len) {
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(kbase + (size_t)p * kHeadDim));
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(vbase + (size_t)p * kHeadDim));
+                    }
+                }
+            }
+        }
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

@@ -172,6 +172,53 @@ def test_error_codes():
     lib.aed_dec_destroy(None)
 
 
+@pytest.mark.parametrize("batch", [130, 300, 520])
+def test_large_batches_bf16(batch):
+    """Row counts beyond one MMA tile: N = 256 tiles, two and three row tiles, with rows retiring at different steps."""
+    rng = np.random.default_rng(batch)
+    enc_lens = rng.integers(1, 90, size=batch)
+    dec_lens = rng.integers(1, 9, size=batch)
+    dec_lens[:3] = [12, 1, 7]
+    w = wl.make_custom(MID, enc_lens, dec_lens, dtype="bf16", seed=40 + batch)
+    rows = [0, 1, 2, batch // 2, batch - 2, batch - 1] + [int(r) for r in rng.choice(batch, size=6, replace=False)]
+    _run_both(w, rows=sorted(set(rows)))
+
+
+def test_eos_variant_with_seed_scan():
+    """EOS stopping on the bf16 path: an utterance retires right after emitting eos, the others keep going.
+    Utterances are checked where the checker's margins are clear up to their expected end."""
+    b = _binding()
+    checked = 0
+    for seed in range(20, 30):
+        w = wl.make_custom(SMALL, [12, 20, 7, 33], [10, 10, 10, 10], dtype="bf16", seed=seed)
+        ref = oracle_reference(w)
+        eos = int(ref["next"][1, 3])
+        dec = b.decoder_for_workload(w, eos_id=eos)
+        dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
+        toks, lens = dec.greedy_decode(w.dec_lens)
+        toks, lens = toks.cpu().numpy(), lens.cpu().numpy()
+        dec.close()
+        for u in range(4):
+            hits = [t for t in range(10) if ref["next"][u, t] == eos]
+            expect = hits[0] + 1 if hits else 10
+            if not np.all(ref["margin"][u, :expect] > MARGIN):
+                continue
+            assert lens[u] == expect, (seed, u)
+            assert np.array_equal(toks[u, :expect], ref["next"][u, :expect])
+            assert np.all(toks[u, expect:] == -1)
+            checked += 1 if expect < 10 else 0
+    assert checked > 0        # at least one utterance really stopped early
+
+
+def test_config3_shape_sampled_rows():
+    """4-layer d=1024 bf16 decoder at batch 128 (shallow-decoder variant), sampled utterances against the checker."""
+    w = wl.make_workload("cfg3")
+    order = np.argsort(w.dec_lens)
+    rows = sorted({int(order[1]), int(order[len(order) // 3]), int(np.argmax(w.enc_lens)), 127})
+    rows = [r for r in rows if w.dec_lens[r] <= 60][:4]
+    _run_both(w, rows=rows)
+
+
 def test_config2_shape_sampled_rows():
     """24-layer d=1024 bf16 decoder at batch 64 (the benchmark configuration and launch path): a sample of
     utterances is decoded one by one by the checker and compared with the GPU's full-batch run."""

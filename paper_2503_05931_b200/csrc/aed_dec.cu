@@ -627,17 +627,24 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
                               int K, int rows_ub, sg::StepGemmParams p)
 {
     ProfScope ps(dec, family);
-    const int ni = tc_n_index(rows_ub), n_tile = 16 << ni;
+    // Rows per CTA tile: up to 128 (two ring stages still fit beside the transposition buffer); more rows are
+    // covered by row tiles that re-read the weight tile from L2.
+    int ni = tc_n_index(rows_ub);
+    if (ni > 3) ni = 3;
+    const int n_tile = 16 << ni;
     const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
     const int k_blocks = K / tc::kBlockK;
     const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2 + n_tile * tc::kBlockK * 4;
-    int kb_cta = kTcSmemBudget / stage_bytes;
-    if (kb_cta > sg::kMaxKb) kb_cta = sg::kMaxKb;
-    int splits = (k_blocks + kb_cta - 1) / kb_cta;
-    const int want = dec->tc_target_ctas / (m_tiles * row_tiles);
-    if (want > splits) splits = want;
+    int stages = kTcSmemBudget / stage_bytes;
+    if (stages > sg::kMaxKb) stages = sg::kMaxKb;
+    // k-splits only as far as they are needed to occupy the GPU: every split adds rows x features x 4 bytes of
+    // red.global traffic.
+    int splits = dec->tc_target_ctas / (m_tiles * row_tiles);
+    if (splits < 1) splits = 1;
     if (splits > k_blocks) splits = k_blocks;
     const int kb_max = (k_blocks + splits - 1) / splits;
+    if (stages > kb_max) stages = kb_max;
+    p.stages = stages;
     p.a_rows = M;
     p.k_blocks = k_blocks;
     p.n_tile = n_tile;
@@ -646,7 +653,7 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(m_tiles, splits, row_tiles);
     cfg.blockDim = dim3(sg::kSgThreads);
-    cfg.dynamicSmemBytes = (size_t)kb_max * stage_bytes + 1024;
+    cfg.dynamicSmemBytes = (size_t)stages * stage_bytes + 1024;
     cfg.stream = dec->stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -16,7 +16,8 @@
 // run, the producer warps of this kernel compute mean and rstd of the rows assigned to their CTA and store
 // them for the consumer.  A second side job clears the fp32 rows a later split-K projection accumulates into.
 //
-// All k-blocks of a CTA are resident at once (at most 4), so there is no ring to recycle.  Waits are bounded.
+// A CTA walks its k-blocks through a ring of up to 4 stages (weight tile, two planes, fp32 source tile each); with
+// few k-blocks per CTA (small batches, many k-splits) everything is resident at once.  Waits are bounded.
 #pragma once
 #include "tc_gemm.cuh"
 
@@ -25,7 +26,7 @@ namespace sg {
 
 using namespace tc;
 
-constexpr int kMaxKb = 4;             // k-blocks per CTA
+constexpr int kMaxKb = 4;             // ring stages per CTA
 constexpr int kSgThreads = 384;       // warp 0 TMA, warp 1 MMA, warps 2..9 activation tiles (2..5 also epilogue), warps 10..11 side jobs
 
 enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2 };
@@ -34,6 +35,7 @@ struct StepGemmParams {
     int a_rows;                // output features M
     int k_blocks;              // K / 64
     int n_tile;                // MMA N: rows per CTA tile (16..256, multiple of 16)
+    int stages;                // ring depth, 1..kMaxKb
     // activation source [rows, ld_src] fp32
     const float *src;
     int ld_src;
@@ -99,6 +101,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     __shared__ __align__(8) uint64_t bar_a[kMaxKb];
     __shared__ __align__(8) uint64_t bar_s[kMaxKb];
     __shared__ __align__(8) uint64_t bar_b[kMaxKb];
+    __shared__ __align__(8) uint64_t bar_e[kMaxKb];
     __shared__ __align__(8) uint64_t bar_done;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -110,7 +113,8 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     const int row0 = blockIdx.z * p.n_tile;
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
-    const int n_kb = kb_end - kb_begin;          // 1..kMaxKb by construction of the grid
+    const int n_kb = kb_end - kb_begin;
+    const int S = p.stages;
 
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
     const int plane_bytes = p.n_tile * kBlockK * 2;
@@ -120,7 +124,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     while (tmem_cols < static_cast<uint32_t>(p.n_tile)) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMaxKb; ++s) { mbar_init(&bar_a[s], 1); mbar_init(&bar_s[s], 1); mbar_init(&bar_b[s], 8); }
+        for (int s = 0; s < kMaxKb; ++s) { mbar_init(&bar_a[s], 1); mbar_init(&bar_s[s], 1); mbar_init(&bar_b[s], 8); mbar_init(&bar_e[s], 1); }
         mbar_init(&bar_done, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -137,17 +141,25 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         if (lane == 0) {
             prefetch_tensormap(&map_w);
             prefetch_tensormap(&map_src);
-            for (int i = 0; i < n_kb; ++i) {      // weights: independent of every earlier kernel
+            const int pre = n_kb < S ? n_kb : S;
+            for (int i = 0; i < pre; ++i) {       // weights: independent of every earlier kernel
                 mbar_expect_tx(&bar_a[i], kATileBytes);
                 tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[i]);
             }
         }
         pdl_wait();
         if (lane == 0) {
-            for (int i = 0; i < n_kb; ++i) {      // fp32 activation source, written by the previous kernels
-                mbar_expect_tx(&bar_s[i], src_bytes);
-                tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes + kATileBytes + 2 * plane_bytes, &map_src,
-                            (kb_begin + i) * kBlockK, row0, &bar_s[i]);
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % S;
+                uint8_t *stage = tiles + static_cast<size_t>(s) * stage_bytes;
+                if (i >= S) {                     // the stage is free once the MMAs of k-block i - S have read it
+                    if (!mbar_wait(&bar_e[s], ((i / S) - 1) & 1, &abort_flag)) break;
+                    mbar_expect_tx(&bar_a[s], kATileBytes);
+                    tma_load_2d(stage, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[s]);
+                }
+                // fp32 activation source, written by the previous kernels
+                mbar_expect_tx(&bar_s[s], src_bytes);
+                tma_load_2d(stage + kATileBytes + 2 * plane_bytes, &map_src, (kb_begin + i) * kBlockK, row0, &bar_s[s]);
             }
         }
     } else if (warp == 1) {
@@ -156,23 +168,26 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             const uint32_t idesc = instr_desc_bf16(p.n_tile);
             bool ok = true;
             for (int i = 0; i < n_kb && ok; ++i) {
-                ok = mbar_wait(&bar_b[i], 0, &abort_flag) && mbar_wait(&bar_a[i], 0, &abort_flag);
+                const int s = i % S;
+                const uint32_t par = (i / S) & 1;
+                ok = mbar_wait(&bar_b[s], par, &abort_flag) && mbar_wait(&bar_a[s], par, &abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t sa = smem_u32(tiles + static_cast<size_t>(i) * stage_bytes);
+                const uint32_t sa = smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
                 const uint64_t da = smem_desc_sw128(sa), dh = smem_desc_sw128(sa + kATileBytes),
                                dl = smem_desc_sw128(sa + kATileBytes + plane_bytes);
 #pragma unroll
                 for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(tmem_base, da + 2 * k, dh + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
 #pragma unroll
                 for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(tmem_base, da + 2 * k, dl + 2 * k, idesc, 1u);
+                if (i + S < n_kb) mma_commit(&bar_e[s]);      // someone is waiting to refill this stage
             }
             if (ok) mma_commit(&bar_done);
             else {
-                // the weight copies were requested whatever happens: let them land before the block retires
-                for (int i = 0; i < n_kb; ++i) {
+                // weight copies that were requested must land before the block retires
+                for (int s = 0; s < S && s < n_kb; ++s) {
                     const long long start = clock64();
-                    while (!mbar_try_wait(&bar_a[i], 0) && clock64() - start < kWaitCycles / 8) {}
+                    while (!mbar_try_wait(&bar_a[s], 0) && clock64() - start < kWaitCycles / 8) {}
                 }
             }
         }
@@ -237,14 +252,15 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const float bias = (warp < 6 && p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
         bool ok = true;
         for (int i = 0; i < n_kb && ok; ++i) {
-            uint8_t *stage = tiles + static_cast<size_t>(i) * stage_bytes;
+            const int s = i % S;
+            uint8_t *stage = tiles + static_cast<size_t>(s) * stage_bytes;
             uint8_t *hi_tile = stage + kATileBytes, *lo_tile = hi_tile + plane_bytes;
             const float *src_tile = reinterpret_cast<const float *>(lo_tile + plane_bytes);
             const int k = (kb_begin + i) * kBlockK + c * 8;
             float g[8], c1[8], c2[8];
             if (MODE == B_GAMMA) load8(p.gamma + k, g);
             if (MODE == B_LN_RELU) { load8(p.c1 + k, c1); load8(p.c2 + k, c2); }
-            ok = mbar_wait(&bar_s[i], 0, &abort_flag);
+            ok = mbar_wait(&bar_s[s], (i / S) & 1, &abort_flag);
             if (!ok) break;
             for (int rl = rbase; rl < p.n_tile; rl += 32) {
                 const int r = row0 + rl;
@@ -271,7 +287,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
             __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b[i])) : "memory");
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b[s])) : "memory");
         }
         if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 42);  // activation tiles written
         if (warp < 6) {                                   // only warps 2..5 own accumulator lanes
@@ -284,7 +300,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         float *trans = reinterpret_cast<float *>(tiles);
         constexpr int kPitch = kTileM + 4;
         const int rows_here = min(p.n_tile, max(n_rows - row0, 0));
-        const bool fits = static_cast<size_t>(p.n_tile) * kPitch * 4 <= static_cast<size_t>(n_kb) * stage_bytes;
+        const bool fits = static_cast<size_t>(p.n_tile) * kPitch * 4 <= static_cast<size_t>(n_kb < S ? n_kb : S) * stage_bytes;
         if (ok && fits) {
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             for (int c0 = 0; c0 < rows_here; c0 += 16) {

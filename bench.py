@@ -91,6 +91,25 @@ def roofline_seconds(w, peaks):
     return dec, pre
 
 
+def reduce_over_ranks(total_ms: float, n_tok: float, n_frames: float, device: str, world: int):
+    """Whole-job figures of a weak-scaling run: the slowest rank's time, tokens and frames summed over ranks.
+    Ranks decode independent batches, so these two reductions are the only communication of the benchmark."""
+    if world <= 1:
+        return total_ms, n_tok, n_frames
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([n_tok, n_frames], dtype=torch.float64, device=device)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(c[0].item()), float(c[1].item())
+
+
+def rank_seed(workload: str, rank: int) -> int:
+    """Every rank draws its own batch from the same distribution."""
+    return wl.BASE_SEED + wl._CONFIG_INDEX[workload] + 1000 * rank
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -195,6 +214,71 @@ def cpu_baseline(w, budget_tokens: int = 0):
             "rtfx": float(sub.enc_lens.sum()) * wl.FRAME_SECONDS / dt}
 
 
+def run_stream(args):
+    """cfg5: the same 4096 utterances decoded as random batches of 128 and as 2D buckets on (encoder length,
+    output length), 8 x 4 quantile bins with a 64k frame+token budget per batch.  Reports padding fractions,
+    tokens/s and RTFx of both arms in one JSON line (value = the bucketed arm)."""
+    import torch
+    from paper_2503_05931_b200 import binding, bucketing
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    device = "cuda:0"
+    torch.cuda.set_device(0)
+    w = wl.make_workload("cfg5")
+    peaks = load_peaks()
+    rng = np.random.default_rng(5)
+    arms = {"random128": bucketing.random_batches(w.batch, 128, rng),
+            "bucketed8x4": bucketing.bucket_batches_2d(w.enc_lens, w.dec_lens)}
+    all_batches = [b for bs in arms.values() for b in bs]
+    dec = binding.Decoder(w.model, w.weights, w.dtype, max_batch=max(len(b) for b in all_batches),
+                          max_total_enc_frames=max(int(w.enc_lens[b].sum()) for b in all_batches),
+                          max_enc_len=int(w.enc_lens.max()), max_dec_len=int(w.dec_lens.max()), bos_id=w.bos_id,
+                          eos_id=w.eos_id, ln_eps=w.ln_eps, device=device)
+    enc_all = torch.from_numpy(w.enc).to(device).to(dec.tdtype)
+    off = w.enc_offsets
+    toks = torch.empty((dec.max_batch, dec.max_dec_len), dtype=torch.int32, device=device)
+    lens = torch.empty(dec.max_batch, dtype=torch.int32, device=device)
+    result = {}
+    for name, batches in arms.items():
+        packed = [torch.cat([enc_all[off[u]:off[u + 1]] for u in b]) for b in batches]      # resident before timing
+        def run_arm():
+            for b, enc in zip(batches, packed):
+                dec.precompute_cross_kv(enc, w.enc_lens[b])
+                dec.greedy_decode(w.dec_lens[b], toks, lens)
+        run_arm()                                   # warm-up: captures the step graphs of this arm
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = dec.launch_count()
+        e0.record()
+        for _ in range(args.steps):
+            run_arm()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        pad_enc, pad_dec = bucketing.padding_fractions(w.enc_lens, w.dec_lens, batches)
+        roof = 0.0
+        for b in batches:
+            sub = w.subset_lengths(b)
+            d_s, p_s = roofline_seconds(sub, peaks)
+            roof += d_s + p_s
+        result[name] = {"batches": len(batches), "pad_enc": pad_enc, "pad_dec": pad_dec, "ms": ms,
+                        "tokens_per_s": float(w.dec_lens.sum()) / (ms * 1e-3), "rtfx": w.audio_seconds / (ms * 1e-3),
+                        "roofline_ms": 1e3 * roof, "roofline_frac": 1e3 * roof / ms,
+                        "gpu_launches": int((dec.launch_count() - launches0) / args.steps)}
+        del packed
+    dec.sync_status()
+    dec.close()
+    best = result["bucketed8x4"]
+    line = {"metric": "decoder output tokens/s", "value": best["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": 1, "ms_per_step": best["ms"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "cfg5", **w.model, "utterances": w.batch, "step": "one pass over the whole stream",
+                       "l2": "inputs larger than L2"},
+            "rtfx": best["rtfx"], "arms": result, "gpu_launches": best["gpu_launches"]}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -211,6 +295,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload == "cfg5":
+        run_stream(args)
         return
 
     import torch
@@ -229,7 +316,7 @@ def main():
 
     # Every rank decodes its own batch of the same distribution (utterances are independent: no collective
     # on the data path, weak scaling).
-    w = wl.make_workload(args.workload, seed=wl.BASE_SEED + wl._CONFIG_INDEX[args.workload] + 1000 * rank)
+    w = wl.make_workload(args.workload, seed=rank_seed(args.workload, rank))
     if args.clip_len > 0:
         w.dec_lens = np.minimum(w.dec_lens, args.clip_len).astype(np.int32)
     peaks = load_peaks()
@@ -268,10 +355,6 @@ def main():
         barrier()
         per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
         total_ms = ev[0].elapsed_time(ev[steps])
-        if world > 1:
-            t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
         return total_ms, per
 
     for _ in range(max(args.warmup, 3)):
@@ -287,10 +370,8 @@ def main():
     e2e_ms, _ = timed(True, args.steps)
     dec.sync_status()
 
-    tok_all = torch.tensor([n_tok, int(w.enc_lens.sum())], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(tok_all)
-    total_tokens, total_frames = float(tok_all[0].item()), float(tok_all[1].item())
+    e2e_ms, _, _ = reduce_over_ranks(e2e_ms, 0.0, 0.0, device, world)
+    total_ms, total_tokens, total_frames = reduce_over_ranks(total_ms, float(n_tok), float(w.enc_lens.sum()), device, world)
     value = total_tokens * args.steps / (total_ms * 1e-3)
     e2e_value = total_tokens * args.steps / (e2e_ms * 1e-3)
     rtfx = total_frames * wl.FRAME_SECONDS * args.steps / (total_ms * 1e-3)

@@ -124,6 +124,12 @@ class Workload:
     def audio_seconds(self) -> float:
         return float(self.enc_lens.sum()) * FRAME_SECONDS
 
+    def subset_lengths(self, rows) -> "Workload":
+        """Lengths only (no tensors) of the given utterances: enough for byte and flop accounting."""
+        rows = [int(r) for r in rows]
+        return dataclasses.replace(self, enc_lens=self.enc_lens[rows].copy(), dec_lens=self.dec_lens[rows].copy(),
+                                   durations=self.durations[rows].copy(), enc=None, weights=None)
+
     def subset(self, rows) -> "Workload":
         """The same model with only the given utterances (in the given order)."""
         rows = [int(r) for r in rows]

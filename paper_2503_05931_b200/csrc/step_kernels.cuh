@@ -370,6 +370,17 @@ template <> struct Raw8<__nv_bfloat16> {
     uint4 v;
     __device__ __forceinline__ void load(const __nv_bfloat16 *p) { v = *reinterpret_cast<const uint4 *>(p); }
     __device__ __forceinline__ void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
+    __device__ __forceinline__ void set(const float (&f)[8])          // rounds to bf16, as the cache stores it
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 pr = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&pr);
+        }
+        v = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __device__ __forceinline__ void store(__nv_bfloat16 *p) const { *reinterpret_cast<uint4 *>(p) = v; }
     __device__ __forceinline__ void get(float (&f)[8]) const
     {
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -381,6 +392,8 @@ template <> struct Raw8<float> {
     float4 a, b;
     __device__ __forceinline__ void load(const float *p) { a = *reinterpret_cast<const float4 *>(p); b = *reinterpret_cast<const float4 *>(p + 4); }
     __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+    __device__ __forceinline__ void set(const float (&f)[8]) { a = make_float4(f[0], f[1], f[2], f[3]); b = make_float4(f[4], f[5], f[6], f[7]); }
+    __device__ __forceinline__ void store(float *p) const { *reinterpret_cast<float4 *>(p) = a; *reinterpret_cast<float4 *>(p + 4) = b; }
     __device__ __forceinline__ void get(float (&f)[8]) const
     { f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w; }
 };
@@ -389,7 +402,7 @@ constexpr int kFusedChunk = 16;       // positions per warp and iteration
 constexpr int kFusedMaxWarps = 8;
 
 template <typename CT, bool kCross, bool kAppend>
-__global__ void __launch_bounds__(kFusedMaxWarps * 32, 4)
+__global__ void __launch_bounds__(kFusedMaxWarps * 32, (kAppend ? 2 : 4))      // self-attention holds the new key/value as well
 attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ q, int ldq,
                   CT *__restrict__ cache, int n_heads, int seq_capacity, float scale,
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo,
@@ -418,26 +431,29 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         kbase = cache + (((size_t)u * 2 + 0) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
         vbase = cache + (((size_t)u * 2 + 1) * n_heads + h) * (size_t)seq_capacity * kHeadDim;
     }
+    // Positions that earlier steps (or the precompute) wrote are static for this kernel; the position appended
+    // by this step (self-attention only) is taken from the projection output after the dependency wait.
+    const int len_static = (kAppend && !kCross) ? len - 1 : len;
+    const int dg = lane & 7, pg = lane >> 3;
     Raw8<CT> rk[4], rv[4];
-    if (kCross) {
-        // The encoder keys and values of this warp's first chunk start streaming while the kernel that produces
-        // the query is still running.
+    {
+        // This warp's first chunk starts streaming while the kernel that produces the query is still running.
         const int p0 = warp * kFusedChunk;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int p = p0 + i * 4 + (lane >> 3);
-            if (p < len) {
-                rk[i].load(kbase + (size_t)p * kHeadDim + (lane & 7) * 8);
-                rv[i].load(vbase + (size_t)p * kHeadDim + (lane & 7) * 8);
+            const int p = p0 + i * 4 + pg;
+            if (p < len_static) {
+                rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
+                rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
             } else { rk[i].zero(); rv[i].zero(); }
         }
         // later chunks of this warp: pull them into L2 now (one 128-byte row per lane group)
-        if ((lane & 7) == 0) {
-            for (int q0 = p0 + n_warps * kFusedChunk; q0 < len; q0 += n_warps * kFusedChunk) {
+        if (dg == 0) {
+            for (int q0 = p0 + n_warps * kFusedChunk; q0 < len_static; q0 += n_warps * kFusedChunk) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int p = q0 + i * 4 + (lane >> 3);
-                    if (p < len) {
+                    const int p = q0 + i * 4 + pg;
+                    if (p < len_static) {
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(kbase + (size_t)p * kHeadDim));
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(vbase + (size_t)p * kHeadDim));
                     }
@@ -448,57 +464,70 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     AED_TRACE_BEGIN(state, 3);
-    const int dg = lane & 7, pg = lane >> 3;
-    // When the projection ran on gamma*x (LayerNorm folded), its raw output y becomes rstd*(y - mean*c1) + c2 here.
+    // Everything this block needs from earlier kernels is requested in one round: statistics, query, and (in the
+    // warp that owns the new position) the new key and value, with the LayerNorm-fold constants of their columns.
+    // When the projection ran on gamma*x, its raw output y becomes rstd*(y - mean*c1) + c2 here.
+    const int new_chunk = (len - 1) / kFusedChunk;
+    const bool owns_new = kAppend && !kCross && warp == new_chunk % n_warps;
+    const int d_model = n_heads * kHeadDim;
+    const int qcol = h * kHeadDim + dg * 8;
     float2 st = make_float2(0.f, 1.f);
+    float qv[8], qc1[8], qc2[8], kn[8], vn[8], kc1[8], kc2[8], vc1[8], vc2[8];
     if (ln_stats) st = ln_stats[r];
-    if (kAppend && !kCross) {
-        if (warp == 0 && lane < 16) {
-            const int kv = lane >> 3, d_model = n_heads * kHeadDim;
-            const int col = (1 + kv) * d_model + h * kHeadDim + dg * 8;
-            float nv[8];
-            load8(q + (size_t)r * ldq + col, nv);
-            if (ln_stats) {
-                float c1[8], c2[8];
-                load8(ln_c1 + col, c1);
-                load8(ln_c2 + col, c2);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) nv[i] = fmaf(st.y, nv[i] - st.x * c1[i], c2[i]);
-            }
-            CT *dst = const_cast<CT *>(kv ? vbase : kbase) + (size_t)(len - 1) * kHeadDim + dg * 8;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = from_f32<CT>(nv[i]);
+    load8(q + (size_t)r * ldq + qcol, qv);
+    if (ln_stats) { load8(ln_c1 + qcol, qc1); load8(ln_c2 + qcol, qc2); }
+    if (owns_new) {
+        load8(q + (size_t)r * ldq + d_model + qcol, kn);
+        load8(q + (size_t)r * ldq + 2 * d_model + qcol, vn);
+        if (ln_stats) {
+            load8(ln_c1 + d_model + qcol, kc1); load8(ln_c2 + d_model + qcol, kc2);
+            load8(ln_c1 + 2 * d_model + qcol, vc1); load8(ln_c2 + 2 * d_model + qcol, vc2);
         }
-        __syncthreads();
     }
-    float qv[8];
-    load8(q + (size_t)r * ldq + h * kHeadDim + dg * 8, qv);
     if (ln_stats) {
-        float c1[8], c2[8];
-        load8(ln_c1 + h * kHeadDim + dg * 8, c1);
-        load8(ln_c2 + h * kHeadDim + dg * 8, c2);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * c1[i], c2[i]);
+        for (int i = 0; i < 8; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * qc1[i], qc2[i]);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) qv[i] *= scale;
+    Raw8<CT> new_k, new_v;
+    if (owns_new) {
+        if (ln_stats) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                kn[i] = fmaf(st.y, kn[i] - st.x * kc1[i], kc2[i]);
+                vn[i] = fmaf(st.y, vn[i] - st.x * vc1[i], vc2[i]);
+            }
+        }
+        new_k.set(kn);
+        new_v.set(vn);
+        if (pg == 0) {      // append to the cache; no other block reads this position during the kernel
+            new_k.store(const_cast<CT *>(kbase) + (size_t)(len - 1) * kHeadDim + dg * 8);
+            new_v.store(const_cast<CT *>(vbase) + (size_t)(len - 1) * kHeadDim + dg * 8);
+        }
+    }
 
     float m = -INFINITY, l = 0.f, acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    bool loaded = kCross;
+    bool loaded = true;
     for (int p0 = warp * kFusedChunk; p0 < len; p0 += n_warps * kFusedChunk) {
         if (!loaded) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {          // keys and values of the chunk are requested together
                 const int p = p0 + i * 4 + pg;
-                if (p < len) {
+                if (p < len_static) {
                     rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
                     rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
                 } else { rk[i].zero(); rv[i].zero(); }
             }
         }
         loaded = false;
+        if (owns_new && p0 == new_chunk * kFusedChunk) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (p0 + i * 4 + pg == len - 1) { rk[i] = new_k; rv[i] = new_v; }
+        }
         float s[4], cmax = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

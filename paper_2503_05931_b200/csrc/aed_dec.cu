@@ -305,10 +305,8 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
     if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
     if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
-    // Attention starts early and holds its first chunk in registers: with many rows, 4 warps per cross-attention
-    // block keep every block of the step resident at once (8 blocks per SM) and longer rows loop, finding their
-    // later chunks in L2; with few rows residency is no issue and 8 warps halve the number of passes.
-    if (kCross && warps > 4 && rows_ub > 32) warps = 4;
+    // Attention starts early (programmatic launch) and holds each warp's first chunk in registers; rows longer than
+    // 8 x 16 positions loop and find their later chunks prefetched in L2.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(rows_ub * dec->cfg.n_heads);
     cfg.blockDim = dim3(warps * 32);

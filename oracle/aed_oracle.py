@@ -55,6 +55,21 @@ def build(force: bool = False) -> None:
         os.replace(tmp, out)
 
 
+def load_custom(tag: str, path: str) -> None:
+    """Register another build of the checker under ``precision=tag`` (tests that plant mistakes use this)."""
+    lib = C.CDLL(path)
+    _set_signatures(lib)
+    _LIBS[tag] = lib
+
+
+def _set_signatures(lib: C.CDLL) -> None:
+    lib.orc_decode.restype = C.c_int
+    lib.orc_decode_full_recompute.restype = C.c_int
+    lib.orc_decode_batch.restype = C.c_int
+    lib.orc_argmax_f64.restype = C.c_int32
+    lib.orc_real_bytes.restype = C.c_int
+
+
 def _lib(precision: str) -> C.CDLL:
     if precision not in _LIBS:
         build()

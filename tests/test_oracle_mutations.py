@@ -1,0 +1,113 @@
+"""Do the pins bite?  Each case plants one plausible mistake in a copy of the checker's C source (a dropped
+term, a wrong sign or index, a transposed operand, a wrong constant), builds it, and demands that the pins
+that do not depend on the checker itself notice: agreement with torch.nn.TransformerDecoderLayer in fp64,
+incremental == full recompute, and the closed forms.  The mistakes live only in the temporary copy."""
+import math
+import os
+import subprocess
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import aed_oracle as orc
+from paper_2503_05931_b200 import workloads as wl
+
+SRC = os.path.join(os.path.dirname(orc.__file__), "aed_oracle.c")
+
+MUTATIONS = [
+    ("attention scale dropped", "real scale = (real)1 / (real)sqrt((double)dh);", "real scale = (real)1;"),
+    ("softmax without max subtraction sign", "score[j] = (real)exp((double)(score[j] - mx));", "score[j] = (real)exp((double)(mx - score[j]));"),
+    ("layernorm unbiased variance", "var /= (real)d;", "var /= (real)(d - 1);"),
+    ("layernorm eps outside sqrt", "real inv = (real)1 / (real)sqrt((double)var + eps);", "real inv = (real)1 / ((real)sqrt((double)var) + (real)eps);"),
+    ("embedding scale dropped", "double sq = sqrt((double)d);", "double sq = 1.0;"),
+    ("sin and cos swapped", "double pe = (i % 2 == 0) ? sin(angle) : cos(angle);", "double pe = (i % 2 == 0) ? cos(angle) : sin(angle);"),
+    ("position exponent uses i instead of the pair", "double angle = (double)t / pow(10000.0, (2.0 * pair) / (double)d);", "double angle = (double)t / pow(10000.0, (2.0 * i) / (double)d);"),
+    ("key and value blocks swapped", "memcpy(Kl + (size_t)t * d, qkv + d, sizeof(real) * d);\n            memcpy(Vl + (size_t)t * d, qkv + 2 * d, sizeof(real) * d);",
+     "memcpy(Kl + (size_t)t * d, qkv + 2 * d, sizeof(real) * d);\n            memcpy(Vl + (size_t)t * d, qkv + d, sizeof(real) * d);"),
+    ("self-attention misses the current position", "attend(qkv, Kl, Vl, t + 1, H, dh, s,", "attend(qkv, Kl, Vl, t > 0 ? t : 1, H, dh, s,"),
+    ("cross-attention residual dropped", "linear(w->w_o_c[l], BIAS(b_o_c, l), s, d, d, o);\n            for (int i = 0; i < d; ++i) x[i] += o[i];\n            /* feed-forward */",
+     "linear(w->w_o_c[l], BIAS(b_o_c, l), s, d, d, o);\n            for (int i = 0; i < d; ++i) x[i] = o[i];\n            /* feed-forward */"),
+    ("relu dropped", "for (int i = 0; i < F; ++i) if (hid[i] < 0) hid[i] = 0;", "for (int i = 0; i < F; ++i) if (hid[i] < -1e30) hid[i] = 0;"),
+    ("ffn uses ln2 parameters", "orc_layernorm(x, w->ln3_g[l], w->ln3_b[l], d, cfg->ln_eps, a);\n            linear(w->w_ff1[l]", "orc_layernorm(x, w->ln2_g[l], w->ln2_b[l], d, cfg->ln_eps, a);\n            linear(w->w_ff1[l]"),
+    ("weight matrix read transposed", "for (int i = 0; i < n_in; ++i) acc += (real)w[i] * x[i];\n        y[o] = acc;\n    }\n}\n\n/* same with a float input vector",
+     "for (int i = 0; i < n_in; ++i) acc += (real)W[(size_t)i * n_out + o] * x[i];\n        y[o] = acc;\n    }\n}\n\n/* same with a float input vector"),
+    ("heads read with the wrong stride", "for (int c = 0; c < dh; ++c) s += q[h * dh + c] * K[(size_t)j * d + h * dh + c];", "for (int c = 0; c < dh; ++c) s += q[h * dh + c] * K[(size_t)j * d + c * (d / dh) + h];"),
+    ("argmax prefers the highest index on ties", "for (int i = 1; i < n; ++i) if (z[i] > z[best]) best = i;", "for (int i = 1; i < n; ++i) if (z[i] >= z[best]) best = i;"),
+    ("cross values taken from the key block", "memcpy(Vc + (size_t)j * d, tmp + d, sizeof(real) * d);", "memcpy(Vc + (size_t)j * d, tmp, sizeof(real) * d);"),
+    ("incremental decoder forgets the final layernorm bias", "orc_layernorm(x, w->final_ln_g, w->final_ln_b, d, cfg->ln_eps, a);\n        linear(w->w_out, w->b_out, a, V, d, z);\n        if (logits) for (int v = 0; v < V; ++v) logits[(size_t)t * V + v] = (double)z[v];\n        tok =",
+     "orc_layernorm(x, w->final_ln_g, w->final_ln_g, d, cfg->ln_eps, a);\n        linear(w->w_out, w->b_out, a, V, d, z);\n        if (logits) for (int v = 0; v < V; ++v) logits[(size_t)t * V + v] = (double)z[v];\n        tok ="),
+]
+
+
+def _pos_enc(t, d):
+    pe = np.zeros(d)
+    for i in range(0, d, 2):
+        ang = t / (10000.0 ** (i / d))
+        pe[i], pe[i + 1] = math.sin(ang), math.cos(ang)
+    return pe
+
+
+def _pins(precision):
+    """The checker-independent pins on a small model; raises AssertionError if any fails."""
+    model = dict(n_layers=2, d_model=32, n_heads=4, d_ffn=48, vocab=29, d_enc=32)
+    w = wl.make_custom(model, [7], [6], seed=4, bias_std=0.3)
+    rng = np.random.default_rng(9)
+    d, NL = model["d_model"], model["n_layers"]
+    for name in ("ln1", "ln2", "ln3"):
+        w.weights[name + "_g"] = [rng.normal(1, 0.3, d).astype(np.float32) for _ in range(NL)]
+        w.weights[name + "_b"] = [rng.normal(0, 0.3, d).astype(np.float32) for _ in range(NL)]
+    w.weights["final_ln_g"] = rng.normal(1, 0.3, d).astype(np.float32)
+    w.weights["final_ln_b"] = rng.normal(0, 0.3, d).astype(np.float32)
+    for name in ("w_qkv", "w_o", "w_q_c", "w_kv_c", "w_o_c", "w_ff1", "w_ff2"):
+        w.weights[name] = [(a * 8).astype(np.float32) for a in w.weights[name]]
+    w.weights["w_out"][5] = w.weights["w_out"][17]          # a planted tie for the argmax rule
+    m = orc.Model(w.model, w.weights)
+    L = 6
+    forced = rng.integers(0, model["vocab"], size=L)
+    out = orc.decode(m, w.enc, L, forced=forced, precision=precision)
+    full = orc.decode(m, w.enc, L, forced=forced, precision=precision, full_recompute=True)
+    assert np.max(np.abs(out["logits"] - full["logits"])) <= 1e-12
+    t64 = lambda a: torch.tensor(np.asarray(a), dtype=torch.float64)
+    x = torch.stack([t64(w.weights["embed"][y]) * math.sqrt(d) + t64(_pos_enc(t, d)) for t, y in enumerate(forced)])[None]
+    mem = t64(w.enc)[None]
+    mask = torch.nn.Transformer.generate_square_subsequent_mask(L, dtype=torch.float64)
+    with torch.no_grad():
+        for l in range(NL):
+            lay = torch.nn.TransformerDecoderLayer(d, model["n_heads"], model["d_ffn"], dropout=0.0, activation="relu",
+                                                   batch_first=True, norm_first=True, dtype=torch.float64)
+            lay.self_attn.in_proj_weight.copy_(t64(w.weights["w_qkv"][l])); lay.self_attn.in_proj_bias.copy_(t64(w.weights["b_qkv"][l]))
+            lay.self_attn.out_proj.weight.copy_(t64(w.weights["w_o"][l])); lay.self_attn.out_proj.bias.copy_(t64(w.weights["b_o"][l]))
+            lay.multihead_attn.in_proj_weight.copy_(t64(np.concatenate([w.weights["w_q_c"][l], w.weights["w_kv_c"][l]])))
+            lay.multihead_attn.in_proj_bias.copy_(t64(np.concatenate([w.weights["b_q_c"][l], w.weights["b_kv_c"][l]])))
+            lay.multihead_attn.out_proj.weight.copy_(t64(w.weights["w_o_c"][l])); lay.multihead_attn.out_proj.bias.copy_(t64(w.weights["b_o_c"][l]))
+            lay.linear1.weight.copy_(t64(w.weights["w_ff1"][l])); lay.linear1.bias.copy_(t64(w.weights["b_ff1"][l]))
+            lay.linear2.weight.copy_(t64(w.weights["w_ff2"][l])); lay.linear2.bias.copy_(t64(w.weights["b_ff2"][l]))
+            for i, nm in ((1, "ln1"), (2, "ln2"), (3, "ln3")):
+                getattr(lay, f"norm{i}").weight.copy_(t64(w.weights[nm + "_g"][l]))
+                getattr(lay, f"norm{i}").bias.copy_(t64(w.weights[nm + "_b"][l]))
+            x = lay.eval()(x, mem, tgt_mask=mask)
+        x = torch.nn.functional.layer_norm(x, (d,), t64(w.weights["final_ln_g"]), t64(w.weights["final_ln_b"]), 1e-5)
+        z = (x @ t64(w.weights["w_out"]).T)[0].numpy()
+    np.testing.assert_allclose(out["logits"], z, atol=1e-10)
+    assert not np.any(out["next"] == 17)                    # ties go to the lowest index
+    idx, _ = orc.argmax(np.array([1.0, 3.0, 3.0, 2.0]), precision=precision)
+    assert idx == 1
+
+
+def test_pins_pass_on_the_real_checker():
+    _pins("f64")
+
+
+@pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_planted_mistake_is_caught(tmp_path, name, old, new):
+    src = open(SRC).read()
+    assert src.count(old) >= 1, f"snippet of '{name}' not found in the checker source"
+    mutated = tmp_path / "mut.c"
+    mutated.write_text(src.replace(old, new, 1))
+    lib = tmp_path / "libmut.so"
+    subprocess.run(["gcc", "-O1", "-std=c11", "-fPIC", "-shared", "-fopenmp", str(mutated), "-o", str(lib), "-lm"], check=True)
+    tag = "mut_" + name
+    orc.load_custom(tag, str(lib))
+    with pytest.raises(AssertionError):
+        _pins(tag)

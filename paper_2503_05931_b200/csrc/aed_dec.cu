@@ -16,6 +16,7 @@
 #include "step_kernels.cuh"
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
+#include "cluster_step.cuh"
 
 using namespace aed;
 
@@ -49,6 +50,7 @@ struct Layout {
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
     size_t actd_hi, actd_lo, actf_hi, actf_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
+    size_t x1, x2;                        // the other two buffers of the rotating residual stream (cluster path)
     size_t fold_layer_floats;
     int rows_cap;
 };
@@ -117,6 +119,8 @@ Layout make_layout(const aed_dec_config_t &c)
         L.fold_c = take(L.fold_layer_floats * c.n_layers * 4);
         L.ln_stats = take((size_t)3 * rows_bucket(c.max_batch) * 8);
         L.qc = take(B * d * 4);
+        L.x1 = take(B * d * 4);
+        L.x2 = take(B * d * 4);
     }
     L.total = off;
     return L;
@@ -149,6 +153,9 @@ struct aed_dec {
     size_t prof_used = 0;
     // bf16 mode: TMA descriptors of the weight matrices and of the activation planes (one per MMA N in 16..256)
     struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2, kvc; };
+    struct ClLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };      // boxes of 64 rows x 64 k
+    std::vector<ClLayerMaps> cl_layers;
+    bool use_cluster = false;             // head-parallel cluster kernels for steps of at most 64 rows
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
     CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]
@@ -202,10 +209,11 @@ aed_status_t fail(aed_dec *d, aed_status_t code, const char *fmt, ...)
 
 enum KernelFamily { KF_BOOKKEEPING = 0, KF_EMBED, KF_LAYERNORM, KF_GEMM_QKV, KF_ATTN_SELF, KF_ATTN_COMBINE, KF_GEMM_O,
                     KF_GEMM_QC, KF_ATTN_CROSS, KF_GEMM_OC, KF_GEMM_FF1, KF_GEMM_FF2, KF_GEMM_VOCAB, KF_PRECOMPUTE,
-                    KF_COUNT };
+                    KF_BLOCK_SELF, KF_BLOCK_CROSS, KF_BLOCK_FFN, KF_COUNT };
 const char *const kFamilyNames[KF_COUNT] = {"bookkeeping", "embed", "layernorm", "gemm_qkv", "attn_self", "attn_combine",
                                             "gemm_o", "gemm_qc", "attn_cross", "gemm_oc", "gemm_ff1", "gemm_ff2",
-                                            "gemm_vocab", "precompute_cross_kv"};
+                                            "gemm_vocab", "precompute_cross_kv", "block_self", "block_cross",
+                                            "block_ffn"};
 
 // Records an event before and after the launches issued while it is alive (profiling mode only).
 struct ProfScope {
@@ -493,6 +501,36 @@ aed_status_t tc_setup(aed_dec *dec)
     dec->act_planes = (planes && planes[0] == '1') ? 1 : 2;
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
     if (ctas && atoi(ctas) > 0) dec->tc_target_ctas = atoi(ctas);
+    // head-parallel cluster path: shapes whose projections split evenly over 8 CTAs and 16 clusters
+    {
+        const char *v = getenv("AED_DEC_NO_CLUSTER");
+        const bool want = !(v && v[0] == '1');
+        const bool shape_ok = (d == 512 || d == 1024) && c.n_heads <= cl::kClusters && F % 256 == 0 &&
+                              F / 256 <= (size_t)cl::kClusters;
+        if (want && shape_ok && dec->use_fused) {
+            dec->cl_layers.resize(c.n_layers);
+            bool ok2 = true;
+            for (int l = 0; l < c.n_layers; ++l) {
+                const LayerWeights &w = dec->layers[l];
+                aed_dec::ClLayerMaps &m = dec->cl_layers[l];
+                ok2 = ok2 && encode_map(&m.qkv, w.w_qkv, 3 * d, d, 64) && encode_map(&m.o, w.w_o, d, d, 64) &&
+                      encode_map(&m.qc, w.w_q_c, d, d, 64) && encode_map(&m.oc, w.w_o_c, d, d, 64) &&
+                      encode_map(&m.ff1, w.w_ff1, F, d, 64) && encode_map(&m.ff2, w.w_ff2, d, F, 64);
+            }
+            if (!ok2) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the cluster path");
+            const int kbs = (int)d / cl::kCS / tc::kBlockK;
+            cudaError_t e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_SELF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                  cl::cl_layout(cl::K_SELF, cl::kMaxRows, kbs).total + 1024);
+            if (e2 == cudaSuccess)
+                e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_CROSS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          cl::cl_layout(cl::K_CROSS, cl::kMaxRows, kbs).total + 1024);
+            if (e2 == cudaSuccess)
+                e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_FFN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          cl::cl_layout(cl::K_FFN, cl::kMaxRows, kbs).total + 1024);
+            if (e2 != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "cluster path set-up: %s", cudaGetErrorString(e2));
+            dec->use_cluster = true;
+        }
+    }
     dec->use_tc = true;
     return AED_OK;
 }
@@ -752,6 +790,97 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
     return AED_OK;
 }
 
+// ---- head-parallel cluster step (bf16 mode, at most 64 rows): 3 cluster kernels per layer ----------------------
+
+template <int KIND>
+aed_status_t launch_cluster_block(aed_dec *dec, int family, const CUtensorMap &map_w1, const CUtensorMap &map_w2,
+                                  int rows_ub, cl::ClusterParams p)
+{
+    ProfScope ps(dec, family);
+    const auto &c = dec->cfg;
+    p.d = c.d_model; p.n_heads = c.n_heads; p.d_ffn = c.d_ffn;
+    p.n_tile = 16 << tc_n_index(rows_ub);
+    p.row_info = dec->at<int4>(dec->lay.row_info);
+    p.scale = 1.0f / sqrtf((float)kHeadDim);
+    p.eps = c.ln_eps;
+    p.state = dec->state();
+    const int kbs = c.d_model / cl::kCS / tc::kBlockK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cl::kClusters * cl::kCS);
+    cfg.blockDim = dim3(cl::kClThreads);
+    cfg.dynamicSmemBytes = (size_t)cl::cl_layout(KIND, p.n_tile, kbs).total + 1024;
+    cfg.stream = dec->stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, cl::cluster_block_kernel<KIND>, map_w1, map_w2, p);
+    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "cluster block launch: %s", cudaGetErrorString(e));
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
+aed_status_t forward_step_cluster(aed_dec *dec, int rows_ub, const int32_t *tokens, float *logits_out)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const int d = c.d_model, F = c.d_ffn, V = c.vocab;
+    float *xb[3] = {dec->at<float>(L.x), dec->at<float>(L.x1), dec->at<float>(L.x2)};
+    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
+    {
+        ProfScope ps(dec, KF_EMBED);
+        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), xb[0], xb[1], d);
+        AED_LAUNCHED(dec);
+    }
+    const size_t e2 = sizeof(T);
+    int blk = 0;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        const aed_dec::ClLayerMaps &m = dec->cl_layers[l];
+        const int ln = (l + 1) % c.n_layers;               // next layer (or layer 0 of the next step)
+        const LayerWeights &wn = dec->layers[ln];
+        T *self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
+        T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+        const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
+        cl::ClusterParams p{};
+        // self-attention block; the next block streams the cross-attention weights and this layer's encoder K/V
+        p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3]; ++blk;
+        p.gamma = (const T *)w.ln1_g; p.c1 = fc; p.c2 = fc + 3 * d; p.bias2 = (const T *)w.b_o;
+        p.cache = self_cache; p.seq_capacity = c.max_dec_len;
+        p.pf_ptr[0] = w.w_q_c; p.pf_bytes[0] = (size_t)d * d * e2; p.pf_ptr[1] = w.w_o_c; p.pf_bytes[1] = (size_t)d * d * e2;
+        p.pf_cache = cross; p.pf_capacity = c.max_total_enc_frames; p.pf_cross = 1;
+        AED_TRY(launch_cluster_block<cl::K_SELF>(dec, KF_BLOCK_SELF, m.qkv, m.o, rows_ub, p));
+        // cross-attention block; next: the feed-forward weights
+        p = cl::ClusterParams{};
+        p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3]; ++blk;
+        p.gamma = (const T *)w.ln2_g; p.c1 = fc + 6 * d; p.c2 = fc + 7 * d; p.bias2 = (const T *)w.b_o_c;
+        p.cache = cross; p.seq_capacity = c.max_total_enc_frames;
+        p.pf_ptr[0] = w.w_ff1; p.pf_bytes[0] = (size_t)F * d * e2; p.pf_ptr[1] = w.w_ff2; p.pf_bytes[1] = (size_t)F * d * e2;
+        AED_TRY(launch_cluster_block<cl::K_CROSS>(dec, KF_BLOCK_CROSS, m.qc, m.oc, rows_ub, p));
+        // feed-forward block; next: the self-attention weights and cache of the next layer
+        p = cl::ClusterParams{};
+        p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3]; ++blk;
+        p.gamma = (const T *)w.ln3_g; p.c1 = fc + 8 * d; p.c2 = fc + 8 * d + F; p.bias2 = (const T *)w.b_ff2;
+        p.pf_ptr[0] = wn.w_qkv; p.pf_bytes[0] = (size_t)3 * d * d * e2; p.pf_ptr[1] = wn.w_o; p.pf_bytes[1] = (size_t)d * d * e2;
+        p.pf_cache = dec->at<T>(L.self_cache) + (size_t)ln * L.self_layer_elems; p.pf_capacity = c.max_dec_len; p.pf_cross = 0;
+        AED_TRY(launch_cluster_block<cl::K_FFN>(dec, KF_BLOCK_FFN, m.ff1, m.ff2, rows_ub, p));
+    }
+    // 3 blocks per layer: the result is back in the first buffer
+    AED_TRY(launch_ln_planes(dec, rows_ub, xb[0], dec->final_ln_g, dec->final_ln_b, nullptr, 0));
+    tc::TcParams tp{};
+    tp.bias = (const T *)dec->b_out;
+    tp.logits_out = logits_out;
+    tp.keys = dec->at<unsigned long long>(L.keys);
+    tp.active_list = active_list;
+    AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, tp));
+    return AED_OK;
+}
+
 // Cross K/V of every layer on tensor cores: D[frame, feature] = enc[frame, :] . w_kv_c[feature, :]
 aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
 {
@@ -967,7 +1096,8 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_build_active(dec, active));
     const int rows_ub = dec->batch;
     const int self_len_ub = dec->steps_issued + 1 < dec->cfg.max_dec_len ? dec->steps_issued + 1 : dec->cfg.max_dec_len;
-    aed_status_t s = dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out) : forward_step_tc(dec, rows_ub, self_len_ub, tokens_in, logits_out))
+    aed_status_t s = (dec->use_cluster && rows_ub <= cl::kMaxRows) ? forward_step_cluster(dec, rows_ub, tokens_in, logits_out)
+                     : dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out) : forward_step_tc(dec, rows_ub, self_len_ub, tokens_in, logits_out))
                      : dec->cfg.dtype == AED_DTYPE_BF16
                          ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tokens_in, logits_out)
                          : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
@@ -1040,7 +1170,8 @@ aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int
     if (self_len_ub > dec->cfg.max_dec_len) self_len_ub = dec->cfg.max_dec_len;
     AED_TRY(launch_build_active(dec, nullptr));
     const int32_t *tok = dec->at<int32_t>(L.cur_tok);
-    aed_status_t st = dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr) : forward_step_tc(dec, rows_ub, self_len_ub, tok, nullptr))
+    aed_status_t st = (dec->use_cluster && rows_ub <= cl::kMaxRows) ? forward_step_cluster(dec, rows_ub, tok, nullptr)
+                      : dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr) : forward_step_tc(dec, rows_ub, self_len_ub, tok, nullptr))
                       : dec->cfg.dtype == AED_DTYPE_BF16 ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tok, nullptr)
                                                          : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
     if (st != AED_OK) return st;

@@ -223,3 +223,55 @@ def test_config2_shape_sampled_rows():
     # keep the checker's work bounded: drop sampled rows longer than 40 tokens
     rows = [r for r in rows if w.dec_lens[r] <= 40][:4]
     _run_both(w, rows=rows)
+
+
+# ---- head-parallel cluster path (bf16, d_model 512 or 1024, at most 64 rows per step) -----------------------------
+
+CLUSTER_A = dict(n_layers=2, d_model=512, n_heads=8, d_ffn=1024, vocab=600, d_enc=256)     # 8 heads, 4 hidden chunks
+CLUSTER_B = dict(n_layers=1, d_model=1024, n_heads=16, d_ffn=768, vocab=520, d_enc=128)    # 16 heads, 3 hidden chunks
+
+
+@pytest.mark.parametrize("batch", [1, 7, 16, 17, 40, 64])
+def test_cluster_path_row_counts(batch):
+    """Every MMA row-tile width of the cluster kernels (16, 32, 64), with partly filled tiles, ragged encoder
+    lengths from 1 frame to several attention chunks, and rows retiring at different steps."""
+    rng = np.random.default_rng(900 + batch)
+    enc_lens = rng.integers(1, 150, size=batch)
+    dec_lens = rng.integers(1, 24, size=batch)
+    enc_lens[0], dec_lens[0] = 1, 40              # one frame; longer than two 16-position chunks of the self cache
+    w = wl.make_custom(CLUSTER_A, enc_lens, dec_lens, dtype="bf16", seed=300 + batch)
+    rows = sorted({0, batch - 1, batch // 2, int(np.argmax(enc_lens))})
+    _run_both(w, rows=rows)
+
+
+def test_cluster_path_d1024():
+    rng = np.random.default_rng(31)
+    batch = 24
+    w = wl.make_custom(CLUSTER_B, rng.integers(1, 200, size=batch), rng.integers(1, 20, size=batch), dtype="bf16", seed=77)
+    _run_both(w, rows=[0, 5, 23])
+
+
+def test_cluster_path_matches_kernel_chain(monkeypatch):
+    """The cluster kernels and the one-kernel-per-projection path compute the same step: logits of both agree far
+    inside the tolerance against the checker (both keep two bf16 planes of every activation)."""
+    import torch
+    b = _binding()
+    rng = np.random.default_rng(5)
+    batch = 33
+    w = wl.make_custom(CLUSTER_A, rng.integers(1, 120, size=batch), [6] * batch, dtype="bf16", seed=9)
+    outs = []
+    for no_cluster in ("0", "1"):
+        monkeypatch.setenv("AED_DEC_NO_CLUSTER", no_cluster)
+        dec = b.decoder_for_workload(w)
+        dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
+        logits = torch.zeros((batch, CLUSTER_A["vocab"]), dtype=torch.float32, device="cuda:0")
+        toks = torch.full((batch,), 1, dtype=torch.int32, device="cuda:0")
+        rec = []
+        for t in range(6):
+            dec.step(toks, None, logits, None)
+            toks.fill_(2 + t)
+            rec.append(logits.cpu().numpy().copy())
+        dec.sync_status()
+        dec.close()
+        outs.append(np.stack(rec))
+    assert np.max(np.abs(outs[0] - outs[1])) < 2e-3

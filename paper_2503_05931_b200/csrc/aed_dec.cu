@@ -1,6 +1,7 @@
 // Host side of the AED decoder library: handle, workspace layout, launch sequences, C ABI.
 #include "../../include/aed_dec.h"
 
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -156,6 +157,7 @@ struct aed_dec {
     struct ClLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };      // boxes of 64 rows x 64 k
     std::vector<ClLayerMaps> cl_layers;
     bool use_cluster = false;             // head-parallel cluster kernels for steps of at most 64 rows
+    int cl_prefetch = 3;                  // bit 0: next block's weights, bit 1: next block's K/V rows (L2 prefetch)
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
     CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]
@@ -503,10 +505,11 @@ aed_status_t tc_setup(aed_dec *dec)
     if (ctas && atoi(ctas) > 0) dec->tc_target_ctas = atoi(ctas);
     // head-parallel cluster path: shapes whose projections split evenly over 8 CTAs and 16 clusters
     {
-        const char *v = getenv("AED_DEC_NO_CLUSTER");
-        const bool want = !(v && v[0] == '1');
-        const bool shape_ok = (d == 512 || d == 1024) && c.n_heads <= cl::kClusters && F % 256 == 0 &&
-                              F / 256 <= (size_t)cl::kClusters;
+        // opt-in until it beats the kernel-per-projection path at every row count
+        const char *v = getenv("AED_DEC_CLUSTER");
+        const bool want = v && v[0] == '1';
+        const bool shape_ok = (d == 512 || d == 1024) && c.n_heads <= cl::kClusters / 2 && F % 128 == 0 &&
+                              F / 128 <= (size_t)cl::kClusters;
         if (want && shape_ok && dec->use_fused) {
             dec->cl_layers.resize(c.n_layers);
             bool ok2 = true;
@@ -519,16 +522,43 @@ aed_status_t tc_setup(aed_dec *dec)
             }
             if (!ok2) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the cluster path");
             const int kbs = (int)d / cl::kCS / tc::kBlockK;
+            auto max_smem = [&](int kind) {
+                int m = 0;
+                for (int n = 16; n <= cl::kMaxRows; n <<= 1) m = std::max(m, cl::cl_layout(kind, n, kbs).total + 1024);
+                return m;
+            };
             cudaError_t e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_SELF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                  cl::cl_layout(cl::K_SELF, cl::kMaxRows, kbs).total + 1024);
+                                                  max_smem(cl::K_SELF));
             if (e2 == cudaSuccess)
                 e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_CROSS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          cl::cl_layout(cl::K_CROSS, cl::kMaxRows, kbs).total + 1024);
+                                          max_smem(cl::K_CROSS));
             if (e2 == cudaSuccess)
                 e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_FFN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          cl::cl_layout(cl::K_FFN, cl::kMaxRows, kbs).total + 1024);
+                                          max_smem(cl::K_FFN));
             if (e2 != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "cluster path set-up: %s", cudaGetErrorString(e2));
-            dec->use_cluster = true;
+            // All clusters of a launch must be resident at once, or the launch runs in two waves and loses more
+            // than the path gains: ask the device (the answer depends on how many SMs each GPC of this chip has).
+            bool resident = true;
+            for (int kind = 0; kind < 3 && resident; ++kind) {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(cl::kClusters * cl::kCS);
+                cfg.blockDim = dim3(cl::kClThreads);
+                cfg.dynamicSmemBytes = (size_t)max_smem(kind);
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                int n = 0;
+                cudaError_t e3 = kind == 0   ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_SELF>, &cfg)
+                                 : kind == 1 ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_CROSS>, &cfg)
+                                             : cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_FFN>, &cfg);
+                if (e3 != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+                resident = n >= cl::kClusters;
+            }
+            dec->use_cluster = resident;
+            const char *pf = getenv("AED_DEC_CL_PREFETCH");
+            if (pf) dec->cl_prefetch = atoi(pf);
         }
     }
     dec->use_tc = true;
@@ -804,6 +834,8 @@ aed_status_t launch_cluster_block(aed_dec *dec, int family, const CUtensorMap &m
     p.scale = 1.0f / sqrtf((float)kHeadDim);
     p.eps = c.ln_eps;
     p.state = dec->state();
+    if (!(dec->cl_prefetch & 1)) p.pf_ptr[0] = p.pf_ptr[1] = nullptr;
+    if (!(dec->cl_prefetch & 2)) p.pf_cache = nullptr;
     const int kbs = c.d_model / cl::kCS / tc::kBlockK;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cl::kClusters * cl::kCS);
@@ -1295,6 +1327,27 @@ extern "C" int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, co
 }
 
 #ifdef AED_TRACE
+// Debug builds only: how many clusters of a block kernel the device holds at once (row tile n_tile).
+extern "C" int32_t aed_dec_cluster_occupancy(aed_dec_t *dec, int32_t kind, int32_t n_tile)
+{
+    if (!dec || !dec->use_cluster) return -1;
+    const int kbs = dec->cfg.d_model / cl::kCS / tc::kBlockK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cl::kClusters * cl::kCS);
+    cfg.blockDim = dim3(cl::kClThreads);
+    cfg.dynamicSmemBytes = (size_t)cl::cl_layout(kind, n_tile, kbs).total + 1024;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = -1;
+    cudaError_t e = kind == 0   ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_SELF>, &cfg)
+                    : kind == 1 ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_CROSS>, &cfg)
+                                : cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_FFN>, &cfg);
+    return e == cudaSuccess ? n : -2;
+}
+
 // Debug builds only: copy out the device-side start-time trace (ids and nanosecond stamps) and clear it.
 extern "C" int32_t aed_dec_trace_read(aed_dec_t *dec, int32_t max_events, uint32_t *ids, unsigned long long *t_ns)
 {

@@ -5,30 +5,35 @@
 // Everything between two such places can be split over attention heads (or over slices of the FFN hidden layer)
 // without any exchange between the parts, so a layer is run as three "blocks":
 //
-//   K_SELF   x_out = x_in + Wo  . selfattn (LN1(x_in))      cluster c = head c
-//   K_CROSS  x_out = x_in + Woc . crossattn(LN2(x_in))      cluster c = head c
-//   K_FFN    x_out = x_in + W2 . relu(W1 . LN3(x_in) + b1) + b2      cluster c = hidden features 256c .. 256c+255
+//   K_SELF   x_out = x_in + Wo  . selfattn (LN1(x_in))      cluster = (head, rows of one parity)
+//   K_CROSS  x_out = x_in + Woc . crossattn(LN2(x_in))      cluster = (head, rows of one parity)
+//   K_FFN    x_out = x_in + W2 . relu(W1 . LN3(x_in) + b1) + b2      cluster = 128 hidden features, all rows
 //
-// Each block is one launch of 16 clusters of 8 CTAs.  Inside a cluster the 8 CTAs split the contraction dimension
-// of the first projection (K = d_model, d/8 columns each) and the output features of the second one (d/8 each);
-// partial results travel through distributed shared memory:
+// Each block is one launch of 32 clusters of 4 CTAs (a B200 holds 36 such clusters at once, but only 15 clusters
+// of 8).  Inside a cluster the 4 CTAs split the contraction dimension of the first projection (K = d_model, d/4
+// columns each) and the output features of the second one (d/4 each); partial results travel through distributed
+// shared memory:
 //
-//   1. every CTA loads its d/8 columns of x_in for all rows, folds the LayerNorm scale in (gamma*x, bf16 high and
-//      low planes) and computes the (mean, M2) of its slice of every row;
+//   1. every CTA loads its d/4 columns of x_in for the cluster's rows, folds the LayerNorm scale in (gamma*x, bf16
+//      high and low planes) and computes the (mean, M2) of its slice of every row;
 //   2. tcgen05.mma: partial[feature, row] over the CTA's K slice (weights are the A operand, fetched by TMA before
 //      the dependency wait because they are static);
-//   3. the partials are scattered to the CTA that owns the row (attention blocks: row r belongs to CTA r mod 8) or
-//      the hidden feature (FFN: 32 features per CTA), together with the slice statistics; an mbarrier with
+//   3. the partials are scattered to the CTA that owns the row (attention blocks: local row l belongs to CTA l mod 4)
+//      or the hidden feature (FFN: 32 features per CTA), together with the slice statistics; an mbarrier with
 //      cluster-scope release/acquire marks the end of the exchange;
-//   4. the owner sums the 8 partials, finishes the LayerNorm (rstd*(raw - mean*c1) + c2, see step_gemm.cuh) and
+//   4. the owner sums the 4 partials, finishes the LayerNorm (rstd*(raw - mean*c1) + c2, see step_gemm.cuh) and
 //      runs attention for its rows over the ragged cache (or applies ReLU), then writes the result as bf16 planes
-//      straight into the B-operand tile of all 8 CTAs;
-//   5. tcgen05.mma of the second projection over the head's 64 (or the chunk's 256) input features, d/8 output
-//      features per CTA, and red.global.add of the partial into x_out, which was cleared by an earlier block.
+//      straight into the B-operand tile of all 4 CTAs;
+//   5. tcgen05.mma of the second projection over the head's 64 (or the chunk's 128) input features, d/4 output
+//      features per CTA, and 16-byte red.global.add of the partial into x_out, which an earlier block cleared.
 //
 // x rotates through three buffers (read, accumulate, clear) so that a fast cluster can never add into rows that a
 // slow cluster of the same launch still reads.  Only the sum over heads / hidden chunks goes through global
 // memory: three exchanges per layer instead of eight.
+//
+// Attention inside a CTA: the 16-position chunks of its rows form one list that is dealt to the 8 worker warps in
+// equal contiguous runs; each warp streams its chunks through a ring in shared memory filled by bulk async copies
+// (the first stages before the dependency wait, since cached keys and values are static during a step).
 //
 // Every wait is bounded; a CTA that gives up still performs all its cluster arrivals, so that its peers do not
 // wait for it, and raises the error word of the decode state.
@@ -41,12 +46,15 @@ namespace cl {
 
 using namespace tc;
 
-constexpr int kCS = 8;               // CTAs per cluster
-constexpr int kClusters = 16;
+constexpr int kCS = 4;               // CTAs per cluster
+constexpr int kClusters = 32;
 constexpr int kClThreads = 384;      // warp 0 TMA, warp 1 MMA, warps 2..9 workers, warps 10..11 side jobs
 constexpr int kSlot = 16384;         // one weight tile: 128 rows x 64 k, bf16
-constexpr int kMaxTiles = 8;
+constexpr int kMaxTiles = 10;
+constexpr int kMaxRing = 4;
 constexpr int kMaxRows = 64;
+constexpr int kMaxSlots = 8;         // rows of one CTA in an attention block
+constexpr int kFfnSlots = 7;         // weight slots of the FFN block
 constexpr int kTmemCols = 256;
 
 enum Kind { K_SELF = 0, K_CROSS = 1, K_FFN = 2 };
@@ -71,24 +79,56 @@ struct ClusterParams {
 };
 
 struct ClSmem {
-    int n_slots, w_off, recv_off, r2_off, ap_off, stats_off, total;
+    int recv_off, r2_off, ap_off, stats_off, tab_off, ring_off, ring_stages, total;
 };
 
-// Dynamic shared memory of one block kind: weight slots | receive buffer | operand planes | attention planes | stats
+constexpr int kRingStage = 4096;                // 16 positions: keys 2 KB | values 2 KB
+constexpr int kPartStride = 68;                 // floats per attention partial: max, sum, pad, pad, 64 accumulators
+constexpr int kDynSmemCap = 232448 - 3072;      // what a CTA may take, less the static part of the kernel
+
+// MMA N of a block: the attention blocks see every second row of the step
+__host__ __device__ inline int cl_mma_n(int kind, int n_tile) { return kind == K_FFN ? n_tile : (n_tile / 2 < 16 ? 16 : n_tile / 2); }
+
+// Byte offset of weight tile t in the weight area (kbs = k-blocks of the CTA's K slice, mt2 = 128-row tiles of its
+// output features).  Tiles of 64 rows take 8 KB; the MMA reads 128 rows from the tile base whatever follows it
+// (rows 64..127 only feed accumulator lanes nobody reads).
+//   K_SELF : per k-block  query|key rows 16 KB, value rows 8 KB; the output-projection tiles later reuse the
+//            query|key areas of the first k-blocks
+//   K_CROSS: query tiles 8 KB each, then the output-projection tiles
+//   K_FFN  : 7 slots of 16 KB, tile t in slot t mod 7
+__host__ __device__ inline int cl_tile_off(int kind, int t, int kbs)
+{
+    if (kind == K_SELF) return t < 2 * kbs ? (t >> 1) * 24576 + (t & 1) * 16384 : (t - 2 * kbs) * 24576;
+    if (kind == K_CROSS) return t < kbs ? t * 8192 : kbs * 8192 + (t - kbs) * kSlot;
+    return (t % kFfnSlots) * kSlot;
+}
+
+// Dynamic shared memory of one block kind:
+// weight tiles | receive buffer (later: attention partials) | operand planes | attention planes | statistics |
+// attention tables | K/V ring (8 warps x stages x 4 KB)
 __host__ __device__ inline ClSmem cl_layout(int kind, int n_tile, int kbs)
 {
     ClSmem s;
-    const int tiles = kind == K_SELF ? 2 * kbs + 1 : kind == K_CROSS ? kbs + 1 : 2 * kbs + 4;
-    s.n_slots = tiles < 5 ? tiles : 5;
-    const int recv = kind == K_SELF ? n_tile * 768 : kind == K_CROSS ? n_tile * 256 : n_tile * 1024;
-    const int r2 = kind == K_FFN ? n_tile * 1024 : kbs * 2 * n_tile * 128;
-    const int ap = kind == K_FFN ? 0 : 2 * n_tile * 128;
-    s.w_off = 0;
-    s.recv_off = s.w_off + s.n_slots * kSlot;
+    const int mt2 = kbs / 2, nm = cl_mma_n(kind, n_tile);
+    const int tiles_ffn = kbs + 2 * mt2;
+    const int w_bytes = kind == K_SELF ? kbs * 24576 : kind == K_CROSS ? kbs * 8192 + mt2 * kSlot
+                                                                        : (tiles_ffn < kFfnSlots ? tiles_ffn : kFfnSlots) * kSlot;
+    int recv = kind == K_SELF ? n_tile * 384 : kind == K_CROSS ? n_tile * 272 : n_tile * 512;
+    recv = (recv + 1023) / 1024 * 1024;
+    const int r2 = kbs * 2 * nm * 128;
+    const int ap = kind == K_FFN ? 0 : 2 * nm * 128;
+    s.recv_off = w_bytes;
     s.r2_off = s.recv_off + recv;
     s.ap_off = s.r2_off + r2;
     s.stats_off = s.ap_off + ap;
-    s.total = s.stats_off + kCS * kMaxRows * 8;
+    s.tab_off = s.stats_off + kCS * kMaxRows * 8;
+    s.ring_off = s.tab_off + (kind == K_FFN ? 0 : 5120);
+    s.ring_stages = 0;
+    if (kind != K_FFN) {
+        int st = (kDynSmemCap - s.ring_off - 1024) / (8 * kRingStage);
+        s.ring_stages = st < 1 ? 1 : st > kMaxRing ? kMaxRing : st;
+    }
+    s.total = s.ring_off + s.ring_stages * 8 * kRingStage;
     return s;
 }
 
@@ -155,9 +195,15 @@ __device__ __forceinline__ void cluster_sync_all()
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// contiguous global -> shared copy by the async engine; completes on an mbarrier of this CTA
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-// (mean, rstd) of a row from the (mean, M2) of its 8 equally long slices
+// (mean, rstd) of a row from the (mean, M2) of its equally long slices, one per CTA of the cluster
 __device__ __forceinline__ float2 merge_stats(const float2 *slices, int stride, int ks, int d, float eps)
 {
     float2 s[kCS];
@@ -171,7 +217,7 @@ __device__ __forceinline__ float2 merge_stats(const float2 *slices, int stride, 
     return make_float2(mean, rsqrtf(m2 / d + eps));
 }
 
-// grid: 128 CTAs = 16 clusters of 8.  map_w1 / map_w2: weight matrices of the first and second projection,
+// grid: 128 CTAs = 32 clusters of 4.  map_w1 / map_w2: weight matrices of the first and second projection,
 // boxes of 64 rows x 64 k.
 template <int KIND>
 __global__ void __launch_bounds__(kClThreads, 1)
@@ -183,34 +229,45 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float sm_c1[192], sm_c2[192];
-    __shared__ float sm_m[8], sm_l[8];
-    __shared__ __align__(16) float sm_acc[8][kHeadDim];
+    __shared__ __align__(8) uint64_t ring_bar[8][kMaxRing];   // K/V ring of each worker warp
+    __shared__ const __nv_bfloat16 *sm_kptr[kMaxSlots], *sm_vptr[kMaxSlots];      // per row slot of this CTA
+    __shared__ int sm_len[kMaxSlots], sm_lenst[kMaxSlots], sm_cum[kMaxSlots + 1];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = static_cast<int>(cluster_ctarank());
     const int c = static_cast<int>(cluster_index());
-    const int d = p.d, ks = d / kCS, kbs = ks / kBlockK, of = ks;
+    const int d = p.d, ks = d / kCS, kbs = ks / kBlockK, of = ks, mt2 = of / kTileM;
     const int N = p.n_tile;
-    const int n_work = KIND == K_FFN ? p.d_ffn / 256 : p.n_heads;      // clusters that have a head / hidden chunk
-    const bool has_work = c < n_work;
+    // attention blocks: cluster = (head, row parity); local row l is row 2 l + parity of the step
+    const int head = c >> 1, parity = c & 1;
+    const int Nm = cl_mma_n(KIND, N);                // MMA N = rows of the operand tiles
+    const int n_work = KIND == K_FFN ? p.d_ffn / 128 : p.n_heads;      // heads / hidden chunks that exist
+    const bool has_work = KIND == K_FFN ? c < n_work : head < n_work;
     const ClSmem lay = cl_layout(KIND, N, kbs);
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint8_t *w_slots = base + lay.w_off;
+    uint8_t *w_tiles = base;
     float *recv = reinterpret_cast<float *>(base + lay.recv_off);
     uint8_t *r2 = base + lay.r2_off;                 // x planes; K_FFN: later the hidden planes
     uint8_t *ap = base + lay.ap_off;                 // attention output planes
     float2 *stats_recv = reinterpret_cast<float2 *>(base + lay.stats_off);
-    const int pb = N * 128;                          // bytes of one plane of one k-block
-    const int n_tiles1 = KIND == K_SELF ? 2 * kbs : KIND == K_CROSS ? kbs : 2 * kbs;
-    const int n_tiles2 = KIND == K_FFN ? 4 : 1;
+    float *sm_q = reinterpret_cast<float *>(base + lay.tab_off);                                  // [8][64] scaled queries
+    __nv_bfloat16 *sm_knew = reinterpret_cast<__nv_bfloat16 *>(base + lay.tab_off + 2048);         // [8][64] new keys
+    __nv_bfloat16 *sm_vnew = sm_knew + kMaxSlots * kHeadDim;                                       // [8][64] new values
+    uint8_t *ring = base + lay.ring_off;
+    float *part = recv;                              // attention partials reuse the receive buffer
+    const int RS = lay.ring_stages;
+    const int pb = Nm * 128;                         // bytes of one plane of one k-block
+    const int n_tiles1 = KIND == K_SELF ? 2 * kbs : kbs;
+    const int n_tiles2 = KIND == K_FFN ? 2 * mt2 : mt2;
     const int n_tiles = n_tiles1 + n_tiles2;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kMaxTiles; ++i) mbar_init(&bar_w[i], 1);
+        for (int i = 0; i < 8 * kMaxRing; ++i) mbar_init(&ring_bar[0][0] + i, 1);
         mbar_init(&bar_b, 8);
         mbar_init(&bar_d1, 1);
         mbar_init(&bar_d2, 1);
-        mbar_init(&cbar0, kCS * 8);                  // 8 worker warps of each of the 8 CTAs
+        mbar_init(&cbar0, kCS * 8);                  // 8 worker warps of each CTA of the cluster
         mbar_init(&cbar1, kCS * 8);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -222,7 +279,6 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
     const uint32_t tmem_base = tmem_slot;
     cluster_sync_all();                              // every CTA of the cluster has its barriers in place
     sg::pdl_launch_dependents();
-    AED_TRACE_BEGIN(p.state, 24 + KIND);
 
     if (warp == 0) {
         // ---- weight tiles by TMA: static data, requested before the dependency wait ---------------------------
@@ -231,55 +287,57 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             prefetch_tensormap(&map_w2);
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
-                if (t >= lay.n_slots) {              // K_FFN: the slot held a tile of the first projection
+                // tiles that reuse the area of a tile of the first projection wait for its MMAs
+                if ((KIND == K_SELF && t >= n_tiles1) || (KIND == K_FFN && t >= kFfnSlots)) {
                     ok = mbar_wait(&bar_d1, 0, &abort_flag);
                     if (!ok) break;
                 }
-                uint8_t *slot = w_slots + static_cast<size_t>(t % lay.n_slots) * kSlot;
+                uint8_t *slot = w_tiles + cl_tile_off(KIND, t, kbs);
                 if (t < n_tiles1) {
-                    const int kb = KIND == K_SELF ? t >> 1 : KIND == K_CROSS ? t : t % kbs;
+                    const int kb = KIND == K_SELF ? t >> 1 : t;
                     const int kc = j * ks + kb * kBlockK;
                     if (KIND == K_SELF) {
-                        if ((t & 1) == 0) {          // query rows | key rows of head c
+                        if ((t & 1) == 0) {          // query rows | key rows of the head
                             mbar_expect_tx(&bar_w[t], 2 * 8192);
-                            tma_load_2d(slot, &map_w1, kc, c * kHeadDim, &bar_w[t]);
-                            tma_load_2d(slot + 8192, &map_w1, kc, d + c * kHeadDim, &bar_w[t]);
+                            tma_load_2d(slot, &map_w1, kc, head * kHeadDim, &bar_w[t]);
+                            tma_load_2d(slot + 8192, &map_w1, kc, d + head * kHeadDim, &bar_w[t]);
                         } else {                     // value rows
                             mbar_expect_tx(&bar_w[t], 8192);
-                            tma_load_2d(slot, &map_w1, kc, 2 * d + c * kHeadDim, &bar_w[t]);
+                            tma_load_2d(slot, &map_w1, kc, 2 * d + head * kHeadDim, &bar_w[t]);
                         }
                     } else if (KIND == K_CROSS) {
                         mbar_expect_tx(&bar_w[t], 8192);
-                        tma_load_2d(slot, &map_w1, kc, c * kHeadDim, &bar_w[t]);
-                    } else {                         // 128 hidden features of chunk c
-                        const int mt = t / kbs;
+                        tma_load_2d(slot, &map_w1, kc, head * kHeadDim, &bar_w[t]);
+                    } else {                         // the 128 hidden features of chunk c
                         mbar_expect_tx(&bar_w[t], 2 * 8192);
-                        tma_load_2d(slot, &map_w1, kc, c * 256 + mt * 128, &bar_w[t]);
-                        tma_load_2d(slot + 8192, &map_w1, kc, c * 256 + mt * 128 + 64, &bar_w[t]);
+                        tma_load_2d(slot, &map_w1, kc, c * 128, &bar_w[t]);
+                        tma_load_2d(slot + 8192, &map_w1, kc, c * 128 + 64, &bar_w[t]);
                     }
-                } else {                             // second projection: this CTA's d/8 output features
-                    const int q = t - n_tiles1;
-                    const int kc = KIND == K_FFN ? c * 256 + q * kBlockK : c * kHeadDim;
-                    mbar_expect_tx(&bar_w[t], of * 128);
-                    for (int b = 0; b < of / 64; ++b) tma_load_2d(slot + b * 8192, &map_w2, kc, j * of + b * 64, &bar_w[t]);
+                } else {                             // second projection: 128 of this CTA's d/4 output features
+                    const int u = t - n_tiles1;
+                    const int m = KIND == K_FFN ? u >> 1 : u;
+                    const int kc = KIND == K_FFN ? c * 128 + (u & 1) * kBlockK : head * kHeadDim;
+                    mbar_expect_tx(&bar_w[t], 2 * 8192);
+                    tma_load_2d(slot, &map_w2, kc, j * of + m * kTileM, &bar_w[t]);
+                    tma_load_2d(slot + 8192, &map_w2, kc, j * of + m * kTileM + 64, &bar_w[t]);
                 }
             }
         }
     } else if (warp == 1) {
         // ---- MMA issue --------------------------------------------------------------------------------------------
         if (lane == 0 && has_work) {
-            const uint32_t idesc = instr_desc_bf16(N);
+            const uint32_t idesc = instr_desc_bf16(Nm);
             bool ok = mbar_wait(&bar_b, 0, &abort_flag);
             for (int t = 0; t < n_tiles1 && ok; ++t) {
                 ok = mbar_wait(&bar_w[t], 0, &abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const int kb = KIND == K_SELF ? t >> 1 : KIND == K_CROSS ? t : t % kbs;
-                const int acc = KIND == K_SELF ? (t & 1) : KIND == K_CROSS ? 0 : t / kbs;
-                const uint32_t sa = smem_u32(w_slots + static_cast<size_t>(t % lay.n_slots) * kSlot);
+                const int kb = KIND == K_SELF ? t >> 1 : t;
+                const int acc = KIND == K_SELF ? (t & 1) : 0;
+                const uint32_t sa = smem_u32(w_tiles + cl_tile_off(KIND, t, kbs));
                 const uint32_t sb = smem_u32(r2 + static_cast<size_t>(kb) * 2 * pb);
                 const uint64_t da = smem_desc_sw128(sa), dh = smem_desc_sw128(sb), dl = smem_desc_sw128(sb + pb);
-                const uint32_t td = tmem_base + acc * N;
+                const uint32_t td = tmem_base + acc * Nm;
 #pragma unroll
                 for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(td, da + 2 * k, dh + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
 #pragma unroll
@@ -291,15 +349,16 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             if (ok) {
                 fence_async_proxy();
                 tc_fence_after_sync();
-                const uint32_t td = tmem_base + 2 * N;
-                for (int q = 0; q < n_tiles2 && ok; ++q) {
-                    const int t = n_tiles1 + q;
+                for (int u = 0; u < n_tiles2 && ok; ++u) {
+                    const int t = n_tiles1 + u;
                     ok = mbar_wait(&bar_w[t], 0, &abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t sa = smem_u32(w_slots + static_cast<size_t>(t % lay.n_slots) * kSlot);
+                    const int m = KIND == K_FFN ? u >> 1 : u, q = KIND == K_FFN ? (u & 1) : 0;
+                    const uint32_t sa = smem_u32(w_tiles + cl_tile_off(KIND, t, kbs));
                     const uint32_t sb = smem_u32(KIND == K_FFN ? r2 + static_cast<size_t>(q) * 2 * pb : ap);
                     const uint64_t da = smem_desc_sw128(sa), dh = smem_desc_sw128(sb), dl = smem_desc_sw128(sb + pb);
+                    const uint32_t td = tmem_base + (2 + m) * Nm;
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(td, da + 2 * k, dh + 2 * k, idesc, (q > 0 || k > 0) ? 1u : 0u);
 #pragma unroll
@@ -319,19 +378,20 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             for (size_t k = static_cast<size_t>(cta) * 64 + st; k < pieces; k += static_cast<size_t>(n_cta) * 64)
                 asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src + k * 4096), "r"(4096) : "memory");
         }
-        if (p.pf_cache && c < p.n_heads) {
-            // keys and values that this CTA's rows read in the next attention block: thread = (row slot, k|v)
+        if (p.pf_cache && head < p.n_heads) {
+            // keys and values that the (head, parity) rows of this CTA read in the next attention block:
+            // thread = (row slot, k|v)
             const int slot = st >> 1, kv = st & 1;
-            if (slot < N / kCS) {
-                const int4 ri = p.row_info[j + kCS * slot];
+            if (slot < N / 2 / kCS) {
+                const int4 ri = p.row_info[2 * (j + kCS * slot) + parity];
                 if (ri.x >= 0) {
                     const __nv_bfloat16 *src;
                     int len;
                     if (p.pf_cross) {
-                        src = p.pf_cache + ((size_t)(kv * p.n_heads + c) * p.pf_capacity + ri.w) * kHeadDim;
+                        src = p.pf_cache + ((size_t)(kv * p.n_heads + head) * p.pf_capacity + ri.w) * kHeadDim;
                         len = ri.z;
                     } else {
-                        src = p.pf_cache + (((size_t)ri.x * 2 + kv) * p.n_heads + c) * (size_t)p.pf_capacity * kHeadDim;
+                        src = p.pf_cache + (((size_t)ri.x * 2 + kv) * p.n_heads + head) * (size_t)p.pf_capacity * kHeadDim;
                         len = ri.y;
                     }
                     for (int off = 0; off < len; off += 32) {
@@ -352,140 +412,178 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
     } else {
         // ---- workers: 8 warps ---------------------------------------------------------------------------------
         const int ww = warp - 2, pt = threadIdx.x - 64, quarter = warp & 3;
+        // timeline of the first worker thread of block 0 and of block 72
+        AED_TRACE_RESERVE(tcur, p.state, (pt == 0 && (blockIdx.x == 0 || blockIdx.x == 72)) ? 96u : 0u);
+        AED_TRACE_PUT(p.state, tcur, (blockIdx.x == 0 ? 24 : 124) + KIND);
         const uint32_t recv_s = smem_u32(recv), stats_s = smem_u32(stats_recv);
         const uint32_t cbar0_s = smem_u32(&cbar0), cbar1_s = smem_u32(&cbar1);
         const uint32_t ap_s = smem_u32(ap), r2_s = smem_u32(r2);
-        // x slice geometry: thread = (row within pass, 8-column chunk cc)
-        const int cpr = ks >> 3, rows_per_pass = 256 / cpr;
+        // x slice geometry: thread = (local row within pass, 8-column chunk cc)
+        const int cpr = ks >> 3, rows_per_pass = 256 / cpr;          // 16 or 32 chunks per row
         const int cc = pt % cpr, r_in_pass = pt / cpr;
-        const int SL = N / kCS;                            // row slots per CTA in the attention blocks
-        // attention geometry: G warps per row slot
-        const int G = 8 / (SL < 1 ? 1 : SL);
-        const int slot = ww / G, g = ww % G;
-        const int r_att = j + kCS * slot;
+        const int n_loc_cap = KIND == K_FFN ? N : N / 2;            // local rows of the cluster (capacity)
+        const int SL = N / 2 / kCS;                        // row slots per CTA in the attention blocks: local row = j + 4 slot
         const int dg = lane & 7, pg = lane >> 3;
-        int4 ri = make_int4(-1, 0, 0, 0);
-        const __nv_bfloat16 *kbase = nullptr, *vbase = nullptr;
-        int len = 0, len_static = 0;
-        Raw8<__nv_bfloat16> rk[4], rv[4];
         float gam[8];
+        // Attention work of this CTA: the 16-position chunks of all its rows, numbered row after row and dealt out
+        // to the 8 warps in equal contiguous runs (a long row is shared by several warps, a warp rarely changes
+        // row).  The i-th item of a warp goes through stage i mod RS of the warp's K/V ring.
+        auto issue_item = [&](int item, int stage, int &sl) {      // sl: row-slot cursor, only moves forward
+            while (item >= sm_cum[sl + 1]) ++sl;
+            const int p0 = (item - sm_cum[sl]) * kFusedChunk;
+            const int n_st = min(kFusedChunk, sm_lenst[sl] - p0);
+            if (n_st > 0 && lane == 0) {
+                uint64_t *bar = &ring_bar[ww][stage];
+                uint8_t *dst = ring + (static_cast<size_t>(ww) * RS + stage) * kRingStage;
+                mbar_expect_tx(bar, n_st * 256);
+                bulk_load(dst, sm_kptr[sl] + static_cast<size_t>(p0) * kHeadDim, n_st * 128, bar);
+                bulk_load(dst + 2048, sm_vptr[sl] + static_cast<size_t>(p0) * kHeadDim, n_st * 128, bar);
+            }
+        };
         if (has_work) {
             load8(p.gamma + j * ks + cc * 8, gam);
             // fold constants of the output features this CTA finishes
             if (KIND == K_SELF) {
                 if (pt < 192) {
-                    const int col = (pt >> 6) * d + c * kHeadDim + (pt & 63);
+                    const int col = (pt >> 6) * d + head * kHeadDim + (pt & 63);
                     sm_c1[pt] = p.c1[col];
                     sm_c2[pt] = p.c2[col];
                 }
             } else if (KIND == K_CROSS) {
-                if (pt < 64) { sm_c1[pt] = p.c1[c * kHeadDim + pt]; sm_c2[pt] = p.c2[c * kHeadDim + pt]; }
+                if (pt < 64) { sm_c1[pt] = p.c1[head * kHeadDim + pt]; sm_c2[pt] = p.c2[head * kHeadDim + pt]; }
             } else {
-                if (pt < 32) { sm_c1[pt] = p.c1[c * 256 + j * 32 + pt]; sm_c2[pt] = p.c2[c * 256 + j * 32 + pt]; }
+                if (pt < 32) { sm_c1[pt] = p.c1[c * 128 + j * 32 + pt]; sm_c2[pt] = p.c2[c * 128 + j * 32 + pt]; }
             }
-            if (KIND != K_FFN) {
-                ri = p.row_info[r_att];
-                if (ri.x >= 0) {
-                    len = KIND == K_CROSS ? ri.z : ri.y + 1;
-                    len_static = KIND == K_CROSS ? len : len - 1;
-                    if (KIND == K_CROSS) {
-                        kbase = p.cache + ((size_t)(0 * p.n_heads + c) * p.seq_capacity + ri.w) * kHeadDim;
-                        vbase = p.cache + ((size_t)(1 * p.n_heads + c) * p.seq_capacity + ri.w) * kHeadDim;
-                    } else {
-                        kbase = p.cache + (((size_t)ri.x * 2 + 0) * p.n_heads + c) * (size_t)p.seq_capacity * kHeadDim;
-                        vbase = p.cache + (((size_t)ri.x * 2 + 1) * p.n_heads + c) * (size_t)p.seq_capacity * kHeadDim;
+            if (KIND != K_FFN && ww == 0) {
+                // row table of this CTA (static during the step) -> lengths, cache pointers, chunk prefix sums
+                int len = 0;
+                if (lane < SL) {
+                    const int4 ri = p.row_info[2 * (j + kCS * lane) + parity];
+                    const __nv_bfloat16 *kb = p.cache, *vb = p.cache;
+                    int lst = 0;
+                    if (ri.x >= 0) {
+                        len = KIND == K_CROSS ? ri.z : ri.y + 1;
+                        lst = KIND == K_CROSS ? len : len - 1;
+                        if (KIND == K_CROSS) {
+                            kb = p.cache + ((size_t)(0 * p.n_heads + head) * p.seq_capacity + ri.w) * kHeadDim;
+                            vb = p.cache + ((size_t)(1 * p.n_heads + head) * p.seq_capacity + ri.w) * kHeadDim;
+                        } else {
+                            kb = p.cache + (((size_t)ri.x * 2 + 0) * p.n_heads + head) * (size_t)p.seq_capacity * kHeadDim;
+                            vb = p.cache + (((size_t)ri.x * 2 + 1) * p.n_heads + head) * (size_t)p.seq_capacity * kHeadDim;
+                        }
                     }
-                    // first chunk of this warp: static positions, streamed while the previous block still runs
-                    const int p0 = g * kFusedChunk;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int pos = p0 + i * 4 + pg;
-                        if (pos < len_static) {
-                            rk[i].load(kbase + (size_t)pos * kHeadDim + dg * 8);
-                            rv[i].load(vbase + (size_t)pos * kHeadDim + dg * 8);
-                        } else { rk[i].zero(); rv[i].zero(); }
-                    }
+                    sm_kptr[lane] = kb; sm_vptr[lane] = vb; sm_len[lane] = len; sm_lenst[lane] = lst;
                 }
+                int chunks = (len + kFusedChunk - 1) / kFusedChunk;       // 0 for lanes without a row
+                int incl = chunks;
+#pragma unroll
+                for (int o = 1; o < kMaxSlots; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                if (lane < kMaxSlots) sm_cum[lane + 1] = incl;
+                if (lane == 0) sm_cum[0] = 0;
             }
         }
-        worker_sync();                                     // fold constants staged
+        worker_sync();                                     // fold constants and row table staged
+        int item0 = 0, item1 = 0, sl_issue = 0, sl_use = 0;
+        if (KIND != K_FFN && has_work) {
+            const int n_items = sm_cum[SL], per = (n_items + 7) / 8;
+            item0 = min(ww * per, n_items);
+            item1 = min(item0 + per, n_items);
+            // the first chunks of this warp are static data: they stream while the previous block still runs
+            for (int i = 0; i < RS; ++i)
+                if (item0 + i < item1) issue_item(item0 + i, i, sl_issue);
+        }
         sg::pdl_wait();
+        AED_TRACE_PUT(p.state, tcur, 50);          // dependency resolved
         const int n_rows = p.state->n_active;
+        // local rows of this cluster that exist, and the step row of local row l
+        const int n_loc = KIND == K_FFN ? min(n_rows, N) : min(max((n_rows - parity + 1) / 2, 0), N / 2);
+        auto step_row = [&](int l) { return KIND == K_FFN ? l : 2 * l + parity; };
         bool ok = true;
         if (has_work) {
             // ---- 1. x slice -> statistics of the slice, gamma*x as bf16 planes -----------------------------------
-            float xv[4][8];
+            for (int ps0 = 0; ps0 * rows_per_pass < n_loc_cap; ps0 += 4) {
+                float xv[4][8];
 #pragma unroll
-            for (int ps = 0; ps < 4; ++ps) {
-                const int r = ps * rows_per_pass + r_in_pass;
-                if (r < N && r < n_rows) load8(p.x_in + (size_t)r * d + j * ks + cc * 8, xv[ps]);
-                else {
+                for (int ps = 0; ps < 4; ++ps) {
+                    const int l = (ps0 + ps) * rows_per_pass + r_in_pass;
+                    if (l < n_loc) load8(p.x_in + (size_t)step_row(l) * d + j * ks + cc * 8, xv[ps]);
+                    else {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) xv[ps][e] = 0.f;
-                }
-            }
-#pragma unroll
-            for (int ps = 0; ps < 4; ++ps) {
-                const int r = ps * rows_per_pass + r_in_pass;
-                if (ps * rows_per_pass >= N) break;        // uniform over the block
-                float s = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) s += xv[ps][e];
-                s += __shfl_xor_sync(0xffffffffu, s, 1);
-                s += __shfl_xor_sync(0xffffffffu, s, 2);
-                s += __shfl_xor_sync(0xffffffffu, s, 4);
-                if (cpr == 16) s += __shfl_xor_sync(0xffffffffu, s, 8);
-                const float mean = s / ks;
-                float q = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) { const float dv = xv[ps][e] - mean; q = fmaf(dv, dv, q); }
-                q += __shfl_xor_sync(0xffffffffu, q, 1);
-                q += __shfl_xor_sync(0xffffffffu, q, 2);
-                q += __shfl_xor_sync(0xffffffffu, q, 4);
-                if (cpr == 16) q += __shfl_xor_sync(0xffffffffu, q, 8);
-                if (r < N) {
-                    if (r < n_rows) {
-                        if (KIND == K_FFN) {               // every CTA of the cluster needs every row's statistics
-                            if (cc < kCS) st_cluster_f32x2(map_to_cta(stats_s, cc) + (j * kMaxRows + r) * 8, mean, q);
-                        } else if (cc == 0) {              // the CTA that owns the row
-                            st_cluster_f32x2(map_to_cta(stats_s, r & 7) + (j * kMaxRows + (r >> 3)) * 8, mean, q);
-                        }
+                        for (int e = 0; e < 8; ++e) xv[ps][e] = 0.f;
                     }
-                    float y[8];
+                }
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = xv[ps][e] * gam[e];
-                    uint4 hi, lo;
-                    sg::split_planes(y, hi, lo);
-                    const int kb = cc >> 3, ch = cc & 7;
-                    uint8_t *tile = r2 + static_cast<size_t>(kb) * 2 * pb;
-                    const int off = r * 128 + ((ch ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4 *>(tile + off) = hi;
-                    *reinterpret_cast<uint4 *>(tile + pb + off) = lo;
+                for (int ps = 0; ps < 4; ++ps) {
+                    const int l = (ps0 + ps) * rows_per_pass + r_in_pass;
+                    if ((ps0 + ps) * rows_per_pass >= n_loc_cap) break;        // uniform over the block
+                    float s = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) s += xv[ps][e];
+                    s += __shfl_xor_sync(0xffffffffu, s, 1);
+                    s += __shfl_xor_sync(0xffffffffu, s, 2);
+                    s += __shfl_xor_sync(0xffffffffu, s, 4);
+                    s += __shfl_xor_sync(0xffffffffu, s, 8);
+                    if (cpr == 32) s += __shfl_xor_sync(0xffffffffu, s, 16);
+                    const float mean = s / ks;
+                    float q = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { const float dv = xv[ps][e] - mean; q = fmaf(dv, dv, q); }
+                    q += __shfl_xor_sync(0xffffffffu, q, 1);
+                    q += __shfl_xor_sync(0xffffffffu, q, 2);
+                    q += __shfl_xor_sync(0xffffffffu, q, 4);
+                    q += __shfl_xor_sync(0xffffffffu, q, 8);
+                    if (cpr == 32) q += __shfl_xor_sync(0xffffffffu, q, 16);
+                    if (l < n_loc_cap) {
+                        if (l < n_loc) {
+                            if (KIND == K_FFN) {           // every CTA of the cluster needs every row's statistics
+                                if (cc < kCS) st_cluster_f32x2(map_to_cta(stats_s, cc) + (j * kMaxRows + l) * 8, mean, q);
+                            } else if (cc == 0) {          // the CTA that owns the row
+                                st_cluster_f32x2(map_to_cta(stats_s, l & 3) + (j * kMaxRows + (l >> 2)) * 8, mean, q);
+                            }
+                        }
+                        float y[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) y[e] = xv[ps][e] * gam[e];
+                        uint4 hi, lo;
+                        sg::split_planes(y, hi, lo);
+                        const int kb = cc >> 3, ch = cc & 7;
+                        uint8_t *tile = r2 + static_cast<size_t>(kb) * 2 * pb;
+                        const int off = l * 128 + ((ch ^ (l & 7)) << 4);
+                        *reinterpret_cast<uint4 *>(tile + off) = hi;
+                        *reinterpret_cast<uint4 *>(tile + pb + off) = lo;
+                    }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b)) : "memory");
+            AED_TRACE_PUT(p.state, tcur, 51);      // operand planes written
 
             // ---- 3. partial sums of the first projection -> the CTA that finishes them ----------------------------
             ok = mbar_wait(&bar_d1, 0, &abort_flag);
             tc_fence_after_sync();
+            AED_TRACE_PUT(p.state, tcur, 52);      // first projection complete
             if (ok) {
-                const int acc = (KIND == K_CROSS) ? 0 : (ww < 4 ? 0 : 1);
+                const int acc = (KIND == K_SELF && ww >= 4) ? 1 : 0;
                 const bool lanes_ok = KIND == K_SELF ? (acc == 0 || quarter < 2) : KIND == K_CROSS ? quarter < 2 : true;
-                const int col_lo = KIND == K_CROSS ? (ww < 4 ? 0 : N / 2) : 0;
-                const int col_hi = KIND == K_CROSS ? (ww < 4 ? N / 2 : N) : N;
+                // two warps share a quarter of the lanes where one accumulator serves all 8 warps: split the columns
+                const bool split_cols = KIND != K_SELF;
+                const int col_lo = split_cols && ww >= 4 ? Nm / 2 : 0;
+                const int col_hi = min(split_cols && ww < 4 ? Nm / 2 : Nm, n_loc);
                 if (lanes_ok) {
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * N;
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * Nm;
                     if (KIND == K_FFN) {
-                        // lanes = 32 consecutive hidden features, all owned by CTA acc*4 + quarter
-                        const uint32_t dst = map_to_cta(recv_s, acc * 4 + quarter) + (static_cast<uint32_t>(j) * N * 32 + lane) * 4;
-                        for (int c0 = 0; c0 < N; c0 += 16) {
+                        // lanes = 32 consecutive hidden features, all owned by CTA quarter
+                        const uint32_t dst = map_to_cta(recv_s, quarter) + (static_cast<uint32_t>(j) * N * 32 + lane) * 4;
+                        for (int c0 = (col_lo / 16) * 16; c0 < col_hi; c0 += 16) {
                             float v[16];
                             tmem_ld16(taddr + c0, v);
 #pragma unroll
                             for (int jj = 0; jj < 16; ++jj)
-                                if (c0 + jj < n_rows) st_cluster_f32(dst + (c0 + jj) * 128, v[jj]);
+                                if (c0 + jj >= col_lo && c0 + jj < col_hi) st_cluster_f32(dst + (c0 + jj) * 128, v[jj]);
                         }
                     } else {
                         const int FE = KIND == K_SELF ? 192 : 64;
@@ -493,13 +591,13 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                         uint32_t peer[kCS];
 #pragma unroll
                         for (int o = 0; o < kCS; ++o) peer[o] = map_to_cta(recv_s, o) + (static_cast<uint32_t>(j) * SL * FE + feat) * 4;
-                        for (int c0 = 0; c0 < N; c0 += 16) {
+                        for (int c0 = (col_lo / 16) * 16; c0 < col_hi; c0 += 16) {
                             float v[16];
                             tmem_ld16(taddr + c0, v);
 #pragma unroll
                             for (int jj = 0; jj < 16; ++jj) {
-                                const int r = c0 + jj;                 // owner r & 7 = jj & 7, slot r >> 3
-                                if (r >= col_lo && r < col_hi && r < n_rows) st_cluster_f32(peer[jj & 7] + (r >> 3) * FE * 4, v[jj]);
+                                const int l = c0 + jj;                 // owner l & 3 = jj & 3, slot l >> 2
+                                if (l >= col_lo && l < col_hi) st_cluster_f32(peer[jj & 3] + (l >> 2) * FE * 4, v[jj]);
                             }
                         }
                     }
@@ -507,12 +605,14 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             }
             __syncwarp();
             if (lane < kCS) arrive_remote(map_to_cta(cbar0_s, lane));     // first exchange, also on the abort path
+            AED_TRACE_PUT(p.state, tcur, 53);      // partials sent
             ok = mbar_wait_cluster(&cbar0, 0, &abort_flag) && ok;
+            AED_TRACE_PUT(p.state, tcur, 54);      // first exchange complete
 
             if (KIND == K_FFN) {
                 // ---- 4. hidden activations of this CTA's 32 features, written into every CTA's operand tile ------
                 const int r = pt >> 2, c4 = pt & 3;
-                if (ok && r < N && r < n_rows) {
+                if (ok && r < n_loc) {
                     float a[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) a[e] = 0.f;
@@ -541,37 +641,36 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                 }
             } else {
                 // ---- 4. attention for the rows of this CTA -------------------------------------------------------------
-                float m = -INFINITY, l = 0.f, acc8[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc8[e] = 0.f;
-                const bool row_ok = ok && ri.x >= 0 && r_att < n_rows;
-                if (row_ok) {
-                    const int FE = KIND == K_SELF ? 192 : 64;
-                    const float2 st = merge_stats(stats_recv + slot, kMaxRows, ks, d, p.eps);
+                const int FE = KIND == K_SELF ? 192 : 64;
+                // 4a. warp s finishes the query (and the new key / value) of row slot s
+                if (ok && ww < SL && sm_len[ww] > 0) {
+                    const int sl = ww;
+                    const float2 st = merge_stats(stats_recv + sl, kMaxRows, ks, d, p.eps);
                     float qv[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) qv[e] = 0.f;
 #pragma unroll
-                    for (int s = 0; s < kCS; ++s) {
+                    for (int s8 = 0; s8 < kCS; ++s8) {
                         float t8[8];
-                        load8(recv + (static_cast<size_t>(s) * SL + slot) * FE + dg * 8, t8);
+                        load8(recv + (static_cast<size_t>(s8) * SL + sl) * FE + dg * 8, t8);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) qv[e] += t8[e];
                     }
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
                         qv[e] = fmaf(st.y, qv[e] - st.x * sm_c1[dg * 8 + e], sm_c2[dg * 8 + e]) * p.scale;
-                    const int new_chunk = (len - 1) / kFusedChunk;
-                    const bool owns_new = KIND == K_SELF && g == new_chunk % G;
-                    Raw8<__nv_bfloat16> new_k, new_v;
-                    if (owns_new) {
+                    if (pg == 0) {
+                        *reinterpret_cast<float4 *>(sm_q + sl * kHeadDim + dg * 8) = make_float4(qv[0], qv[1], qv[2], qv[3]);
+                        *reinterpret_cast<float4 *>(sm_q + sl * kHeadDim + dg * 8 + 4) = make_float4(qv[4], qv[5], qv[6], qv[7]);
+                    }
+                    if (KIND == K_SELF) {
                         float kn[8], vn[8];
 #pragma unroll
                         for (int e = 0; e < 8; ++e) { kn[e] = 0.f; vn[e] = 0.f; }
 #pragma unroll
-                        for (int s = 0; s < kCS; ++s) {
+                        for (int s8 = 0; s8 < kCS; ++s8) {
                             float t8[8];
-                            const float *src = recv + (static_cast<size_t>(s) * SL + slot) * FE + dg * 8;
+                            const float *src = recv + (static_cast<size_t>(s8) * SL + sl) * FE + dg * 8;
                             load8(src + 64, t8);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) kn[e] += t8[e];
@@ -584,89 +683,139 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                             kn[e] = fmaf(st.y, kn[e] - st.x * sm_c1[64 + dg * 8 + e], sm_c2[64 + dg * 8 + e]);
                             vn[e] = fmaf(st.y, vn[e] - st.x * sm_c1[128 + dg * 8 + e], sm_c2[128 + dg * 8 + e]);
                         }
+                        Raw8<__nv_bfloat16> new_k, new_v;
                         new_k.set(kn);
                         new_v.set(vn);
-                        if (pg == 0) {      // append; nobody else reads this position during this launch
-                            new_k.store(const_cast<__nv_bfloat16 *>(kbase) + (size_t)(len - 1) * kHeadDim + dg * 8);
-                            new_v.store(const_cast<__nv_bfloat16 *>(vbase) + (size_t)(len - 1) * kHeadDim + dg * 8);
+                        if (pg == 0) {      // append to the cache (nobody reads this position during this launch) and keep a copy
+                            const int pos = sm_len[sl] - 1;
+                            new_k.store(const_cast<__nv_bfloat16 *>(sm_kptr[sl]) + (size_t)pos * kHeadDim + dg * 8);
+                            new_v.store(const_cast<__nv_bfloat16 *>(sm_vptr[sl]) + (size_t)pos * kHeadDim + dg * 8);
+                            new_k.store(sm_knew + sl * kHeadDim + dg * 8);
+                            new_v.store(sm_vnew + sl * kHeadDim + dg * 8);
                         }
                     }
-                    bool loaded = true;
-                    for (int p0 = g * kFusedChunk; p0 < len; p0 += G * kFusedChunk) {
-                        if (!loaded) {
+                }
+                worker_sync();          // queries in place; the receive buffer is free for the partials
+                AED_TRACE_PUT(p.state, tcur, 58);
+                if (lane < SL) part[(ww * SL + lane) * kPartStride] = -INFINITY;
+                __syncwarp();
+                // 4b. this warp's chunks
+                {
+                    float m = -INFINITY, l = 0.f, acc8[8], qv[8];
+                    int cur = -1;
+                    auto flush = [&]() {
+                        l += __shfl_xor_sync(0xffffffffu, l, 8);
+                        l += __shfl_xor_sync(0xffffffffu, l, 16);
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int pos = p0 + i * 4 + pg;
-                                if (pos < len_static) {
-                                    rk[i].load(kbase + (size_t)pos * kHeadDim + dg * 8);
-                                    rv[i].load(vbase + (size_t)pos * kHeadDim + dg * 8);
-                                } else { rk[i].zero(); rv[i].zero(); }
-                            }
+                        for (int e = 0; e < 8; ++e) {
+                            acc8[e] += __shfl_xor_sync(0xffffffffu, acc8[e], 8);
+                            acc8[e] += __shfl_xor_sync(0xffffffffu, acc8[e], 16);
                         }
-                        loaded = false;
-                        if (owns_new && p0 == new_chunk * kFusedChunk) {
+                        float *dst = part + (ww * SL + cur) * kPartStride;
+                        if (lane == 0) { dst[0] = m; dst[1] = l; }
+                        if (pg == 0) {
+                            *reinterpret_cast<float4 *>(dst + 4 + dg * 8) = make_float4(acc8[0], acc8[1], acc8[2], acc8[3]);
+                            *reinterpret_cast<float4 *>(dst + 8 + dg * 8) = make_float4(acc8[4], acc8[5], acc8[6], acc8[7]);
+                        }
+                    };
+                    int i = 0;
+                    uint32_t ring_phase = 0;              // bit s: parity of the next copy to land in stage s
+                    for (int item = item0; item < item1 && ok; ++item, ++i) {
+                        const int stage = i % RS;
+                        while (item >= sm_cum[sl_use + 1]) ++sl_use;
+                        const int sl = sl_use;
+                        const int p0 = (item - sm_cum[sl]) * kFusedChunk;
+                        const int len = sm_len[sl], len_st = sm_lenst[sl];
+                        if (sl != cur) {
+                            if (cur >= 0) flush();
+                            cur = sl;
+                            m = -INFINITY; l = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                if (p0 + i * 4 + pg == len - 1) { rk[i] = new_k; rv[i] = new_v; }
+                            for (int e = 0; e < 8; ++e) acc8[e] = 0.f;
+                            load8(sm_q + sl * kHeadDim + dg * 8, qv);
                         }
+                        AED_TRACE_PUT(p.state, tcur, 61);
+                        if (len_st > p0) {                // a chunk that holds only the new position has no copy
+                            ok = mbar_wait(&ring_bar[ww][stage], (ring_phase >> stage) & 1u, &abort_flag);
+                            ring_phase ^= 1u << stage;
+                        }
+                        if (!ok) break;
+                        AED_TRACE_PUT(p.state, tcur, 62);
+                        const uint8_t *stg = ring + (static_cast<size_t>(ww) * RS + stage) * kRingStage;
+                        Raw8<__nv_bfloat16> rk[4], rv[4];
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const int pl = q4 * 4 + pg;                 // position inside the chunk
+                            if (p0 + pl < len_st) {
+                                rk[q4].load(reinterpret_cast<const __nv_bfloat16 *>(stg + pl * 128) + dg * 8);
+                                rv[q4].load(reinterpret_cast<const __nv_bfloat16 *>(stg + 2048 + pl * 128) + dg * 8);
+                            } else if (KIND == K_SELF && p0 + pl == len - 1) {
+                                rk[q4].load(sm_knew + sl * kHeadDim + dg * 8);
+                                rv[q4].load(sm_vnew + sl * kHeadDim + dg * 8);
+                            } else { rk[q4].zero(); rv[q4].zero(); }
+                        }
+                        __syncwarp();                                  // the stage has been read: refill it
+                        AED_TRACE_PUT(p.state, tcur, 63);
+                        if (item + RS < item1) issue_item(item + RS, stage, sl_issue);
+                        AED_TRACE_PUT(p.state, tcur, 64);
                         float s4[4], cmax = -INFINITY;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
+                        for (int q4 = 0; q4 < 4; ++q4) {
                             float kf[8], dot = 0.f;
-                            rk[i].get(kf);
+                            rk[q4].get(kf);
 #pragma unroll
                             for (int e = 0; e < 8; ++e) dot = fmaf(qv[e], kf[e], dot);
                             dot += __shfl_xor_sync(0xffffffffu, dot, 1);
                             dot += __shfl_xor_sync(0xffffffffu, dot, 2);
                             dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-                            s4[i] = (p0 + i * 4 + pg < len) ? dot : -INFINITY;
-                            cmax = fmaxf(cmax, s4[i]);
+                            s4[q4] = (p0 + q4 * 4 + pg < len) ? dot : -INFINITY;
+                            cmax = fmaxf(cmax, s4[q4]);
                         }
                         cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-                        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));
+                        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));      // finite: the chunk has a position
                         const float m_new = fmaxf(m, cmax);
                         const float corr = expf(m - m_new);
                         l *= corr;
 #pragma unroll
                         for (int e = 0; e < 8; ++e) acc8[e] *= corr;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float pr = expf(s4[i] - m_new);
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const float pr = expf(s4[q4] - m_new);
                             float vf[8];
-                            rv[i].get(vf);
+                            rv[q4].get(vf);
                             l += pr;
 #pragma unroll
                             for (int e = 0; e < 8; ++e) acc8[e] = fmaf(pr, vf[e], acc8[e]);
                         }
                         m = m_new;
+                        AED_TRACE_PUT(p.state, tcur, 65);
                     }
-                    l += __shfl_xor_sync(0xffffffffu, l, 8);
-                    l += __shfl_xor_sync(0xffffffffu, l, 16);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        acc8[e] += __shfl_xor_sync(0xffffffffu, acc8[e], 8);
-                        acc8[e] += __shfl_xor_sync(0xffffffffu, acc8[e], 16);
-                    }
+                    if (cur >= 0 && ok) flush();
                 }
-                if (lane == 0) { sm_m[ww] = m; sm_l[ww] = l; }
-                if (pg == 0) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) sm_acc[ww][dg * 8 + e] = acc8[e];
-                }
+                AED_TRACE_PUT(p.state, tcur, 59);
                 worker_sync();
-                if (row_ok && g == 0) {
-                    // merge the G warps of the row; lane group pg sends to CTAs 2 pg and 2 pg + 1
+                AED_TRACE_PUT(p.state, tcur, 60);
+                // 4c. warp s merges the partials of row slot s and sends the result to every CTA's operand tile;
+                //     lane group pg writes to CTA pg
+                if (ok && ww < SL && sm_len[ww] > 0) {
+                    const int sl = ww, r_att = j + kCS * sl;      // local row = row of the operand tile
                     float big = -INFINITY;
-                    for (int w = 0; w < G; ++w) big = fmaxf(big, sm_m[slot * G + w]);
+#pragma unroll
+                    for (int w8 = 0; w8 < 8; ++w8) big = fmaxf(big, part[(w8 * SL + sl) * kPartStride]);
                     float lsum = 0.f, o[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) o[e] = 0.f;
-                    for (int w = 0; w < G; ++w) {
-                        const float mw = sm_m[slot * G + w];
-                        const float wgt = (mw == -INFINITY) ? 0.f : expf(mw - big);
-                        lsum = fmaf(sm_l[slot * G + w], wgt, lsum);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) o[e] = fmaf(sm_acc[slot * G + w][dg * 8 + e], wgt, o[e]);
+                    for (int w8 = 0; w8 < 8; ++w8) {
+                        const float *src = part + (w8 * SL + sl) * kPartStride;
+                        const float mw = src[0];
+                        if (mw == -INFINITY) continue;             // uniform over the warp
+                        const float wgt = expf(mw - big);
+                        lsum = fmaf(src[1], wgt, lsum);
+                        float a8[8];
+                        load8(src + 4 + dg * 8, a8);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[e] = fmaf(a8[e], wgt, o[e]);
                     }
                     const float inv = 1.f / lsum;
 #pragma unroll
@@ -674,57 +823,69 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                     uint4 hi, lo;
                     sg::split_planes(o, hi, lo);
                     const uint32_t off = r_att * 128 + ((dg ^ (r_att & 7)) << 4);
-#pragma unroll
-                    for (int o2 = 0; o2 < 2; ++o2) {
-                        const uint32_t dst = map_to_cta(ap_s, 2 * pg + o2) + off;
-                        st_cluster_b128(dst, hi);
-                        st_cluster_b128(dst + pb, lo);
-                    }
+                    const uint32_t dst = map_to_cta(ap_s, pg) + off;
+                    st_cluster_b128(dst, hi);
+                    st_cluster_b128(dst + pb, lo);
                 }
             }
             fence_async_proxy();
             __syncwarp();
             if (lane < kCS) arrive_remote(map_to_cta(cbar1_s, lane));     // second exchange
+            AED_TRACE_PUT(p.state, tcur, 55);      // attention / activation done
 
             // ---- 5. second projection: partial over this head / chunk, added into x_out -----------------------------
-            // The residual x_in and the bias are one more term of the sum: the cluster with c == r mod n_work adds
-            // them for row r, while the MMAs of the second projection run.
-            const int f = quarter * 32 + lane;
-            const bool f_ok = f < of;
-            const int half = ww < 4 ? 0 : 1;
-            const int col0 = half * (N / 2), col1 = min(col0 + N / 2, n_rows);
-            if (f_ok) {
-                const float bias = p.bias2 ? to_f32(p.bias2[j * of + f]) : 0.f;
-                int r = col0 + ((c - col0 % n_work) + n_work) % n_work;      // first row >= col0 with r mod n_work == c
-                while (r < col1) {
-                    float res[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int ri4 = r + i * n_work;
-                        res[i] = ri4 < col1 ? p.x_in[(size_t)ri4 * d + j * of + f] + bias : 0.f;
+            // The residual x_in and the bias are one more term of the sum: among the clusters that share this
+            // cluster's rows, the one whose head / chunk index equals l mod n_work adds them for local row l, while
+            // the MMAs of the second projection run.  All additions are 16-byte reductions.
+            const int g4n = of / 4;                            // groups of 4 features per row
+            {
+                const int who = KIND == K_FFN ? c : head;
+                const int n_res = n_loc > who ? (n_loc - who + n_work - 1) / n_work : 0;      // local rows who, who + n_work, ...
+                for (int idx = pt; idx < n_res * g4n; idx += 256) {
+                    const int r = step_row(who + n_work * (idx / g4n)), f4 = (idx % g4n) * 4;
+                    float4 v = *reinterpret_cast<const float4 *>(p.x_in + (size_t)r * d + j * of + f4);
+                    if (p.bias2) {
+                        float b4[4];
+                        load4(p.bias2 + j * of + f4, b4);
+                        v.x += b4[0]; v.y += b4[1]; v.z += b4[2]; v.w += b4[3];
                     }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int ri4 = r + i * n_work;
-                        if (ri4 < col1) atomicAdd(p.x_out + (size_t)ri4 * d + j * of + f, res[i]);
-                    }
-                    r += 4 * n_work;
+                    sg::red_add_v4(p.x_out + (size_t)r * d + j * of + f4, v);
                 }
             }
             ok = mbar_wait(&bar_d2, 0, &abort_flag) && ok;
             tc_fence_after_sync();
-            if (ok && f_ok) {
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + 2 * N;
-                for (int c0 = (col0 / 16) * 16; c0 < col1; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + c0, v);
+            AED_TRACE_PUT(p.state, tcur, 56);      // second projection complete
+            // accumulators [feature lane][local row] -> shared memory [local row][feature]; the operand planes (and,
+            // in the FFN block, the receive buffer in front of them) are free now
+            float *trans = KIND == K_FFN ? recv : reinterpret_cast<float *>(r2);
+            const int pitch = of + 4;
+            {
+                const int m = mt2 == 2 ? (ww >> 2) : 0;        // 128-feature tile of this warp
+                const int f = m * kTileM + quarter * 32 + lane;
+                const int col_lo = mt2 == 2 || ww < 4 ? 0 : Nm / 2;
+                const int col_hi = min(mt2 == 2 || ww >= 4 ? Nm : Nm / 2, n_loc);
+                if (ok) {
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + (2 + m) * Nm;
+                    for (int c0 = (col_lo / 16) * 16; c0 < col_hi; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(taddr + c0, v);
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        const int r = c0 + jj;
-                        if (r >= col0 && r < col1) atomicAdd(p.x_out + (size_t)r * d + j * of + f, v[jj]);
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const int l = c0 + jj;
+                            if (l >= col_lo && l < col_hi) trans[l * pitch + f] = v[jj];
+                        }
                     }
                 }
             }
+            worker_sync();
+            if (ok) {
+                for (int idx = pt; idx < n_loc * g4n; idx += 256) {
+                    const int l = idx / g4n, f4 = (idx % g4n) * 4;
+                    const float4 v = *reinterpret_cast<const float4 *>(trans + l * pitch + f4);
+                    sg::red_add_v4(p.x_out + (size_t)step_row(l) * d + j * of + f4, v);
+                }
+            }
+            AED_TRACE_PUT(p.state, tcur, 57);              // reductions issued
         }
     }
     tc_fence_before_sync();

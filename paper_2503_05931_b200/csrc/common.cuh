@@ -46,11 +46,40 @@ __device__ __forceinline__ void trace_mark(const DecState *state, uint32_t id)
         if (i < (1u << 16)) { tb->ev[i].id = id; tb->ev[i].t_ns = t; }
     }
 }
+// Cheap marks for one thread of block 0: a range of the buffer is reserved once (the atomic's latency is paid
+// where nothing waits on it), later marks are plain stores.
+struct TraceCursor { uint32_t next, end; };
+__device__ __forceinline__ TraceCursor trace_reserve(const DecState *state, uint32_t n)
+{
+    TraceCursor c{0u, 0u};
+    if (n > 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+        TraceBuf *tb = reinterpret_cast<TraceBuf *>(reinterpret_cast<char *>(const_cast<DecState *>(state)) + 256);
+        c.next = atomicAdd(&tb->count, n);
+        c.end = c.next + n;
+        if (c.end > (1u << 16)) c.end = c.next;
+    }
+    return c;
+}
+__device__ __forceinline__ void trace_put(const DecState *state, TraceCursor &c, uint32_t id)
+{
+    if (c.next < c.end) {
+        TraceBuf *tb = reinterpret_cast<TraceBuf *>(reinterpret_cast<char *>(const_cast<DecState *>(state)) + 256);
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        tb->ev[c.next].id = id;
+        tb->ev[c.next].t_ns = t;
+        ++c.next;
+    }
+}
 #define AED_TRACE_BEGIN(state, id) trace_begin(state, id)
 #define AED_TRACE_MARK(state, id) trace_mark(state, id)
+#define AED_TRACE_RESERVE(cur, state, n) TraceCursor cur = trace_reserve(state, n)
+#define AED_TRACE_PUT(state, cur, id) trace_put(state, cur, id)
 #else
 #define AED_TRACE_BEGIN(state, id) ((void)0)
 #define AED_TRACE_MARK(state, id) ((void)0)
+#define AED_TRACE_RESERVE(cur, state, n) ((void)0)
+#define AED_TRACE_PUT(state, cur, id) ((void)0)
 #endif
 
 __device__ __forceinline__ float to_f32(float v) { return v; }

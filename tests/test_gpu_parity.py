@@ -214,9 +214,11 @@ def test_config3_shape_sampled_rows():
     _run_both(w, rows=rows)
 
 
-def test_config2_shape_sampled_rows():
-    """24-layer d=1024 bf16 decoder at batch 64 (the benchmark configuration and launch path): a sample of
+@pytest.mark.parametrize("cluster", ["0", "1"])
+def test_config2_shape_sampled_rows(cluster, monkeypatch):
+    """24-layer d=1024 bf16 decoder at batch 64 (the benchmark configuration, on both launch paths): a sample of
     utterances is decoded one by one by the checker and compared with the GPU's full-batch run."""
+    monkeypatch.setenv("AED_DEC_CLUSTER", cluster)
     w = wl.make_workload("cfg2")
     order = np.argsort(w.dec_lens)
     rows = sorted({int(order[0]), int(order[len(order) // 2]), int(order[3]), int(np.argmin(w.enc_lens))})
@@ -232,9 +234,10 @@ CLUSTER_B = dict(n_layers=1, d_model=1024, n_heads=16, d_ffn=768, vocab=520, d_e
 
 
 @pytest.mark.parametrize("batch", [1, 7, 16, 17, 40, 64])
-def test_cluster_path_row_counts(batch):
+def test_cluster_path_row_counts(batch, monkeypatch):
     """Every MMA row-tile width of the cluster kernels (16, 32, 64), with partly filled tiles, ragged encoder
     lengths from 1 frame to several attention chunks, and rows retiring at different steps."""
+    monkeypatch.setenv("AED_DEC_CLUSTER", "1")
     rng = np.random.default_rng(900 + batch)
     enc_lens = rng.integers(1, 150, size=batch)
     dec_lens = rng.integers(1, 24, size=batch)
@@ -244,7 +247,8 @@ def test_cluster_path_row_counts(batch):
     _run_both(w, rows=rows)
 
 
-def test_cluster_path_d1024():
+def test_cluster_path_d1024(monkeypatch):
+    monkeypatch.setenv("AED_DEC_CLUSTER", "1")
     rng = np.random.default_rng(31)
     batch = 24
     w = wl.make_custom(CLUSTER_B, rng.integers(1, 200, size=batch), rng.integers(1, 20, size=batch), dtype="bf16", seed=77)
@@ -260,8 +264,8 @@ def test_cluster_path_matches_kernel_chain(monkeypatch):
     batch = 33
     w = wl.make_custom(CLUSTER_A, rng.integers(1, 120, size=batch), [6] * batch, dtype="bf16", seed=9)
     outs = []
-    for no_cluster in ("0", "1"):
-        monkeypatch.setenv("AED_DEC_NO_CLUSTER", no_cluster)
+    for cluster in ("1", "0"):
+        monkeypatch.setenv("AED_DEC_CLUSTER", cluster)
         dec = b.decoder_for_workload(w)
         dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
         logits = torch.zeros((batch, CLUSTER_A["vocab"]), dtype=torch.float32, device="cuda:0")

@@ -52,6 +52,7 @@ struct Layout {
     size_t actd_hi, actd_lo, actf_hi, actf_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
     size_t x1, x2;                        // the other two buffers of the rotating residual stream (cluster path)
+    size_t cl_blocks, cl_maps;            // block descriptions and tensor maps of the persistent step kernel
     size_t fold_layer_floats;
     int rows_cap;
 };
@@ -122,6 +123,8 @@ Layout make_layout(const aed_dec_config_t &c)
         L.qc = take(B * d * 4);
         L.x1 = take(B * d * 4);
         L.x2 = take(B * d * 4);
+        L.cl_blocks = take((size_t)3 * c.n_layers * sizeof(cl::ClusterParams));
+        L.cl_maps = take((size_t)6 * c.n_layers * sizeof(CUtensorMap));
     }
     L.total = off;
     return L;
@@ -157,6 +160,7 @@ struct aed_dec {
     struct ClLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };      // boxes of 64 rows x 64 k
     std::vector<ClLayerMaps> cl_layers;
     bool use_cluster = false;             // head-parallel cluster kernels for steps of at most 64 rows
+    bool use_persistent = true;           // all blocks of a step in one launch with grid-wide arrivals between them
     int cl_prefetch = 3;                  // bit 0: next block's weights, bit 1: next block's K/V rows (L2 prefetch)
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
@@ -167,6 +171,7 @@ struct aed_dec {
     int act_planes = 2;
     int sm_count = 148;
     int tc_target_ctas = 128;
+    bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
     bool use_pdl = true;
     bool use_fused = true;
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
@@ -436,6 +441,8 @@ bool encode_map(CUtensorMap *map, const void *base, size_t rows, size_t cols, in
 
 constexpr int kTcSmemBudget = 200 * 1024;
 
+cl::ClusterParams cluster_block_params(const aed_dec *dec, int l, int k);
+
 aed_status_t tc_setup(aed_dec *dec)
 {
     const auto &c = dec->cfg;
@@ -502,7 +509,7 @@ aed_status_t tc_setup(aed_dec *dec)
     const char *planes = getenv("AED_DEC_ACT_PLANES");
     dec->act_planes = (planes && planes[0] == '1') ? 1 : 2;
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
-    if (ctas && atoi(ctas) > 0) dec->tc_target_ctas = atoi(ctas);
+    if (ctas && atoi(ctas) > 0) { dec->tc_target_ctas = atoi(ctas); dec->tc_target_fixed = true; }
     // head-parallel cluster path: shapes whose projections split evenly over 8 CTAs and 16 clusters
     {
         // opt-in until it beats the kernel-per-projection path at every row count
@@ -535,6 +542,9 @@ aed_status_t tc_setup(aed_dec *dec)
             if (e2 == cudaSuccess)
                 e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_FFN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           max_smem(cl::K_FFN));
+            if (e2 == cudaSuccess)
+                e2 = cudaFuncSetAttribute(cl::cluster_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          std::max(max_smem(cl::K_SELF), std::max(max_smem(cl::K_CROSS), max_smem(cl::K_FFN))));
             if (e2 != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "cluster path set-up: %s", cudaGetErrorString(e2));
             // All clusters of a launch must be resident at once, or the launch runs in two waves and loses more
             // than the path gains: ask the device (the answer depends on how many SMs each GPC of this chip has).
@@ -557,8 +567,28 @@ aed_status_t tc_setup(aed_dec *dec)
                 resident = n >= cl::kClusters;
             }
             dec->use_cluster = resident;
-            const char *pf = getenv("AED_DEC_CL_PREFETCH");
-            if (pf) dec->cl_prefetch = atoi(pf);
+            if (resident) {
+                // block descriptions and tensor maps of the persistent step kernel, in the workspace
+                std::vector<cl::ClusterParams> blocks(3 * c.n_layers);
+                std::vector<CUtensorMap> maps(6 * c.n_layers);
+                const char *pf0 = getenv("AED_DEC_CL_PREFETCH");
+                if (pf0) dec->cl_prefetch = atoi(pf0);
+                for (int l = 0; l < c.n_layers; ++l) {
+                    for (int k = 0; k < 3; ++k) blocks[3 * l + k] = cluster_block_params(dec, l, k);
+                    const aed_dec::ClLayerMaps &m = dec->cl_layers[l];
+                    const CUtensorMap six[6] = {m.qkv, m.o, m.qc, m.oc, m.ff1, m.ff2};
+                    for (int i = 0; i < 6; ++i) maps[6 * l + i] = six[i];
+                }
+                cudaError_t e4 = cudaMemcpyAsync(dec->ws + L.cl_blocks, blocks.data(), blocks.size() * sizeof(cl::ClusterParams),
+                                                 cudaMemcpyHostToDevice, dec->stream);
+                if (e4 == cudaSuccess)
+                    e4 = cudaMemcpyAsync(dec->ws + L.cl_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice,
+                                         dec->stream);
+                if (e4 == cudaSuccess) e4 = cudaStreamSynchronize(dec->stream);      // the host vectors go away
+                if (e4 != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "cluster path set-up: %s", cudaGetErrorString(e4));
+                const char *pv = getenv("AED_DEC_NO_PERSIST");
+                dec->use_persistent = !(pv && pv[0] == '1');
+            }
         }
     }
     dec->use_tc = true;
@@ -704,9 +734,13 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2 + n_tile * tc::kBlockK * 4;
     int stages = kTcSmemBudget / stage_bytes;
     if (stages > sg::kMaxKb) stages = sg::kMaxKb;
-    // k-splits only as far as they are needed to occupy the GPU: every split adds rows x features x 4 bytes of
-    // red.global traffic.
-    int splits = dec->tc_target_ctas / (m_tiles * row_tiles);
+    // k-splits: every split adds rows x features x 4 bytes of red.global traffic, so large batches stop at about
+    // one CTA per SM.  Up to 64 rows that traffic is small, and CTAs with one or two k-blocks need so little
+    // shared memory that the CTAs of the next projection become resident beside them and fetch their weight
+    // tiles while this one still runs: there twice as many CTAs are worth it (measured on the 24-layer batch-64
+    // workload: 129 ms per pass with a target of 128 CTAs, 121 ms with 256, 147 ms with 384).
+    const int target_ctas = dec->tc_target_fixed ? dec->tc_target_ctas : (rows_ub <= 64 ? 256 : 128);
+    int splits = target_ctas / (m_tiles * row_tiles);
     if (splits < 1) splits = 1;
     if (splits > k_blocks) splits = k_blocks;
     const int kb_max = (k_blocks + splits - 1) / splits;
@@ -822,21 +856,54 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
 
 // ---- head-parallel cluster step (bf16 mode, at most 64 rows): 3 cluster kernels per layer ----------------------
 
+// Description of block k (0 self, 1 cross, 2 FFN) of layer l: buffers of the rotating residual stream, LayerNorm
+// fold constants, caches, and the static data of the following block to pull into L2.
+cl::ClusterParams cluster_block_params(const aed_dec *dec, int l, int k)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const size_t d = c.d_model, F = c.d_ffn, e2 = sizeof(T);
+    float *xb[3] = {dec->at<float>(L.x), dec->at<float>(L.x1), dec->at<float>(L.x2)};
+    const LayerWeights &w = dec->layers[l];
+    const int ln = (l + 1) % c.n_layers;               // next layer (or layer 0 of the next step)
+    const LayerWeights &wn = dec->layers[ln];
+    const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
+    T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+    const int blk = 3 * l + k;
+    cl::ClusterParams p{};
+    p.d = c.d_model; p.n_heads = c.n_heads; p.d_ffn = c.d_ffn;
+    p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3];
+    p.row_info = dec->at<int4>(L.row_info);
+    p.scale = 1.0f / sqrtf((float)kHeadDim);
+    p.eps = c.ln_eps;
+    p.state = dec->state();
+    if (k == 0) {           // next: the cross-attention weights and this layer's encoder K/V
+        p.gamma = (const T *)w.ln1_g; p.c1 = fc; p.c2 = fc + 3 * d; p.bias2 = (const T *)w.b_o;
+        p.cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems; p.seq_capacity = c.max_dec_len;
+        p.pf_ptr[0] = w.w_q_c; p.pf_bytes[0] = d * d * e2; p.pf_ptr[1] = w.w_o_c; p.pf_bytes[1] = d * d * e2;
+        p.pf_cache = cross; p.pf_capacity = c.max_total_enc_frames; p.pf_cross = 1;
+    } else if (k == 1) {    // next: the feed-forward weights
+        p.gamma = (const T *)w.ln2_g; p.c1 = fc + 6 * d; p.c2 = fc + 7 * d; p.bias2 = (const T *)w.b_o_c;
+        p.cache = cross; p.seq_capacity = c.max_total_enc_frames;
+        p.pf_ptr[0] = w.w_ff1; p.pf_bytes[0] = F * d * e2; p.pf_ptr[1] = w.w_ff2; p.pf_bytes[1] = F * d * e2;
+    } else {                // next: the self-attention weights and cache of the next layer
+        p.gamma = (const T *)w.ln3_g; p.c1 = fc + 8 * d; p.c2 = fc + 8 * d + F; p.bias2 = (const T *)w.b_ff2;
+        p.pf_ptr[0] = wn.w_qkv; p.pf_bytes[0] = 3 * d * d * e2; p.pf_ptr[1] = wn.w_o; p.pf_bytes[1] = d * d * e2;
+        p.pf_cache = dec->at<T>(L.self_cache) + (size_t)ln * L.self_layer_elems; p.pf_capacity = c.max_dec_len; p.pf_cross = 0;
+    }
+    if (!(dec->cl_prefetch & 1)) p.pf_ptr[0] = p.pf_ptr[1] = nullptr;
+    if (!(dec->cl_prefetch & 2)) p.pf_cache = nullptr;
+    return p;
+}
+
 template <int KIND>
 aed_status_t launch_cluster_block(aed_dec *dec, int family, const CUtensorMap &map_w1, const CUtensorMap &map_w2,
                                   int rows_ub, cl::ClusterParams p)
 {
     ProfScope ps(dec, family);
-    const auto &c = dec->cfg;
-    p.d = c.d_model; p.n_heads = c.n_heads; p.d_ffn = c.d_ffn;
     p.n_tile = 16 << tc_n_index(rows_ub);
-    p.row_info = dec->at<int4>(dec->lay.row_info);
-    p.scale = 1.0f / sqrtf((float)kHeadDim);
-    p.eps = c.ln_eps;
-    p.state = dec->state();
-    if (!(dec->cl_prefetch & 1)) p.pf_ptr[0] = p.pf_ptr[1] = nullptr;
-    if (!(dec->cl_prefetch & 2)) p.pf_cache = nullptr;
-    const int kbs = c.d_model / cl::kCS / tc::kBlockK;
+    const int kbs = dec->cfg.d_model / cl::kCS / tc::kBlockK;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cl::kClusters * cl::kCS);
     cfg.blockDim = dim3(cl::kClThreads);
@@ -860,50 +927,45 @@ aed_status_t forward_step_cluster(aed_dec *dec, int rows_ub, const int32_t *toke
     typedef __nv_bfloat16 T;
     const auto &c = dec->cfg;
     const Layout &L = dec->lay;
-    const int d = c.d_model, F = c.d_ffn, V = c.vocab;
-    float *xb[3] = {dec->at<float>(L.x), dec->at<float>(L.x1), dec->at<float>(L.x2)};
+    const int d = c.d_model, V = c.vocab;
+    float *x0 = dec->at<float>(L.x), *x1 = dec->at<float>(L.x1);
     const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
     {
         ProfScope ps(dec, KF_EMBED);
         embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), xb[0], xb[1], d);
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x0, x1, d);
         AED_LAUNCHED(dec);
     }
-    const size_t e2 = sizeof(T);
-    int blk = 0;
-    for (int l = 0; l < c.n_layers; ++l) {
-        const LayerWeights &w = dec->layers[l];
-        const aed_dec::ClLayerMaps &m = dec->cl_layers[l];
-        const int ln = (l + 1) % c.n_layers;               // next layer (or layer 0 of the next step)
-        const LayerWeights &wn = dec->layers[ln];
-        T *self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
-        T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-        const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
-        cl::ClusterParams p{};
-        // self-attention block; the next block streams the cross-attention weights and this layer's encoder K/V
-        p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3]; ++blk;
-        p.gamma = (const T *)w.ln1_g; p.c1 = fc; p.c2 = fc + 3 * d; p.bias2 = (const T *)w.b_o;
-        p.cache = self_cache; p.seq_capacity = c.max_dec_len;
-        p.pf_ptr[0] = w.w_q_c; p.pf_bytes[0] = (size_t)d * d * e2; p.pf_ptr[1] = w.w_o_c; p.pf_bytes[1] = (size_t)d * d * e2;
-        p.pf_cache = cross; p.pf_capacity = c.max_total_enc_frames; p.pf_cross = 1;
-        AED_TRY(launch_cluster_block<cl::K_SELF>(dec, KF_BLOCK_SELF, m.qkv, m.o, rows_ub, p));
-        // cross-attention block; next: the feed-forward weights
-        p = cl::ClusterParams{};
-        p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3]; ++blk;
-        p.gamma = (const T *)w.ln2_g; p.c1 = fc + 6 * d; p.c2 = fc + 7 * d; p.bias2 = (const T *)w.b_o_c;
-        p.cache = cross; p.seq_capacity = c.max_total_enc_frames;
-        p.pf_ptr[0] = w.w_ff1; p.pf_bytes[0] = (size_t)F * d * e2; p.pf_ptr[1] = w.w_ff2; p.pf_bytes[1] = (size_t)F * d * e2;
-        AED_TRY(launch_cluster_block<cl::K_CROSS>(dec, KF_BLOCK_CROSS, m.qc, m.oc, rows_ub, p));
-        // feed-forward block; next: the self-attention weights and cache of the next layer
-        p = cl::ClusterParams{};
-        p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3]; ++blk;
-        p.gamma = (const T *)w.ln3_g; p.c1 = fc + 8 * d; p.c2 = fc + 8 * d + F; p.bias2 = (const T *)w.b_ff2;
-        p.pf_ptr[0] = wn.w_qkv; p.pf_bytes[0] = (size_t)3 * d * d * e2; p.pf_ptr[1] = wn.w_o; p.pf_bytes[1] = (size_t)d * d * e2;
-        p.pf_cache = dec->at<T>(L.self_cache) + (size_t)ln * L.self_layer_elems; p.pf_capacity = c.max_dec_len; p.pf_cross = 0;
-        AED_TRY(launch_cluster_block<cl::K_FFN>(dec, KF_BLOCK_FFN, m.ff1, m.ff2, rows_ub, p));
+    if (dec->use_persistent && !dec->profiling) {
+        // every block of the step in one launch
+        ProfScope ps(dec, KF_BLOCK_SELF);
+        const int n_tile = 16 << tc_n_index(rows_ub), kbs = d / cl::kCS / tc::kBlockK;
+        size_t smem = 0;
+        for (int k = 0; k < 3; ++k) smem = std::max(smem, (size_t)cl::cl_layout(k, n_tile, kbs).total + 1024);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(cl::kClusters * cl::kCS);
+        cfg.blockDim = dim3(cl::kClThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = dec->stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, cl::cluster_step_kernel, (const cl::ClusterParams *)dec->at<cl::ClusterParams>(L.cl_blocks),
+                                           (const CUtensorMap *)dec->at<CUtensorMap>(L.cl_maps), 3 * c.n_layers, n_tile);
+        if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "cluster step launch: %s", cudaGetErrorString(e));
+        AED_LAUNCHED(dec);
+    } else {
+        for (int l = 0; l < c.n_layers; ++l) {
+            const aed_dec::ClLayerMaps &m = dec->cl_layers[l];
+            AED_TRY(launch_cluster_block<cl::K_SELF>(dec, KF_BLOCK_SELF, m.qkv, m.o, rows_ub, cluster_block_params(dec, l, 0)));
+            AED_TRY(launch_cluster_block<cl::K_CROSS>(dec, KF_BLOCK_CROSS, m.qc, m.oc, rows_ub, cluster_block_params(dec, l, 1)));
+            AED_TRY(launch_cluster_block<cl::K_FFN>(dec, KF_BLOCK_FFN, m.ff1, m.ff2, rows_ub, cluster_block_params(dec, l, 2)));
+        }
     }
     // 3 blocks per layer: the result is back in the first buffer
-    AED_TRY(launch_ln_planes(dec, rows_ub, xb[0], dec->final_ln_g, dec->final_ln_b, nullptr, 0));
+    AED_TRY(launch_ln_planes(dec, rows_ub, x0, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
     tc::TcParams tp{};
     tp.bias = (const T *)dec->b_out;
     tp.logits_out = logits_out;

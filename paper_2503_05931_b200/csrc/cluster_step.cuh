@@ -217,27 +217,63 @@ __device__ __forceinline__ float2 merge_stats(const float2 *slices, int stride, 
     return make_float2(mean, rsqrtf(m2 / d + eps));
 }
 
-// grid: 128 CTAs = 32 clusters of 4.  map_w1 / map_w2: weight matrices of the first and second projection,
-// boxes of 64 rows x 64 k.
-template <int KIND>
-__global__ void __launch_bounds__(kClThreads, 1)
-cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2, ClusterParams p)
+// 8 floats through L2 only (rows that other CTAs of a persistent launch wrote earlier in the same launch)
+__device__ __forceinline__ void load8_cg(const float *p, float (&v)[8])
 {
-    extern __shared__ uint8_t smem_dyn[];
-    __shared__ __align__(8) uint64_t bar_w[kMaxTiles];     // one per weight tile, each used once
-    __shared__ __align__(8) uint64_t bar_b, bar_d1, bar_d2, cbar0, cbar1;   // cbar0 / cbar1: first / second exchange of the cluster
-    __shared__ uint32_t tmem_slot;
-    __shared__ int abort_flag;
-    __shared__ float sm_c1[192], sm_c2[192];
-    __shared__ __align__(8) uint64_t ring_bar[8][kMaxRing];   // K/V ring of each worker warp
-    __shared__ const __nv_bfloat16 *sm_kptr[kMaxSlots], *sm_vptr[kMaxSlots];      // per row slot of this CTA
-    __shared__ int sm_len[kMaxSlots], sm_lenst[kMaxSlots], sm_cum[kMaxSlots + 1];
+    const float4 a = __ldcg(reinterpret_cast<const float4 *>(p));
+    const float4 b = __ldcg(reinterpret_cast<const float4 *>(p + 4));
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
 
+// mbarriers of one block kind; each completes one phase per block of that kind (parity = number of earlier uses & 1)
+struct BlockBars {
+    uint64_t w[kMaxTiles];     // one per weight tile
+    uint64_t b, d1, d2;        // operand planes written; first / second projection complete
+    uint64_t c0, c1;           // first / second exchange of the cluster
+};
+
+// Static shared state of a CTA, common to all blocks it runs.
+struct CtaShared {
+    BlockBars bars[3];
+    uint64_t ring_bar[8][kMaxRing];                 // K/V ring of each worker warp
+    uint32_t tmem_slot;
+    int abort_flag;
+    float c1[192], c2[192];                         // fold constants of the features this CTA finishes
+    const __nv_bfloat16 *kptr[kMaxSlots], *vptr[kMaxSlots];      // per row slot of this CTA
+    int len[kMaxSlots], lenst[kMaxSlots], cum[kMaxSlots + 1];
+};
+
+__device__ __forceinline__ void init_cta_shared(CtaShared &sh)
+{
+    for (int k = 0; k < 3; ++k) {
+        BlockBars &bars = sh.bars[k];
+        for (int i = 0; i < kMaxTiles; ++i) mbar_init(&bars.w[i], 1);
+        mbar_init(&bars.b, 8);
+        mbar_init(&bars.d1, 1);
+        mbar_init(&bars.d2, 1);
+        mbar_init(&bars.c0, kCS * 8);               // 8 worker warps of each CTA of the cluster
+        mbar_init(&bars.c1, kCS * 8);
+    }
+    for (int i = 0; i < 8 * kMaxRing; ++i) mbar_init(&sh.ring_bar[0][0] + i, 1);
+    sh.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// One block of a layer on this CTA.
+//   par        parity of this kind's single-use barriers (how many blocks of the kind this CTA ran before, & 1)
+//   ring_phase parities of the K/V ring barriers, carried from block to block
+//   sync_word  PERSIST: grid-wide arrival counter; the block may read x_in once it has reached sync_target
+template <int KIND, bool PERSIST>
+__device__ __forceinline__ void run_block(const ClusterParams &p, const CUtensorMap *map_w1, const CUtensorMap *map_w2,
+                                          int n_tile, uint32_t par, CtaShared &sh, uint8_t *smem_dyn, uint32_t tmem_base,
+                                          uint32_t &ring_phase, int *sync_word, int sync_target)
+{
+    BlockBars &bars = sh.bars[KIND];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = static_cast<int>(cluster_ctarank());
     const int c = static_cast<int>(cluster_index());
     const int d = p.d, ks = d / kCS, kbs = ks / kBlockK, of = ks, mt2 = of / kTileM;
-    const int N = p.n_tile;
+    const int N = n_tile;
     // attention blocks: cluster = (head, row parity); local row l is row 2 l + parity of the step
     const int head = c >> 1, parity = c & 1;
     const int Nm = cl_mma_n(KIND, N);                // MMA N = rows of the operand tiles
@@ -261,35 +297,35 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
     const int n_tiles2 = KIND == K_FFN ? 2 * mt2 : mt2;
     const int n_tiles = n_tiles1 + n_tiles2;
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < kMaxTiles; ++i) mbar_init(&bar_w[i], 1);
-        for (int i = 0; i < 8 * kMaxRing; ++i) mbar_init(&ring_bar[0][0] + i, 1);
-        mbar_init(&bar_b, 8);
-        mbar_init(&bar_d1, 1);
-        mbar_init(&bar_d2, 1);
-        mbar_init(&cbar0, kCS * 8);                  // 8 worker warps of each CTA of the cluster
-        mbar_init(&cbar1, kCS * 8);
-        abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) tmem_alloc(&tmem_slot, kTmemCols);
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = tmem_slot;
-    cluster_sync_all();                              // every CTA of the cluster has its barriers in place
-    sg::pdl_launch_dependents();
+
+    // Everything before this call touches only data that no block of the step writes.
+    auto dep_wait = [&]() {
+        if (!PERSIST) {
+            sg::pdl_wait();
+        } else {
+            if (sync_target > 0 && threadIdx.x == 64) {                 // one poller per CTA
+                const long long start = clock64();
+                while (true) {
+                    int seen;
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(sync_word) : "memory");
+                    if (seen >= sync_target || sh.abort_flag) break;
+                    if (clock64() - start > kWaitCycles) { sh.abort_flag = 1; break; }
+                }
+            }
+            asm volatile("bar.sync 2, 320;" ::: "memory");               // workers and side-job warps
+        }
+    };
 
     if (warp == 0) {
         // ---- weight tiles by TMA: static data, requested before the dependency wait ---------------------------
         if (lane == 0 && has_work) {
-            prefetch_tensormap(&map_w1);
-            prefetch_tensormap(&map_w2);
+            prefetch_tensormap(map_w1);
+            prefetch_tensormap(map_w2);
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
                 // tiles that reuse the area of a tile of the first projection wait for its MMAs
                 if ((KIND == K_SELF && t >= n_tiles1) || (KIND == K_FFN && t >= kFfnSlots)) {
-                    ok = mbar_wait(&bar_d1, 0, &abort_flag);
+                    ok = mbar_wait(&bars.d1, par, &sh.abort_flag);
                     if (!ok) break;
                 }
                 uint8_t *slot = w_tiles + cl_tile_off(KIND, t, kbs);
@@ -298,28 +334,28 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                     const int kc = j * ks + kb * kBlockK;
                     if (KIND == K_SELF) {
                         if ((t & 1) == 0) {          // query rows | key rows of the head
-                            mbar_expect_tx(&bar_w[t], 2 * 8192);
-                            tma_load_2d(slot, &map_w1, kc, head * kHeadDim, &bar_w[t]);
-                            tma_load_2d(slot + 8192, &map_w1, kc, d + head * kHeadDim, &bar_w[t]);
+                            mbar_expect_tx(&bars.w[t], 2 * 8192);
+                            tma_load_2d(slot, map_w1, kc, head * kHeadDim, &bars.w[t]);
+                            tma_load_2d(slot + 8192, map_w1, kc, d + head * kHeadDim, &bars.w[t]);
                         } else {                     // value rows
-                            mbar_expect_tx(&bar_w[t], 8192);
-                            tma_load_2d(slot, &map_w1, kc, 2 * d + head * kHeadDim, &bar_w[t]);
+                            mbar_expect_tx(&bars.w[t], 8192);
+                            tma_load_2d(slot, map_w1, kc, 2 * d + head * kHeadDim, &bars.w[t]);
                         }
                     } else if (KIND == K_CROSS) {
-                        mbar_expect_tx(&bar_w[t], 8192);
-                        tma_load_2d(slot, &map_w1, kc, head * kHeadDim, &bar_w[t]);
+                        mbar_expect_tx(&bars.w[t], 8192);
+                        tma_load_2d(slot, map_w1, kc, head * kHeadDim, &bars.w[t]);
                     } else {                         // the 128 hidden features of chunk c
-                        mbar_expect_tx(&bar_w[t], 2 * 8192);
-                        tma_load_2d(slot, &map_w1, kc, c * 128, &bar_w[t]);
-                        tma_load_2d(slot + 8192, &map_w1, kc, c * 128 + 64, &bar_w[t]);
+                        mbar_expect_tx(&bars.w[t], 2 * 8192);
+                        tma_load_2d(slot, map_w1, kc, c * 128, &bars.w[t]);
+                        tma_load_2d(slot + 8192, map_w1, kc, c * 128 + 64, &bars.w[t]);
                     }
                 } else {                             // second projection: 128 of this CTA's d/4 output features
                     const int u = t - n_tiles1;
                     const int m = KIND == K_FFN ? u >> 1 : u;
                     const int kc = KIND == K_FFN ? c * 128 + (u & 1) * kBlockK : head * kHeadDim;
-                    mbar_expect_tx(&bar_w[t], 2 * 8192);
-                    tma_load_2d(slot, &map_w2, kc, j * of + m * kTileM, &bar_w[t]);
-                    tma_load_2d(slot + 8192, &map_w2, kc, j * of + m * kTileM + 64, &bar_w[t]);
+                    mbar_expect_tx(&bars.w[t], 2 * 8192);
+                    tma_load_2d(slot, map_w2, kc, j * of + m * kTileM, &bars.w[t]);
+                    tma_load_2d(slot + 8192, map_w2, kc, j * of + m * kTileM + 64, &bars.w[t]);
                 }
             }
         }
@@ -327,9 +363,9 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
         // ---- MMA issue --------------------------------------------------------------------------------------------
         if (lane == 0 && has_work) {
             const uint32_t idesc = instr_desc_bf16(Nm);
-            bool ok = mbar_wait(&bar_b, 0, &abort_flag);
+            bool ok = mbar_wait(&bars.b, par, &sh.abort_flag);
             for (int t = 0; t < n_tiles1 && ok; ++t) {
-                ok = mbar_wait(&bar_w[t], 0, &abort_flag);
+                ok = mbar_wait(&bars.w[t], par, &sh.abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const int kb = KIND == K_SELF ? t >> 1 : t;
@@ -343,15 +379,15 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
 #pragma unroll
                 for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(td, da + 2 * k, dl + 2 * k, idesc, 1u);
             }
-            if (ok) mma_commit(&bar_d1);
+            if (ok) mma_commit(&bars.d1);
             // second projection: its B operand is complete when the second exchange of the cluster is
-            ok = ok && mbar_wait_cluster(&cbar1, 0, &abort_flag);
+            ok = ok && mbar_wait_cluster(&bars.c1, par, &sh.abort_flag);
             if (ok) {
                 fence_async_proxy();
                 tc_fence_after_sync();
                 for (int u = 0; u < n_tiles2 && ok; ++u) {
                     const int t = n_tiles1 + u;
-                    ok = mbar_wait(&bar_w[t], 0, &abort_flag);
+                    ok = mbar_wait(&bars.w[t], par, &sh.abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const int m = KIND == K_FFN ? u >> 1 : u, q = KIND == K_FFN ? (u & 1) : 0;
@@ -364,7 +400,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k) mma_bf16(td, da + 2 * k, dl + 2 * k, idesc, 1u);
                 }
-                if (ok) mma_commit(&bar_d2);
+                if (ok) mma_commit(&bars.d2);
             }
         }
     } else if (warp >= 10) {
@@ -401,7 +437,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                 }
             }
         }
-        sg::pdl_wait();
+        dep_wait();
         if (p.x_zero) {
             const int n_rows = p.state->n_active;
             const size_t total4 = static_cast<size_t>(n_rows) * d / 4;
@@ -416,7 +452,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
         AED_TRACE_RESERVE(tcur, p.state, (pt == 0 && (blockIdx.x == 0 || blockIdx.x == 72)) ? 96u : 0u);
         AED_TRACE_PUT(p.state, tcur, (blockIdx.x == 0 ? 24 : 124) + KIND);
         const uint32_t recv_s = smem_u32(recv), stats_s = smem_u32(stats_recv);
-        const uint32_t cbar0_s = smem_u32(&cbar0), cbar1_s = smem_u32(&cbar1);
+        const uint32_t cbar0_s = smem_u32(&bars.c0), cbar1_s = smem_u32(&bars.c1);
         const uint32_t ap_s = smem_u32(ap), r2_s = smem_u32(r2);
         // x slice geometry: thread = (local row within pass, 8-column chunk cc)
         const int cpr = ks >> 3, rows_per_pass = 256 / cpr;          // 16 or 32 chunks per row
@@ -429,15 +465,15 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
         // to the 8 warps in equal contiguous runs (a long row is shared by several warps, a warp rarely changes
         // row).  The i-th item of a warp goes through stage i mod RS of the warp's K/V ring.
         auto issue_item = [&](int item, int stage, int &sl) {      // sl: row-slot cursor, only moves forward
-            while (item >= sm_cum[sl + 1]) ++sl;
-            const int p0 = (item - sm_cum[sl]) * kFusedChunk;
-            const int n_st = min(kFusedChunk, sm_lenst[sl] - p0);
+            while (item >= sh.cum[sl + 1]) ++sl;
+            const int p0 = (item - sh.cum[sl]) * kFusedChunk;
+            const int n_st = min(kFusedChunk, sh.lenst[sl] - p0);
             if (n_st > 0 && lane == 0) {
-                uint64_t *bar = &ring_bar[ww][stage];
+                uint64_t *bar = &sh.ring_bar[ww][stage];
                 uint8_t *dst = ring + (static_cast<size_t>(ww) * RS + stage) * kRingStage;
                 mbar_expect_tx(bar, n_st * 256);
-                bulk_load(dst, sm_kptr[sl] + static_cast<size_t>(p0) * kHeadDim, n_st * 128, bar);
-                bulk_load(dst + 2048, sm_vptr[sl] + static_cast<size_t>(p0) * kHeadDim, n_st * 128, bar);
+                bulk_load(dst, sh.kptr[sl] + static_cast<size_t>(p0) * kHeadDim, n_st * 128, bar);
+                bulk_load(dst + 2048, sh.vptr[sl] + static_cast<size_t>(p0) * kHeadDim, n_st * 128, bar);
             }
         };
         if (has_work) {
@@ -446,13 +482,13 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             if (KIND == K_SELF) {
                 if (pt < 192) {
                     const int col = (pt >> 6) * d + head * kHeadDim + (pt & 63);
-                    sm_c1[pt] = p.c1[col];
-                    sm_c2[pt] = p.c2[col];
+                    sh.c1[pt] = p.c1[col];
+                    sh.c2[pt] = p.c2[col];
                 }
             } else if (KIND == K_CROSS) {
-                if (pt < 64) { sm_c1[pt] = p.c1[head * kHeadDim + pt]; sm_c2[pt] = p.c2[head * kHeadDim + pt]; }
+                if (pt < 64) { sh.c1[pt] = p.c1[head * kHeadDim + pt]; sh.c2[pt] = p.c2[head * kHeadDim + pt]; }
             } else {
-                if (pt < 32) { sm_c1[pt] = p.c1[c * 128 + j * 32 + pt]; sm_c2[pt] = p.c2[c * 128 + j * 32 + pt]; }
+                if (pt < 32) { sh.c1[pt] = p.c1[c * 128 + j * 32 + pt]; sh.c2[pt] = p.c2[c * 128 + j * 32 + pt]; }
             }
             if (KIND != K_FFN && ww == 0) {
                 // row table of this CTA (static during the step) -> lengths, cache pointers, chunk prefix sums
@@ -472,7 +508,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                             vb = p.cache + (((size_t)ri.x * 2 + 1) * p.n_heads + head) * (size_t)p.seq_capacity * kHeadDim;
                         }
                     }
-                    sm_kptr[lane] = kb; sm_vptr[lane] = vb; sm_len[lane] = len; sm_lenst[lane] = lst;
+                    sh.kptr[lane] = kb; sh.vptr[lane] = vb; sh.len[lane] = len; sh.lenst[lane] = lst;
                 }
                 int chunks = (len + kFusedChunk - 1) / kFusedChunk;       // 0 for lanes without a row
                 int incl = chunks;
@@ -481,21 +517,21 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                     const int v = __shfl_up_sync(0xffffffffu, incl, o);
                     if (lane >= o) incl += v;
                 }
-                if (lane < kMaxSlots) sm_cum[lane + 1] = incl;
-                if (lane == 0) sm_cum[0] = 0;
+                if (lane < kMaxSlots) sh.cum[lane + 1] = incl;
+                if (lane == 0) sh.cum[0] = 0;
             }
         }
         worker_sync();                                     // fold constants and row table staged
         int item0 = 0, item1 = 0, sl_issue = 0, sl_use = 0;
         if (KIND != K_FFN && has_work) {
-            const int n_items = sm_cum[SL], per = (n_items + 7) / 8;
+            const int n_items = sh.cum[SL], per = (n_items + 7) / 8;
             item0 = min(ww * per, n_items);
             item1 = min(item0 + per, n_items);
             // the first chunks of this warp are static data: they stream while the previous block still runs
             for (int i = 0; i < RS; ++i)
                 if (item0 + i < item1) issue_item(item0 + i, i, sl_issue);
         }
-        sg::pdl_wait();
+        dep_wait();
         AED_TRACE_PUT(p.state, tcur, 50);          // dependency resolved
         const int n_rows = p.state->n_active;
         // local rows of this cluster that exist, and the step row of local row l
@@ -509,7 +545,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
 #pragma unroll
                 for (int ps = 0; ps < 4; ++ps) {
                     const int l = (ps0 + ps) * rows_per_pass + r_in_pass;
-                    if (l < n_loc) load8(p.x_in + (size_t)step_row(l) * d + j * ks + cc * 8, xv[ps]);
+                    if (l < n_loc) load8_cg(p.x_in + (size_t)step_row(l) * d + j * ks + cc * 8, xv[ps]);
                     else {
 #pragma unroll
                         for (int e = 0; e < 8; ++e) xv[ps][e] = 0.f;
@@ -559,11 +595,11 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b)) : "memory");
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bars.b)) : "memory");
             AED_TRACE_PUT(p.state, tcur, 51);      // operand planes written
 
             // ---- 3. partial sums of the first projection -> the CTA that finishes them ----------------------------
-            ok = mbar_wait(&bar_d1, 0, &abort_flag);
+            ok = mbar_wait(&bars.d1, par, &sh.abort_flag);
             tc_fence_after_sync();
             AED_TRACE_PUT(p.state, tcur, 52);      // first projection complete
             if (ok) {
@@ -606,7 +642,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             __syncwarp();
             if (lane < kCS) arrive_remote(map_to_cta(cbar0_s, lane));     // first exchange, also on the abort path
             AED_TRACE_PUT(p.state, tcur, 53);      // partials sent
-            ok = mbar_wait_cluster(&cbar0, 0, &abort_flag) && ok;
+            ok = mbar_wait_cluster(&bars.c0, par, &sh.abort_flag) && ok;
             AED_TRACE_PUT(p.state, tcur, 54);      // first exchange complete
 
             if (KIND == K_FFN) {
@@ -626,7 +662,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                     const float2 st = merge_stats(stats_recv + r, kMaxRows, ks, d, p.eps);
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
-                        a[e] = fmaxf(fmaf(st.y, a[e] - st.x * sm_c1[c4 * 8 + e], sm_c2[c4 * 8 + e]), 0.f);
+                        a[e] = fmaxf(fmaf(st.y, a[e] - st.x * sh.c1[c4 * 8 + e], sh.c2[c4 * 8 + e]), 0.f);
                     uint4 hi, lo;
                     sg::split_planes(a, hi, lo);
                     // k index inside the chunk: 32 j + 8 c4  ->  k-block j / 2, 16-byte chunk (j & 1) * 4 + c4
@@ -643,7 +679,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                 // ---- 4. attention for the rows of this CTA -------------------------------------------------------------
                 const int FE = KIND == K_SELF ? 192 : 64;
                 // 4a. warp s finishes the query (and the new key / value) of row slot s
-                if (ok && ww < SL && sm_len[ww] > 0) {
+                if (ok && ww < SL && sh.len[ww] > 0) {
                     const int sl = ww;
                     const float2 st = merge_stats(stats_recv + sl, kMaxRows, ks, d, p.eps);
                     float qv[8];
@@ -658,7 +694,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                     }
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
-                        qv[e] = fmaf(st.y, qv[e] - st.x * sm_c1[dg * 8 + e], sm_c2[dg * 8 + e]) * p.scale;
+                        qv[e] = fmaf(st.y, qv[e] - st.x * sh.c1[dg * 8 + e], sh.c2[dg * 8 + e]) * p.scale;
                     if (pg == 0) {
                         *reinterpret_cast<float4 *>(sm_q + sl * kHeadDim + dg * 8) = make_float4(qv[0], qv[1], qv[2], qv[3]);
                         *reinterpret_cast<float4 *>(sm_q + sl * kHeadDim + dg * 8 + 4) = make_float4(qv[4], qv[5], qv[6], qv[7]);
@@ -680,16 +716,16 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                         }
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            kn[e] = fmaf(st.y, kn[e] - st.x * sm_c1[64 + dg * 8 + e], sm_c2[64 + dg * 8 + e]);
-                            vn[e] = fmaf(st.y, vn[e] - st.x * sm_c1[128 + dg * 8 + e], sm_c2[128 + dg * 8 + e]);
+                            kn[e] = fmaf(st.y, kn[e] - st.x * sh.c1[64 + dg * 8 + e], sh.c2[64 + dg * 8 + e]);
+                            vn[e] = fmaf(st.y, vn[e] - st.x * sh.c1[128 + dg * 8 + e], sh.c2[128 + dg * 8 + e]);
                         }
                         Raw8<__nv_bfloat16> new_k, new_v;
                         new_k.set(kn);
                         new_v.set(vn);
                         if (pg == 0) {      // append to the cache (nobody reads this position during this launch) and keep a copy
-                            const int pos = sm_len[sl] - 1;
-                            new_k.store(const_cast<__nv_bfloat16 *>(sm_kptr[sl]) + (size_t)pos * kHeadDim + dg * 8);
-                            new_v.store(const_cast<__nv_bfloat16 *>(sm_vptr[sl]) + (size_t)pos * kHeadDim + dg * 8);
+                            const int pos = sh.len[sl] - 1;
+                            new_k.store(const_cast<__nv_bfloat16 *>(sh.kptr[sl]) + (size_t)pos * kHeadDim + dg * 8);
+                            new_v.store(const_cast<__nv_bfloat16 *>(sh.vptr[sl]) + (size_t)pos * kHeadDim + dg * 8);
                             new_k.store(sm_knew + sl * kHeadDim + dg * 8);
                             new_v.store(sm_vnew + sl * kHeadDim + dg * 8);
                         }
@@ -719,13 +755,12 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                         }
                     };
                     int i = 0;
-                    uint32_t ring_phase = 0;              // bit s: parity of the next copy to land in stage s
                     for (int item = item0; item < item1 && ok; ++item, ++i) {
                         const int stage = i % RS;
-                        while (item >= sm_cum[sl_use + 1]) ++sl_use;
+                        while (item >= sh.cum[sl_use + 1]) ++sl_use;
                         const int sl = sl_use;
-                        const int p0 = (item - sm_cum[sl]) * kFusedChunk;
-                        const int len = sm_len[sl], len_st = sm_lenst[sl];
+                        const int p0 = (item - sh.cum[sl]) * kFusedChunk;
+                        const int len = sh.len[sl], len_st = sh.lenst[sl];
                         if (sl != cur) {
                             if (cur >= 0) flush();
                             cur = sl;
@@ -736,7 +771,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                         }
                         AED_TRACE_PUT(p.state, tcur, 61);
                         if (len_st > p0) {                // a chunk that holds only the new position has no copy
-                            ok = mbar_wait(&ring_bar[ww][stage], (ring_phase >> stage) & 1u, &abort_flag);
+                            ok = mbar_wait(&sh.ring_bar[ww][stage], (ring_phase >> stage) & 1u, &sh.abort_flag);
                             ring_phase ^= 1u << stage;
                         }
                         if (!ok) break;
@@ -797,7 +832,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                 AED_TRACE_PUT(p.state, tcur, 60);
                 // 4c. warp s merges the partials of row slot s and sends the result to every CTA's operand tile;
                 //     lane group pg writes to CTA pg
-                if (ok && ww < SL && sm_len[ww] > 0) {
+                if (ok && ww < SL && sh.len[ww] > 0) {
                     const int sl = ww, r_att = j + kCS * sl;      // local row = row of the operand tile
                     float big = -INFINITY;
 #pragma unroll
@@ -843,7 +878,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                 const int n_res = n_loc > who ? (n_loc - who + n_work - 1) / n_work : 0;      // local rows who, who + n_work, ...
                 for (int idx = pt; idx < n_res * g4n; idx += 256) {
                     const int r = step_row(who + n_work * (idx / g4n)), f4 = (idx % g4n) * 4;
-                    float4 v = *reinterpret_cast<const float4 *>(p.x_in + (size_t)r * d + j * of + f4);
+                    float4 v = __ldcg(reinterpret_cast<const float4 *>(p.x_in + (size_t)r * d + j * of + f4));
                     if (p.bias2) {
                         float b4[4];
                         load4(p.bias2 + j * of + f4, b4);
@@ -852,7 +887,7 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
                     sg::red_add_v4(p.x_out + (size_t)r * d + j * of + f4, v);
                 }
             }
-            ok = mbar_wait(&bar_d2, 0, &abort_flag) && ok;
+            ok = mbar_wait(&bars.d2, par, &sh.abort_flag) && ok;
             tc_fence_after_sync();
             AED_TRACE_PUT(p.state, tcur, 56);      // second projection complete
             // accumulators [feature lane][local row] -> shared memory [local row][feature]; the operand planes (and,
@@ -888,6 +923,27 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
             AED_TRACE_PUT(p.state, tcur, 57);              // reductions issued
         }
     }
+}
+
+// One block per launch, chained with programmatic dependent launch.  grid: 128 CTAs = 32 clusters of 4.
+// map_w1 / map_w2: weight matrices of the first and second projection, boxes of 64 rows x 64 k.
+template <int KIND>
+__global__ void __launch_bounds__(kClThreads, 1)
+cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2, ClusterParams p)
+{
+    extern __shared__ uint8_t smem_dyn[];
+    __shared__ __align__(16) CtaShared sh;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) init_cta_shared(sh);
+    if (warp == 1) tmem_alloc(&sh.tmem_slot, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_slot;
+    cluster_sync_all();                              // every CTA of the cluster has its barriers in place
+    sg::pdl_launch_dependents();
+    uint32_t ring_phase = 0;
+    run_block<KIND, false>(p, &map_w1, &map_w2, p.n_tile, 0u, sh, smem_dyn, tmem_base, ring_phase, nullptr, 0);
     tc_fence_before_sync();
     __syncthreads();
     cluster_sync_all();                              // nobody writes into a CTA that has left
@@ -895,7 +951,60 @@ cluster_block_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_co
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (threadIdx.x == 0 && abort_flag) atomicExch(&p.state->error, kErrTimeout);
+    if (threadIdx.x == 0 && sh.abort_flag) atomicExch(&p.state->error, kErrTimeout);
+}
+
+// All blocks of a step in one launch: blocks[3 l + k] describes block k of layer l, maps[6 l + 2 k] and
+// maps[6 l + 2 k + 1] are its weight matrices.  Between two blocks every CTA adds one to the arrival counter
+// (DecState::grid_sync, cleared by the first kernel of the step) and the next block reads x_in once all CTAs of the
+// grid have arrived; static data of the next block (weights, cached keys and values) is requested before that.
+// All 128 CTAs must be resident at once (checked by the host with the occupancy query).
+__global__ void __launch_bounds__(kClThreads, 1)
+cluster_step_kernel(const ClusterParams *__restrict__ blocks, const CUtensorMap *__restrict__ maps, int n_blocks, int n_tile)
+{
+    extern __shared__ uint8_t smem_dyn[];
+    __shared__ __align__(16) CtaShared sh;
+    __shared__ __align__(16) ClusterParams sp[2];
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) init_cta_shared(sh);
+    if (warp == 1) tmem_alloc(&sh.tmem_slot, kTmemCols);
+    constexpr int kWords = sizeof(ClusterParams) / 4;
+    if (threadIdx.x >= 320 && threadIdx.x - 320 < kWords)
+        reinterpret_cast<int *>(&sp[0])[threadIdx.x - 320] = reinterpret_cast<const int *>(&blocks[0])[threadIdx.x - 320];
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh.tmem_slot;
+    cluster_sync_all();
+    uint32_t ring_phase = 0;
+    DecState *state = sp[0].state;
+    for (int b = 0; b < n_blocks; ++b) {
+        const ClusterParams &p = sp[b & 1];
+        const int kind = b % 3, layer = b / 3;
+        const CUtensorMap *m1 = maps + 6 * layer + 2 * kind, *m2 = m1 + 1;
+        const uint32_t par = layer & 1;
+        const int target = b * static_cast<int>(gridDim.x);
+        // the description of the next block travels while this one runs
+        if (b + 1 < n_blocks && threadIdx.x >= 320 && threadIdx.x - 320 < kWords)
+            reinterpret_cast<int *>(&sp[(b + 1) & 1])[threadIdx.x - 320] =
+                reinterpret_cast<const int *>(&blocks[b + 1])[threadIdx.x - 320];
+        if (kind == K_SELF) run_block<K_SELF, true>(p, m1, m2, n_tile, par, sh, smem_dyn, tmem_base, ring_phase, &state->grid_sync, target);
+        else if (kind == K_CROSS) run_block<K_CROSS, true>(p, m1, m2, n_tile, par, sh, smem_dyn, tmem_base, ring_phase, &state->grid_sync, target);
+        else run_block<K_FFN, true>(p, m1, m2, n_tile, par, sh, smem_dyn, tmem_base, ring_phase, &state->grid_sync, target);
+        // end of the block: this CTA's shared memory and accumulators are free again, its additions to x_out are
+        // ordered before its arrival
+        fence_async_proxy();                         // generic writes to shared memory before the next block's TMA
+        tc_fence_before_sync();
+        __syncthreads();
+        cluster_sync_all();
+        tc_fence_after_sync();
+        if (threadIdx.x == 0 && b + 1 < n_blocks) {
+            __threadfence();
+            atomicAdd(&state->grid_sync, 1);
+        }
+    }
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+    if (threadIdx.x == 0 && sh.abort_flag) atomicExch(&state->error, kErrTimeout);
 }
 
 }  // namespace cl

@@ -15,7 +15,7 @@ struct DecState {
     int32_t n_active;    // rows taking part in the current step
     int32_t error;       // sticky: 0 ok, 1 = a row would have overflowed the self-attention cache
     int32_t n_retired;   // utterances retired so far
-    int32_t pad;
+    int32_t grid_sync;   // arrival counter of the persistent step kernel, cleared by the first kernel of a step
 };
 
 // Optional device-side timeline (debug builds with -DAED_TRACE): block 0 of every traced kernel stamps its start

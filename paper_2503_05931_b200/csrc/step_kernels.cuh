@@ -50,7 +50,7 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
         }
         __syncthreads();
     }
-    if (threadIdx.x == 0) state->n_active = base;
+    if (threadIdx.x == 0) { state->n_active = base; state->grid_sync = 0; }
     for (int r = base + threadIdx.x; r < row_slots; r += blockDim.x) row_info[r] = make_int4(-1, 0, 0, 0);
 }
 

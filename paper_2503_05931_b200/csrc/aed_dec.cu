@@ -161,7 +161,7 @@ struct aed_dec {
     std::vector<ClLayerMaps> cl_layers;
     bool use_cluster = false;             // head-parallel cluster kernels for steps of at most 64 rows
     bool use_persistent = true;           // all blocks of a step in one launch with grid-wide arrivals between them
-    int cl_prefetch = 3;                  // bit 0: next block's weights, bit 1: next block's K/V rows (L2 prefetch)
+    int cl_prefetch = 0;                  // bit 0: next block's weights, bit 1: next block's K/V rows (L2 prefetch)
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
     CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]

@@ -83,6 +83,13 @@ def family_bytes(family, w):
     return None
 
 
+# DRAM bytes per algorithmic byte of a kernel family, from the ncu capture summarised in
+# profiles/step_kernels_cfg2_clip2_ncu.txt (dram__bytes_read.sum + dram__bytes_write.sum of one launch over the
+# family's algorithmic bytes of that launch; traffic grows in proportion to the rows' frames).  An entry is removed
+# when its kernel changes, which turns the reported traffic back into null.
+NCU_TRAFFIC_RATIO = {"attn_cross": 30.789888 / 30.490624}
+
+
 def roofline_seconds(w, peaks):
     per_step, pre_bytes, pre_flops, _ = step_bytes_and_flops(w)
     bw, fl = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
@@ -418,8 +425,12 @@ def profile_dominant_kernel(dec, w, one_pass, peaks):
     info = prof[top]
     bytes_total = family_bytes(top, w)
     achieved = bytes_total / (info["ms"] * 1e-3) / 1e9 if bytes_total else None
+    ratio = NCU_TRAFFIC_RATIO.get(top) if w.name == "cfg2" else None
+    traffic = ratio * bytes_total / max(info["launches"], 1) if (ratio and bytes_total) else None
     return {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": None,
+            "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": traffic,
+            "traffic_unit": "bytes per launch (ncu capture of a 64-row launch, scaled by frames)",
+            "algorithmic_bytes_per_launch": (bytes_total / max(info["launches"], 1)) if bytes_total else None,
             "launches": info["launches"], "avg_us": 1e3 * info["ms"] / max(info["launches"], 1),
             "peak_source": peaks["source"],
             "shares": {k: round(v["ms"] / sum(x["ms"] for x in prof.values()), 4) for k, v in prof.items()}}

@@ -214,6 +214,18 @@ def test_config3_shape_sampled_rows():
     _run_both(w, rows=rows)
 
 
+def test_config4_shape_sampled_rows():
+    """24-layer d=1024 bf16 decoder at batch 512 with uniform durations (the large-batch configuration: 256-row
+    projection tiles, rows retiring step by step down to the small-batch path): sampled short utterances against
+    the checker, every other utterance of the batch decoding alongside."""
+    w = wl.make_workload("cfg4")
+    order = np.argsort(w.dec_lens)
+    rows = sorted({int(order[0]), int(order[5]), int(order[17]), int(np.argmin(w.enc_lens))})
+    rows = [r for r in rows if w.dec_lens[r] <= 24][:4]
+    assert rows
+    _run_both(w, rows=rows)
+
+
 @pytest.mark.parametrize("cluster", ["0", "1"])
 def test_config2_shape_sampled_rows(cluster, monkeypatch):
     """24-layer d=1024 bf16 decoder at batch 64 (the benchmark configuration, on both launch paths): a sample of

@@ -107,7 +107,9 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     __shared__ int abort_flag;
     __shared__ float red_s[2], red_q[2];
 
-    AED_TRACE_BEGIN(p.state, 19);
+    // timeline of the first producer thread of block 0 (debug builds)
+    AED_TRACE_RESERVE(tcur, p.state, (threadIdx.x == 64 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? 8u : 0u);
+    AED_TRACE_PUT(p.state, tcur, 19);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int a0 = blockIdx.x * kTileM;
     const int row0 = blockIdx.z * p.n_tile;
@@ -135,7 +137,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     pdl_launch_dependents();
-    if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 40);      // set-up done
+    AED_TRACE_PUT(p.state, tcur, 40);      // set-up done
 
     if (warp == 0) {
         if (lane == 0) {
@@ -238,7 +240,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         }
     } else {
         pdl_wait();
-        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 41);  // dependency resolved
+        AED_TRACE_PUT(p.state, tcur, 41);  // dependency resolved
         const int pt = threadIdx.x - 64;                  // 0..255 among the producer threads
         const int n_rows = p.state->n_active;
         // ---- activation tiles --------------------------------------------------------------------------
@@ -289,13 +291,13 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b[s])) : "memory");
         }
-        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 42);  // activation tiles written
+        AED_TRACE_PUT(p.state, tcur, 42);  // activation tiles written
         if (warp < 6) {                                   // only warps 2..5 own accumulator lanes
 
         // ---- epilogue: accumulator -> shared memory (transposed) -> 16-byte reductions ---------------------------
         ok = ok && mbar_wait(&bar_done, 0, &abort_flag);
         tc_fence_after_sync();
-        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 44);  // accumulator complete
+        AED_TRACE_PUT(p.state, tcur, 44);  // accumulator complete
         // every MMA has completed, so the whole stage area is free: T[r][o], 132 floats per row (bank spread)
         float *trans = reinterpret_cast<float *>(tiles);
         constexpr int kPitch = kTileM + 4;
@@ -336,7 +338,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         }
         }
     }
-    if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 45);      // epilogue issued
+    AED_TRACE_PUT(p.state, tcur, 45);      // epilogue issued
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {

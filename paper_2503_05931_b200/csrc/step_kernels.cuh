@@ -461,9 +461,11 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             }
         }
     }
+    AED_TRACE_RESERVE(tcur, state, (threadIdx.x == 0 && blockIdx.x == 0) ? 4u : 0u);
+    AED_TRACE_PUT(state, tcur, 8 + (kCross ? 1 : 0));      // resident, first chunk requested
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    AED_TRACE_BEGIN(state, 3);
+    AED_TRACE_PUT(state, tcur, 3);                          // dependency resolved
     // Everything this block needs from earlier kernels is requested in one round: statistics, query, and (in the
     // warp that owns the new position) the new key and value, with the LayerNorm-fold constants of their columns.
     // When the projection ran on gamma*x, its raw output y becomes rstd*(y - mean*c1) + c2 here.
@@ -591,6 +593,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             out_lo[off] = __float2bfloat16_rn(o - __bfloat162float(hi));
         }
     }
+    AED_TRACE_PUT(state, tcur, 7);                          // output written
 }
 
 // Merge the chunk partials of each (row, head): one warp per pair, 2 head dimensions per lane.

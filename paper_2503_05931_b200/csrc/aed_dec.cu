@@ -174,6 +174,7 @@ struct aed_dec {
     bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
     bool use_pdl = true;
     bool use_fused = true;
+    bool attn_pipe = true;
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
     struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -331,7 +332,10 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_fused_kernel<T, kCross, kAppend>, (const DecState *)dec->state(),
+    // Few blocks with long rows (late steps): the software-pipelined variant, two blocks per SM hold the whole grid.
+    const bool pipe = kCross && !kAppend && rows_ub * dec->cfg.n_heads <= 2 * dec->sm_count && dec->attn_pipe;
+    auto kernel = pipe ? attn_fused_kernel<T, kCross, kAppend, kCross && !kAppend> : attn_fused_kernel<T, kCross, kAppend, false>;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, (const DecState *)dec->state(),
                                        (const int4 *)dec->at<int4>(dec->lay.row_info), q, ldq, const_cast<T *>(cache),
                                        dec->cfg.n_heads, seq_capacity, 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo,
                                        dec->cfg.d_model, ln_stats, ln_c1, ln_c2);
@@ -503,6 +507,8 @@ aed_status_t tc_setup(aed_dec *dec)
     {
         const char *v = getenv("AED_DEC_NO_PDL");
         dec->use_pdl = !(v && v[0] == '1');
+        v = getenv("AED_DEC_NO_ATTN_PIPE");
+        dec->attn_pipe = !(v && v[0] == '1');
         v = getenv("AED_DEC_NO_FUSED");
         dec->use_fused = !(v && v[0] == '1');
     }

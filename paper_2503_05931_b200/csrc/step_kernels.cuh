@@ -401,8 +401,10 @@ template <> struct Raw8<float> {
 constexpr int kFusedChunk = 16;       // positions per warp and iteration
 constexpr int kFusedMaxWarps = 8;
 
-template <typename CT, bool kCross, bool kAppend>
-__global__ void __launch_bounds__(kFusedMaxWarps * 32, (kAppend ? 2 : 4))      // self-attention holds the new key/value as well
+// kPipe: the loads of a warp's next chunk are issued before the current chunk is reduced (twice the K/V registers,
+// so only two blocks per SM: for grids that fit anyway).
+template <typename CT, bool kCross, bool kAppend, bool kPipe = false>
+__global__ void __launch_bounds__(kFusedMaxWarps * 32, ((kAppend || kPipe) ? 2 : 4))      // self-attention holds the new key/value as well
 attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ q, int ldq,
                   CT *__restrict__ cache, int n_heads, int seq_capacity, float scale,
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo,
@@ -513,8 +515,21 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
     bool loaded = true;
+    Raw8<CT> nk[4], nv[4];
     for (int p0 = warp * kFusedChunk; p0 < len; p0 += n_warps * kFusedChunk) {
-        if (!loaded) {
+        if (kPipe) {
+            const int pn = p0 + n_warps * kFusedChunk;
+            if (pn < len) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int p = pn + i * 4 + pg;
+                    if (p < len_static) {
+                        nk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
+                        nv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
+                    } else { nk[i].zero(); nv[i].zero(); }
+                }
+            }
+        } else if (!loaded) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {          // keys and values of the chunk are requested together
                 const int p = p0 + i * 4 + pg;
@@ -560,6 +575,10 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             for (int j = 0; j < 8; ++j) acc[j] = fmaf(pr, vf[j], acc[j]);
         }
         m = m_new;
+        if (kPipe) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { rk[i] = nk[i]; rv[i] = nv[i]; }
+        }
     }
     // sum the 4 position groups (they share m)
     l += __shfl_xor_sync(0xffffffffu, l, 8);

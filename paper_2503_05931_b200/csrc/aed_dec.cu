@@ -752,6 +752,7 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     const int kb_max = (k_blocks + splits - 1) / splits;
     if (stages > kb_max) stages = kb_max;
     p.stages = stages;
+    p.src_rows = dec->cfg.max_batch;
     p.a_rows = M;
     p.k_blocks = k_blocks;
     p.n_tile = n_tile;

@@ -36,6 +36,7 @@ struct StepGemmParams {
     int k_blocks;              // K / 64
     int n_tile;                // MMA N: rows per CTA tile (16..256, multiple of 16)
     int stages;                // ring depth, 1..kMaxKb
+    int src_rows;              // rows of the source buffer (reads of rows past it are clamped)
     // activation source [rows, ld_src] fp32
     const float *src;
     int ld_src;
@@ -94,7 +95,7 @@ __device__ __forceinline__ void red_add_v4(float *addr, float4 v)
 // Dynamic smem per k-block: weight tile 16 KB | high plane | low plane (n_tile x 128 B each) | fp32 source tile
 // (n_tile x 256 B, filled by TMA, later reused to transpose the accumulator); plus 1024 for alignment.
 template <int MODE>
-__global__ void __launch_bounds__(kSgThreads, 1)
+__global__ void __launch_bounds__(kSgThreads, 2)
 step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_src, StepGemmParams p)
 {
     extern __shared__ uint8_t smem_dyn[];
@@ -117,6 +118,9 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
     const int n_kb = kb_end - kb_begin;
     const int S = p.stages;
+    // Small tiles (at most 32 rows, one or two k-blocks): the producer threads read their 8 source values per k-block
+    // straight from global memory right after the dependency wait instead of waiting for a TMA copy into shared memory.
+    const bool direct = p.n_tile <= 32 && n_kb <= 2;
 
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
     const int plane_bytes = p.n_tile * kBlockK * 2;
@@ -160,8 +164,10 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     tma_load_2d(stage, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[s]);
                 }
                 // fp32 activation source, written by the previous kernels
-                mbar_expect_tx(&bar_s[s], src_bytes);
-                tma_load_2d(stage + kATileBytes + 2 * plane_bytes, &map_src, (kb_begin + i) * kBlockK, row0, &bar_s[s]);
+                if (!direct) {
+                    mbar_expect_tx(&bar_s[s], src_bytes);
+                    tma_load_2d(stage + kATileBytes + 2 * plane_bytes, &map_src, (kb_begin + i) * kBlockK, row0, &bar_s[s]);
+                }
             }
         }
     } else if (warp == 1) {
@@ -252,6 +258,13 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const int a_idx = a0 + quarter * 32 + lane;
         const bool a_ok = a_idx < p.a_rows;
         const float bias = (warp < 6 && p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+        float dv[2][8];
+        if (direct && rbase < p.n_tile) {          // one row per thread (n_tile <= 32), both k-blocks requested at once
+            const int rs = min(row0 + rbase, p.src_rows - 1);
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+                if (i < n_kb) load8(p.src + static_cast<size_t>(rs) * p.ld_src + (kb_begin + i) * kBlockK + c * 8, dv[i]);
+        }
         bool ok = true;
         for (int i = 0; i < n_kb && ok; ++i) {
             const int s = i % S;
@@ -262,13 +275,16 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             float g[8], c1[8], c2[8];
             if (MODE == B_GAMMA) load8(p.gamma + k, g);
             if (MODE == B_LN_RELU) { load8(p.c1 + k, c1); load8(p.c2 + k, c2); }
-            ok = mbar_wait(&bar_s[s], (i / S) & 1, &abort_flag);
+            if (!direct) ok = mbar_wait(&bar_s[s], (i / S) & 1, &abort_flag);
             if (!ok) break;
             for (int rl = rbase; rl < p.n_tile; rl += 32) {
                 const int r = row0 + rl;
                 float y[8];
                 if (r < n_rows) {
-                    load8(src_tile + rl * kBlockK + c * 8, y);
+                    if (direct) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) y[e] = i == 0 ? dv[0][e] : dv[1][e];
+                    } else load8(src_tile + rl * kBlockK + c * 8, y);
                     if (MODE == B_GAMMA) {
 #pragma unroll
                         for (int e = 0; e < 8; ++e) y[e] *= g[e];

@@ -45,7 +45,7 @@ struct LayerWeights {
 // Byte offsets of every region of the caller's workspace.
 struct Layout {
     size_t self_cache, cross_store, x, act, qkv, hid, partials, pe, keys, state;
-    size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, row_info, total;
+    size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, row_info, len_order, total;
     size_t self_layer_elems, cross_layer_elems;
     int max_chunks;
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
@@ -111,6 +111,7 @@ Layout make_layout(const aed_dec_config_t &c)
     L.enc_len = take(B * 4);
     L.max_len = take(B * 4);
     L.row_info = take((size_t)rows_bucket(c.max_batch) * 16);      // grids are sized for the bucket
+    L.len_order = take(B * 4);                                     // utterances by decreasing encoder length
     L.rows_cap = (int)align_up(B, 16);
     if (c.dtype == AED_DTYPE_BF16) {
         L.actd_hi = take((size_t)L.rows_cap * d * 2);
@@ -1043,7 +1044,8 @@ aed_status_t launch_build_active(aed_dec *dec, const uint8_t *mask)
                                                      dec->at<int32_t>(L.t_u), dec->cfg.max_dec_len,
                                                      dec->at<int32_t>(L.active_list), dec->state(),
                                                      dec->at<int32_t>(L.enc_len), dec->at<int32_t>(L.enc_off),
-                                                     dec->at<int4>(L.row_info), rows_bucket(dec->cfg.max_batch));
+                                                     dec->at<int4>(L.row_info), rows_bucket(dec->cfg.max_batch),
+                                                     dec->at<int32_t>(L.len_order));
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -1174,6 +1176,13 @@ extern "C" aed_status_t aed_dec_precompute_cross_kv(aed_dec_t *dec, const void *
     // Pageable host vectors: cudaMemcpyAsync stages them before returning, so the vectors may change afterwards.
     AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.enc_off, dec->enc_off.data(), (batch + 1) * 4, cudaMemcpyHostToDevice, dec->stream));
     AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.enc_len, dec->enc_len.data(), batch * 4, cudaMemcpyHostToDevice, dec->stream));
+    {
+        // visiting order of the row compaction: longest encoder output first (ties by utterance index)
+        std::vector<int32_t> order(batch);
+        for (int u = 0; u < batch; ++u) order[u] = u;
+        std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return enc_lens[a] > enc_lens[b]; });
+        AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.len_order, order.data(), batch * 4, cudaMemcpyHostToDevice, dec->stream));
+    }
     AED_CUDA(dec, cudaMemsetAsync(dec->ws + L.keys, 0, L.enc_off - L.keys, dec->stream));   // keys, state, t_u, retired, lists
     aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed)
                      : dec->cfg.dtype == AED_DTYPE_BF16 ? precompute_impl<__nv_bfloat16>(dec, enc_packed)

@@ -6,7 +6,7 @@
 namespace aed {
 
 // ------------------------------------------------------------------------------------------------------------
-// Row bookkeeping: stable compaction of the utterances that take part in the next step.
+// Row bookkeeping: compaction of the utterances that take part in the next step, in a fixed visiting order.
 //   active_list[r] = utterance id of compact row r;  state->n_active = number of rows.
 // An utterance takes part if it is not retired, the caller's mask (if any) selects it, and its self-attention
 // cache still has room; a selected utterance with a full cache raises the sticky error instead of overflowing.
@@ -17,7 +17,7 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
                                     const int32_t *__restrict__ t_u, int max_dec_len,
                                     int32_t *__restrict__ active_list, DecState *state,
                                     const int32_t *__restrict__ enc_len, const int32_t *__restrict__ enc_off,
-                                    int4 *__restrict__ row_info, int row_slots)
+                                    int4 *__restrict__ row_info, int row_slots, const int32_t *__restrict__ order)
 {
     AED_TRACE_BEGIN(state, 1);
     __shared__ int warp_counts[32];
@@ -26,7 +26,10 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     for (int start = 0; start < batch; start += blockDim.x) {
-        int u = start + threadIdx.x;
+        // utterances are visited in the given order (longest encoder output first), so compact rows come out
+        // sorted by encoder length: the attention blocks of the longest rows are scheduled first
+        const int i = start + threadIdx.x;
+        const int u = i < batch ? order[i] : batch;
         bool take = false;
         if (u < batch) {
             take = retired[u] == 0 && (mask == nullptr || mask[u] != 0);

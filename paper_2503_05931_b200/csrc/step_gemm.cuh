@@ -27,7 +27,7 @@ namespace sg {
 using namespace tc;
 
 constexpr int kMaxKb = 4;             // ring stages per CTA
-constexpr int kSgThreads = 384;       // warp 0 TMA, warp 1 MMA, warps 2..9 activation tiles (2..5 also epilogue), warps 10..11 side jobs
+constexpr int kSgThreads = 384;       // warp 0 TMA, warp 1 MMA, warps 2..9 activation tiles and epilogue, warps 10..11 side jobs
 
 enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2 };
 
@@ -257,7 +257,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const int quarter = warp & 3;
         const int a_idx = a0 + quarter * 32 + lane;
         const bool a_ok = a_idx < p.a_rows;
-        const float bias = (warp < 6 && p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+        const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
         float dv[2][8];
         if (direct && rbase < p.n_tile) {          // one row per thread (n_tile <= 32), both k-blocks requested at once
             const int rs = min(row0 + rbase, p.src_rows - 1);
@@ -308,9 +308,9 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&bar_b[s])) : "memory");
         }
         AED_TRACE_PUT(p.state, tcur, 42);  // activation tiles written
-        if (warp < 6) {                                   // only warps 2..5 own accumulator lanes
-
+        {
         // ---- epilogue: accumulator -> shared memory (transposed) -> 16-byte reductions ---------------------------
+        // Warps w and w + 4 reach the same accumulator lanes (lane quarter = warp & 3): they split the rows in 16s.
         ok = ok && mbar_wait(&bar_done, 0, &abort_flag);
         tc_fence_after_sync();
         AED_TRACE_PUT(p.state, tcur, 44);  // accumulator complete
@@ -318,20 +318,21 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         float *trans = reinterpret_cast<float *>(tiles);
         constexpr int kPitch = kTileM + 4;
         const int rows_here = min(p.n_tile, max(n_rows - row0, 0));
+        const int second = warp >= 6 ? 1 : 0;
         const bool fits = static_cast<size_t>(p.n_tile) * kPitch * 4 <= static_cast<size_t>(n_kb < S ? n_kb : S) * stage_bytes;
         if (ok && fits) {
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            for (int c0 = 0; c0 < rows_here; c0 += 16) {
+            for (int c0 = 16 * second; c0 < rows_here; c0 += 32) {
                 float v[16];
                 tmem_ld16(taddr + c0, v);
 #pragma unroll
                 for (int j = 0; j < 16; ++j) trans[(c0 + j) * kPitch + quarter * 32 + lane] = v[j] + bias;
             }
         }
-        asm volatile("bar.sync 2, 128;" ::: "memory");
+        asm volatile("bar.sync 2, 256;" ::: "memory");
         if (ok && fits) {
             const int o4 = (pt & 31) * 4;
-            for (int rl = pt >> 5; rl < rows_here; rl += 4) {
+            for (int rl = pt >> 5; rl < rows_here; rl += 8) {
                 const float4 v = *reinterpret_cast<const float4 *>(trans + rl * kPitch + o4);
                 float *dst = p.out + static_cast<size_t>(row0 + rl) * p.ldo + a0 + o4;
                 if (a0 + o4 + 3 < p.a_rows) red_add_v4(dst, v);
@@ -344,7 +345,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         } else if (ok) {
             // transposition buffer too small for this shape: scalar reductions straight from the accumulator
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            for (int c0 = 0; c0 < rows_here; c0 += 16) {
+            for (int c0 = 16 * second; c0 < rows_here; c0 += 32) {
                 float v[16];
                 tmem_ld16(taddr + c0, v);
 #pragma unroll

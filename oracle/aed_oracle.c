@@ -186,10 +186,14 @@ static void cross_kv(const orc_config_t *cfg, const orc_weights_t *w, int layer,
  *   enc [T][d_enc]; forced (nullable) [L]: the input token of every step (forced[0] is the start token);
  *   when forced == NULL the run is free-running greedy from `bos`.
  *   logits (nullable) [L][vocab] double; next [L]; margin (nullable) [L].
+ *   eos: end-of-sequence token id, or a negative value to disable it.  When enabled, the step that emits
+ *   eos is the utterance's last: the token is recorded and counted, nothing is computed after it, and
+ *   next[t] = -1 for the remaining steps.  out_len (nullable) receives the number of emitted tokens.
  * Returns 0, or -1 on allocation failure / bad sizes.                                                   */
 int orc_decode(const orc_config_t *cfg, const orc_weights_t *w, const float *enc, int32_t T,
                const int32_t *forced, int32_t bos, int32_t L,
-               double *logits, int32_t *next, double *margin, const orc_trace_t *trace)
+               double *logits, int32_t *next, double *margin, const orc_trace_t *trace,
+               int32_t eos, int32_t *out_len)
 {
     int NL = cfg->n_layers, d = cfg->d_model, H = cfg->n_heads, F = cfg->d_ffn, V = cfg->vocab;
     if (T < 1 || L < 1 || d % H != 0) return -1;
@@ -238,7 +242,14 @@ int orc_decode(const orc_config_t *cfg, const orc_weights_t *w, const float *enc
         if (logits) for (int v = 0; v < V; ++v) logits[(size_t)t * V + v] = (double)z[v];
         tok = orc_argmax(z, V, margin ? margin + t : NULL);
         next[t] = tok;
+        if (eos >= 0 && tok == eos) {          /* emitted and counted; the utterance ends here */
+            for (int r = t + 1; r < L; ++r) { next[r] = -1; if (margin) margin[r] = 0.0; }
+            if (out_len) *out_len = t + 1;
+            free(pool);
+            return 0;
+        }
     }
+    if (out_len) *out_len = L;
     free(pool);
     return 0;
 }
@@ -315,11 +326,12 @@ int orc_decode_full_recompute(const orc_config_t *cfg, const orc_weights_t *w, c
  *   enc_packed [sum T][d_enc] with enc_offsets [B+1] (in frames); lens [B];
  *   forced (nullable) [B][stride]; next [B][stride]; margin (nullable) [B][stride];
  *   logits (nullable): utterance u's [lens[u]][vocab] block starts at logit_offsets[u] rows.
+ *   eos (negative = disabled) and out_lens (nullable) [B]: as in orc_decode.
  * Returns the number of threads used, or a negative value if any utterance failed.                     */
 int orc_decode_batch(const orc_config_t *cfg, const orc_weights_t *w, const float *enc_packed,
                      const int64_t *enc_offsets, int32_t B, const int32_t *forced, int32_t stride, int32_t bos,
                      const int32_t *lens, double *logits, const int64_t *logit_offsets,
-                     int32_t *next, double *margin, int32_t n_threads)
+                     int32_t *next, double *margin, int32_t n_threads, int32_t eos, int32_t *out_lens)
 {
     int failed = 0, used = 1;
 #ifdef _OPENMP
@@ -334,7 +346,8 @@ int orc_decode_batch(const orc_config_t *cfg, const orc_weights_t *w, const floa
                                 (int32_t)(enc_offsets[u + 1] - enc_offsets[u]),
                                 forced ? forced + (size_t)u * stride : NULL, bos, lens[u],
                                 logits ? logits + (size_t)logit_offsets[u] * cfg->vocab : NULL,
-                                next + (size_t)u * stride, margin ? margin + (size_t)u * stride : NULL, NULL);
+                                next + (size_t)u * stride, margin ? margin + (size_t)u * stride : NULL, NULL,
+                                eos, out_lens ? out_lens + u : NULL);
             if (rc != 0) {
 #pragma omp atomic write
                 failed = 1;
@@ -348,7 +361,8 @@ int orc_decode_batch(const orc_config_t *cfg, const orc_weights_t *w, const floa
                             (int32_t)(enc_offsets[u + 1] - enc_offsets[u]),
                             forced ? forced + (size_t)u * stride : NULL, bos, lens[u],
                             logits ? logits + (size_t)logit_offsets[u] * cfg->vocab : NULL,
-                            next + (size_t)u * stride, margin ? margin + (size_t)u * stride : NULL, NULL);
+                            next + (size_t)u * stride, margin ? margin + (size_t)u * stride : NULL, NULL,
+                                eos, out_lens ? out_lens + u : NULL);
         if (rc != 0) failed = 1;
     }
 #endif

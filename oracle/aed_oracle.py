@@ -123,9 +123,11 @@ class Model:
 
 
 def decode(model: Model, enc: np.ndarray, n_steps: int, *, forced: Optional[Sequence[int]] = None, bos: int = 1,
-           want_logits: bool = True, precision: str = "f64", full_recompute: bool = False, trace: bool = False):
-    """Decode one utterance.  Returns dict(next [L] int32, margin [L], logits [L, V] or None,
-    and with trace=True self_probs [L, NL, H, L] and cross_probs [L, NL, H, T])."""
+           want_logits: bool = True, precision: str = "f64", full_recompute: bool = False, trace: bool = False,
+           eos: int = -1):
+    """Decode one utterance.  Returns dict(next [L] int32, margin [L], logits [L, V] or None, len,
+    and with trace=True self_probs [L, NL, H, L] and cross_probs [L, NL, H, T]).  With ``eos`` >= 0 the
+    utterance ends with the step that emits it: ``len`` counts that token and ``next`` is -1 afterwards."""
     lib = _lib(precision)
     enc = _f32(enc)
     T, L, V = int(enc.shape[0]), int(n_steps), model.model["vocab"]
@@ -143,7 +145,9 @@ def decode(model: Model, enc: np.ndarray, n_steps: int, *, forced: Optional[Sequ
               C.c_int32(L), lp, nxt.ctypes.data_as(C.POINTER(C.c_int32)), margin.ctypes.data_as(C.POINTER(C.c_double))]
     out = dict(next=nxt, margin=margin, logits=logits)
     if full_recompute:
+        assert eos < 0, "the brute-force decoder has no end-of-sequence rule"
         rc = lib.orc_decode_full_recompute(*common)
+        out["len"] = L
     else:
         tr = None
         if trace:
@@ -152,7 +156,9 @@ def decode(model: Model, enc: np.ndarray, n_steps: int, *, forced: Optional[Sequ
             out["cross_probs"] = np.zeros((L, nl, h, T), np.float64)
             tr = _Trace(out["self_probs"].ctypes.data_as(C.POINTER(C.c_double)),
                         out["cross_probs"].ctypes.data_as(C.POINTER(C.c_double)))
-        rc = lib.orc_decode(*common, C.byref(tr) if tr is not None else None)
+        n_out = C.c_int32(0)
+        rc = lib.orc_decode(*common, C.byref(tr) if tr is not None else None, C.c_int32(eos), C.byref(n_out))
+        out["len"] = int(n_out.value)
     if rc != 0:
         raise RuntimeError(f"oracle decode failed (rc={rc})")
     return out
@@ -160,9 +166,9 @@ def decode(model: Model, enc: np.ndarray, n_steps: int, *, forced: Optional[Sequ
 
 def decode_batch(model: Model, enc_packed: np.ndarray, enc_lens: Sequence[int], dec_lens: Sequence[int], *,
                  forced: Optional[np.ndarray] = None, bos: int = 1, want_logits: bool = False,
-                 precision: str = "f64", n_threads: int = 0):
+                 precision: str = "f64", n_threads: int = 0, eos: int = -1):
     """Decode utterances independently (OpenMP over utterances).  Returns dict(next [B, Lmax] int32 (-1 padded),
-    margin [B, Lmax], logits: list of [L_u, V] arrays or None, threads)."""
+    margin [B, Lmax], logits: list of [L_u, V] arrays or None, lens [B] emitted tokens, threads)."""
     lib = _lib(precision)
     enc_packed = _f32(enc_packed)
     enc_lens = np.asarray(enc_lens, dtype=np.int64)
@@ -177,6 +183,7 @@ def decode_batch(model: Model, enc_packed: np.ndarray, enc_lens: Sequence[int], 
     loff = np.zeros(B + 1, np.int64)
     np.cumsum(lens, out=loff[1:])
     logits = np.zeros((int(loff[-1]), V), np.float64) if want_logits else None
+    out_lens = np.zeros(B, np.int32)
     f_arr = None
     if forced is not None:
         f_arr = np.ascontiguousarray(forced, dtype=np.int32)
@@ -188,11 +195,12 @@ def decode_batch(model: Model, enc_packed: np.ndarray, enc_lens: Sequence[int], 
         lens.ctypes.data_as(C.POINTER(C.c_int32)),
         logits.ctypes.data_as(C.POINTER(C.c_double)) if logits is not None else None,
         loff.ctypes.data_as(C.POINTER(C.c_int64)),
-        nxt.ctypes.data_as(C.POINTER(C.c_int32)), margin.ctypes.data_as(C.POINTER(C.c_double)), C.c_int32(n_threads))
+        nxt.ctypes.data_as(C.POINTER(C.c_int32)), margin.ctypes.data_as(C.POINTER(C.c_double)), C.c_int32(n_threads),
+        C.c_int32(eos), out_lens.ctypes.data_as(C.POINTER(C.c_int32)))
     if rc < 0:
         raise RuntimeError("oracle batch decode failed")
     per_utt = [logits[loff[u]:loff[u + 1]] for u in range(B)] if logits is not None else None
-    return dict(next=nxt, margin=margin, logits=per_utt, threads=int(rc))
+    return dict(next=nxt, margin=margin, logits=per_utt, lens=out_lens, threads=int(rc))
 
 
 def layernorm(x, g, b, eps: float = 1e-5, precision: str = "f64") -> np.ndarray:

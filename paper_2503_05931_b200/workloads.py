@@ -163,16 +163,24 @@ def draw_lengths(rng: np.random.Generator, batch: int, law: str):
     return durations, enc_lens, dec_lens
 
 
-def draw_weights(rng: np.random.Generator, model: Dict[str, int], dtype: str, bias_std: float = 0.02):
-    """All decoder tensors as float32 (bf16-representable when dtype == 'bf16')."""
+def draw_weights(rng: np.random.Generator, model: Dict[str, int], dtype: str, bias_std: float = 0.02,
+                 ln_std: float = 0.0, out_bias_std: float = 0.0, embed_offset: float = 0.0):
+    """All decoder tensors as float32 (bf16-representable when dtype == 'bf16').
+
+    The named workloads keep LayerNorm gamma = 1, beta = 0 and no output bias (``ln_std = out_bias_std = 0``).
+    Property tests ask for more: ``ln_std`` > 0 draws gamma ~ N(1, ln_std) and beta ~ N(0, ln_std),
+    ``out_bias_std`` > 0 draws an output-projection bias, and ``embed_offset`` shifts every entry of the
+    embedding table by a constant so that the residual stream has a mean far from zero."""
     def one(shape, kind):
-        if kind == "g":
-            return np.ones(shape, np.float32)
-        if kind == "b":
-            return np.zeros(shape, np.float32)
+        if kind in ("g", "b") and ln_std <= 0.0:
+            return np.ones(shape, np.float32) if kind == "g" else np.zeros(shape, np.float32)
         std = 0.02 if len(shape) == 2 else bias_std
+        if kind in ("g", "b"):
+            std = ln_std
         a = rng.standard_normal(size=shape, dtype=np.float32)
         a *= np.float32(std)
+        if kind == "g":
+            a += np.float32(1.0)
         return round_to_bf16(a) if dtype == "bf16" else a
 
     w: Dict[str, object] = {}
@@ -181,6 +189,12 @@ def draw_weights(rng: np.random.Generator, model: Dict[str, int], dtype: str, bi
     for name, shape_fn, kind in _LAYER_TENSORS:
         w[name] = [one(shape_fn(model), kind) for _ in range(model["n_layers"])]
     w["b_out"] = None
+    if out_bias_std > 0.0:
+        b = rng.standard_normal(size=(model["vocab"],), dtype=np.float32) * np.float32(out_bias_std)
+        w["b_out"] = round_to_bf16(b) if dtype == "bf16" else b
+    if embed_offset != 0.0:
+        e = w["embed"] + np.float32(embed_offset)
+        w["embed"] = round_to_bf16(e) if dtype == "bf16" else e
     return w
 
 
@@ -210,12 +224,14 @@ def make_workload(name: str, *, seed: Optional[int] = None, batch: Optional[int]
 
 
 def make_custom(model: Dict[str, int], enc_lens, dec_lens, *, dtype: str = "fp32", seed: int = 0,
-                bias_std: float = 0.02, name: str = "custom") -> Workload:
-    """A workload with explicit lengths (edge cases, property tests)."""
+                bias_std: float = 0.02, name: str = "custom", ln_std: float = 0.0, out_bias_std: float = 0.0,
+                embed_offset: float = 0.0) -> Workload:
+    """A workload with explicit lengths (edge cases, property tests); see ``draw_weights`` for the options."""
     rng = np.random.default_rng(seed)
     enc_lens = np.asarray(enc_lens, dtype=np.int32)
     dec_lens = np.asarray(dec_lens, dtype=np.int32)
-    weights = draw_weights(rng, model, dtype, bias_std=bias_std)
+    weights = draw_weights(rng, model, dtype, bias_std=bias_std, ln_std=ln_std, out_bias_std=out_bias_std,
+                           embed_offset=embed_offset)
     enc = draw_encoder_states(rng, int(enc_lens.sum()), model["d_enc"], dtype)
     return Workload(name=name, model=dict(model), dtype=dtype, seed=seed, enc_lens=enc_lens, dec_lens=dec_lens,
                     durations=enc_lens.astype(np.float64) * FRAME_SECONDS, weights=weights, enc=enc)

@@ -351,3 +351,52 @@ def test_argmax_lowest_index_on_ties():
     out = orc.decode(m, utt_enc(w, 0), 6)
     assert np.all(out["logits"][:, 31] == out["logits"][:, 12])
     assert not np.any(out["next"] == 31)
+
+
+# ----------------------------------------------------------------------------------------------
+# End-of-sequence rule: the token is emitted and counted, then the utterance stops.  Pinned against the
+# run without the rule, which the pins above fix independently.
+# ----------------------------------------------------------------------------------------------
+def test_eos_run_is_the_free_run_cut_after_the_first_eos():
+    w = small_workload(seed=12, enc_lens=(6, 4, 9, 5), dec_lens=(12, 12, 12, 12))
+    m = orc.Model(w.model, w.weights)
+    stopped_early = 0
+    for u in range(w.batch):
+        L = int(w.dec_lens[u])
+        free = orc.decode(m, utt_enc(w, u), L)
+        assert free["len"] == L and np.all(free["next"] >= 0)
+        # every token the free run emits, as the end-of-sequence id: first step, a middle step, the last step
+        for eos in sorted(set(int(t) for t in free["next"])):
+            first = int(np.flatnonzero(free["next"] == eos)[0])
+            cut = orc.decode(m, utt_enc(w, u), L, eos=eos)
+            assert cut["len"] == first + 1
+            assert np.array_equal(cut["next"][:first + 1], free["next"][:first + 1])
+            assert np.all(cut["next"][first + 1:] == -1)
+            assert np.array_equal(cut["logits"][:first + 1], free["logits"][:first + 1])
+            assert np.all(cut["logits"][first + 1:] == 0.0)          # nothing is computed after the stop
+            stopped_early += first + 1 < L
+        assert orc.decode(m, utt_enc(w, u), L, eos=int(free["next"][0]))["len"] == 1          # planted at step 0
+        last_only = [int(t) for i, t in enumerate(free["next"]) if i == L - 1 and t not in free["next"][:L - 1]]
+        for eos in last_only:                                                                   # only at the last step
+            assert orc.decode(m, utt_enc(w, u), L, eos=eos)["len"] == L
+        absent = next(v for v in range(w.model["vocab"]) if v not in free["next"])
+        same = orc.decode(m, utt_enc(w, u), L, eos=absent)
+        assert same["len"] == L and np.array_equal(same["next"], free["next"])
+    assert stopped_early > 0
+
+
+def test_eos_in_a_batch_stops_each_utterance_on_its_own():
+    w = small_workload(seed=12, enc_lens=(6, 4, 9, 5), dec_lens=(12, 7, 12, 3))
+    m = orc.Model(w.model, w.weights)
+    free = orc.decode_batch(m, w.enc, w.enc_lens, w.dec_lens)
+    assert np.array_equal(free["lens"], w.dec_lens)
+    eos = int(free["next"][0, 4])
+    cut = orc.decode_batch(m, w.enc, w.enc_lens, w.dec_lens, eos=eos)
+    for u in range(w.batch):
+        L = int(w.dec_lens[u])
+        hits = np.flatnonzero(free["next"][u, :L] == eos)
+        expect = int(hits[0]) + 1 if len(hits) else L
+        assert cut["lens"][u] == expect
+        assert np.array_equal(cut["next"][u, :expect], free["next"][u, :expect])
+        assert np.all(cut["next"][u, expect:] == -1)
+    assert cut["lens"][0] <= 5

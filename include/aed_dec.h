@@ -152,10 +152,12 @@ aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, const uint8_
  * library image instead of the workspace region; everything else is as in aed_dec_step, with the same
  * arguments, results and errors.  It calls no cudaMalloc / cudaFree and no allocating library routine.
  *
+ *   - Only the fp32 configuration splits attention into chunks and therefore uses the scratch; the bf16 step
+ *     merges its chunks inside one thread block, writes no partials, and runs unchanged through this call.
  *   - The array holds aed_dec_static_scratch_bytes() = 8 MiB, and every GPU whose context loads the library
- *     keeps that much memory until the process exits.  A batch that needs more
+ *     keeps that much memory until the process exits.  An fp32 batch that needs more
  *     (batch x n_heads x ceil(max(max_enc_len, max_dec_len) / 64) x 264 bytes) is refused with
- *     AED_ERR_CAPACITY and nothing is launched.
+ *     AED_ERR_CAPACITY and nothing is launched; bf16 batches are never refused on this ground.
  *   - The first call on each device looks up the array's device address (the device of the handle's stream
  *     must be current, as for every call); make that first call outside any stream capture.
  *   - All handles and all calls on one device share the one array, and it keeps whatever the previous call
@@ -181,6 +183,13 @@ aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max_len, int32
 
 /* Synchronise the stream and report any sticky device-side error (AED_OK if none). */
 aed_status_t aed_dec_sync_status(aed_dec_t *dec);
+
+/*
+ * The status that a value of the device-side error word stands for (host-only helper, no device access; the
+ * paper has no counterpart): 0 -> AED_OK, 1 (a step was asked of an utterance whose self-attention cache is
+ * full) -> AED_ERR_CAPACITY, anything else (a kernel gave up a bounded wait) -> AED_ERR_TIMEOUT.
+ */
+aed_status_t aed_dec_status_of_error_word(int32_t error_word);
 
 /*
  * Measurement aid (the paper has no counterpart): with profiling enabled the library records a CUDA event on

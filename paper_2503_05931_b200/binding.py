@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = [
     "aed_dec_workspace_bytes", "aed_dec_create", "aed_dec_precompute_cross_kv", "aed_dec_step",
     "aed_dec_greedy_decode", "aed_dec_sync_status", "aed_dec_launch_count", "aed_dec_destroy",
     "aed_dec_last_error", "aed_dec_create_error", "aed_dec_profile_enable", "aed_dec_profile_read",
-    "aed_dec_step_static_scratch", "aed_dec_static_scratch_bytes",
+    "aed_dec_step_static_scratch", "aed_dec_static_scratch_bytes", "aed_dec_status_of_error_word",
 ]
 
 _GLOBAL_FIELDS = ["embed", "final_ln_g", "final_ln_b", "w_out", "b_out"]
@@ -78,6 +78,8 @@ def load_library() -> C.CDLL:
     lib.aed_dec_greedy_decode.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_void_p, C.c_void_p]
     lib.aed_dec_sync_status.restype = C.c_int
     lib.aed_dec_sync_status.argtypes = [C.c_void_p]
+    lib.aed_dec_status_of_error_word.restype = C.c_int
+    lib.aed_dec_status_of_error_word.argtypes = [C.c_int32]
     lib.aed_dec_launch_count.restype = C.c_int64
     lib.aed_dec_launch_count.argtypes = [C.c_void_p]
     lib.aed_dec_destroy.restype = None

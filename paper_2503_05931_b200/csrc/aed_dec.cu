@@ -1040,7 +1040,7 @@ aed_status_t launch_build_active(aed_dec *dec, const uint8_t *mask)
 {
     const Layout &L = dec->lay;
     ProfScope ps(dec, KF_BOOKKEEPING);
-    build_active_kernel<<<1, 1024, 0, dec->stream>>>(dec->batch, mask, dec->at<int32_t>(L.retired),
+    build_active_kernel<<<1, 1024, 0, dec->stream>>>(mask, dec->at<int32_t>(L.retired),
                                                      dec->at<int32_t>(L.t_u), dec->cfg.max_dec_len,
                                                      dec->at<int32_t>(L.active_list), dec->state(),
                                                      dec->at<int32_t>(L.enc_len), dec->at<int32_t>(L.enc_off),
@@ -1184,6 +1184,7 @@ extern "C" aed_status_t aed_dec_precompute_cross_kv(aed_dec_t *dec, const void *
         AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.len_order, order.data(), batch * 4, cudaMemcpyHostToDevice, dec->stream));
     }
     AED_CUDA(dec, cudaMemsetAsync(dec->ws + L.keys, 0, L.enc_off - L.keys, dec->stream));   // keys, state, t_u, retired, lists
+    AED_CUDA(dec, cudaMemcpyAsync(&dec->state()->batch, &dec->batch, sizeof(int32_t), cudaMemcpyHostToDevice, dec->stream));
     aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed)
                      : dec->cfg.dtype == AED_DTYPE_BF16 ? precompute_impl<__nv_bfloat16>(dec, enc_packed)
                                                         : precompute_impl<float>(dec, enc_packed);
@@ -1259,7 +1260,9 @@ extern "C" aed_status_t aed_dec_step_static_scratch(aed_dec_t *dec, const int32_
     if (!dec) return AED_ERR_INVALID_ARG;
     if (!dec->have_batch)
         return fail(dec, AED_ERR_STATE, "aed_dec_step_static_scratch needs a batch: call aed_dec_precompute_cross_kv first");
-    const size_t need = (size_t)dec->batch * dec->cfg.n_heads * dec->lay.max_chunks * kPartialStride * sizeof(float);
+    // Only the fp32 path splits attention over chunks and writes partials; the bf16 step merges inside one block
+    // and touches no scratch, so no batch is refused there.
+    const size_t need = dec->use_tc ? 0 : (size_t)dec->batch * dec->cfg.n_heads * dec->lay.max_chunks * kPartialStride * sizeof(float);
     if (need > kStaticScratchBytes)
         return fail(dec, AED_ERR_CAPACITY,
                     "batch %d x %d heads x %d chunks needs %zu bytes of attention scratch; the built-in array holds %zu",
@@ -1367,9 +1370,19 @@ extern "C" aed_status_t aed_dec_sync_status(aed_dec_t *dec)
     DecState host{};
     AED_CUDA(dec, cudaMemcpyAsync(&host, dec->state(), sizeof host, cudaMemcpyDeviceToHost, dec->stream));
     AED_CUDA(dec, cudaStreamSynchronize(dec->stream));
-    if (host.error == 1) return fail(dec, AED_ERR_CAPACITY, "a step was asked of an utterance whose self-attention cache is full");
-    if (host.error != 0) return fail(dec, AED_ERR_TIMEOUT, "device-side error %d", host.error);
+    const aed_status_t s = aed_dec_status_of_error_word(host.error);
+    if (s == AED_ERR_CAPACITY) return fail(dec, s, "a step was asked of an utterance whose self-attention cache is full");
+    if (s != AED_OK) return fail(dec, s, "a bounded wait on the device ran out (device-side error %d)", host.error);
     return AED_OK;
+}
+
+// The sticky error word of the device-side decode state as a status: 0 = fine, 1 = a self-attention cache was full,
+// anything else = a kernel gave up waiting.
+extern "C" aed_status_t aed_dec_status_of_error_word(int32_t error_word)
+{
+    if (error_word == 0) return AED_OK;
+    if (error_word == 1) return AED_ERR_CAPACITY;
+    return AED_ERR_TIMEOUT;
 }
 
 extern "C" aed_status_t aed_dec_profile_enable(aed_dec_t *dec, int32_t enable)

@@ -16,6 +16,7 @@ struct DecState {
     int32_t error;       // sticky: 0 ok, 1 = a row would have overflowed the self-attention cache
     int32_t n_retired;   // utterances retired so far
     int32_t grid_sync;   // arrival counter of the persistent step kernel, cleared by the first kernel of a step
+    int32_t batch;       // utterances of the current batch (written by the cross-K/V precompute)
 };
 
 // Optional device-side timeline (debug builds with -DAED_TRACE): block 0 of every traced kernel stamps its start

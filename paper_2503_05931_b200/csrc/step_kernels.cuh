@@ -13,7 +13,9 @@ namespace aed {
 // ------------------------------------------------------------------------------------------------------------
 // It also fills the row table: row_info[r] = (utterance, t_u, encoder length, encoder offset) for every compact
 // row, and utterance -1 for the slots past the last row, so that a kernel needs one 16-byte load per row.
-__global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask, const int32_t *__restrict__ retired,
+// The batch size is read from the decode state, not passed by value: a captured step graph outlives the batch it
+// was recorded for and is replayed for later batches of other sizes.
+__global__ void build_active_kernel(const uint8_t *__restrict__ mask, const int32_t *__restrict__ retired,
                                     const int32_t *__restrict__ t_u, int max_dec_len,
                                     int32_t *__restrict__ active_list, DecState *state,
                                     const int32_t *__restrict__ enc_len, const int32_t *__restrict__ enc_off,
@@ -22,6 +24,7 @@ __global__ void build_active_kernel(int batch, const uint8_t *__restrict__ mask,
     AED_TRACE_BEGIN(state, 1);
     __shared__ int warp_counts[32];
     __shared__ int base;
+    const int batch = state->batch;
     if (threadIdx.x == 0) base = 0;
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;

@@ -19,6 +19,7 @@
 #pragma once
 #include <cuda.h>
 
+#include "bounded_wait.h"
 #include "common.cuh"
 
 namespace aed {
@@ -55,13 +56,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // Bounded wait.  Returns false if the phase did not complete in time or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long start = clock64();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - start > kWaitCycles) { *abort_flag = 1; return false; }
-    }
+    return bounded_poll([&] { return mbar_try_wait(bar, parity); }, [] { return clock64(); }, kWaitCycles, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c_inner, int c_outer, uint64_t *bar)

@@ -164,13 +164,15 @@ def draw_lengths(rng: np.random.Generator, batch: int, law: str):
 
 
 def draw_weights(rng: np.random.Generator, model: Dict[str, int], dtype: str, bias_std: float = 0.02,
-                 ln_std: float = 0.0, out_bias_std: float = 0.0, embed_offset: float = 0.0):
+                 ln_std: float = 0.0, out_bias_std: float = 0.0, embed_offset: float = 0.0, out_std: float = 0.02):
     """All decoder tensors as float32 (bf16-representable when dtype == 'bf16').
 
     The named workloads keep LayerNorm gamma = 1, beta = 0 and no output bias (``ln_std = out_bias_std = 0``).
     Property tests ask for more: ``ln_std`` > 0 draws gamma ~ N(1, ln_std) and beta ~ N(0, ln_std),
     ``out_bias_std`` > 0 draws an output-projection bias, and ``embed_offset`` shifts every entry of the
-    embedding table by a constant so that the residual stream has a mean far from zero."""
+    embedding table by a constant so that the residual stream has a mean far from zero.  ``out_std`` is the
+    spread of the output projection: a larger one widens the gaps between logits, so that more greedy choices
+    are clear of near-ties."""
     def one(shape, kind):
         if kind in ("g", "b") and ln_std <= 0.0:
             return np.ones(shape, np.float32) if kind == "g" else np.zeros(shape, np.float32)
@@ -186,6 +188,9 @@ def draw_weights(rng: np.random.Generator, model: Dict[str, int], dtype: str, bi
     w: Dict[str, object] = {}
     for name, shape_fn, kind in _GLOBAL_TENSORS:
         w[name] = one(shape_fn(model), kind)
+        if name == "w_out" and out_std != 0.02:
+            a = w[name] * np.float32(out_std / 0.02)
+            w[name] = round_to_bf16(a) if dtype == "bf16" else a
     for name, shape_fn, kind in _LAYER_TENSORS:
         w[name] = [one(shape_fn(model), kind) for _ in range(model["n_layers"])]
     w["b_out"] = None
@@ -225,13 +230,13 @@ def make_workload(name: str, *, seed: Optional[int] = None, batch: Optional[int]
 
 def make_custom(model: Dict[str, int], enc_lens, dec_lens, *, dtype: str = "fp32", seed: int = 0,
                 bias_std: float = 0.02, name: str = "custom", ln_std: float = 0.0, out_bias_std: float = 0.0,
-                embed_offset: float = 0.0) -> Workload:
+                embed_offset: float = 0.0, out_std: float = 0.02) -> Workload:
     """A workload with explicit lengths (edge cases, property tests); see ``draw_weights`` for the options."""
     rng = np.random.default_rng(seed)
     enc_lens = np.asarray(enc_lens, dtype=np.int32)
     dec_lens = np.asarray(dec_lens, dtype=np.int32)
     weights = draw_weights(rng, model, dtype, bias_std=bias_std, ln_std=ln_std, out_bias_std=out_bias_std,
-                           embed_offset=embed_offset)
+                           embed_offset=embed_offset, out_std=out_std)
     enc = draw_encoder_states(rng, int(enc_lens.sum()), model["d_enc"], dtype)
     return Workload(name=name, model=dict(model), dtype=dtype, seed=seed, enc_lens=enc_lens, dec_lens=dec_lens,
                     durations=enc_lens.astype(np.float64) * FRAME_SECONDS, weights=weights, enc=enc)

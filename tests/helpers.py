@@ -7,12 +7,24 @@ TOL = {"fp32": 1e-4, "bf16": 3e-2}       # max-abs tolerance on teacher-forced l
 MARGIN = 0.1                             # greedy ids must match where the checker's top-2 margin exceeds this
 
 
-def oracle_reference(w, rows=None, want_logits=True, n_threads=0):
+def oracle_reference(w, rows=None, want_logits=True, n_threads=0, eos=-1):
     """Free-running greedy decode of the given utterances (default: all) by the CPU checker."""
     sub = w if rows is None else w.subset(rows)
     model = orc.Model(w.model, w.weights, ln_eps=w.ln_eps)
     return orc.decode_batch(model, sub.enc, sub.enc_lens, sub.dec_lens, bos=w.bos_id, want_logits=want_logits,
-                            n_threads=n_threads)
+                            n_threads=n_threads, eos=eos)
+
+
+def comparable_tokens(w, ref, rows=None):
+    """How many greedy tokens the checker fixes: per utterance, the steps before its first near-tie."""
+    rows = list(range(w.batch)) if rows is None else [int(r) for r in rows]
+    n = 0
+    for i, u in enumerate(rows):
+        for t in range(int(w.dec_lens[u])):
+            if ref["margin"][i, t] <= MARGIN:
+                break
+            n += 1
+    return n
 
 
 def teacher_forced_compare(dec, w, ref, rows=None, check_rows_only=True):
@@ -73,4 +85,5 @@ def greedy_compare(dec, w, ref, rows=None):
                 break
             assert toks[u, t] == ref["next"][i, t], f"utterance {u} step {t}: {toks[u, t]} vs {ref['next'][i, t]}"
             compared += 1
+    assert compared == comparable_tokens(w, ref, rows)
     return compared, toks

@@ -21,16 +21,23 @@ def _binding():
     return binding
 
 
-def _run_both(w, rows=None):
+def _run_both(w, rows=None, need_tokens=True, label=""):
+    """Teacher-forced logits and argmax at every step (this comparison carries the weight: it never stops at a
+    near-tie), then the free-running greedy decode up to each utterance's first near-tie.  ``need_tokens``: demand
+    that the greedy comparison covered at least one token."""
     b = _binding()
     ref = oracle_reference(w, rows)
     dec = b.decoder_for_workload(w)
     try:
         worst, compared, bad = teacher_forced_compare(dec, w, ref, rows)
         assert compared > 0
+        print(f"[parity] {label or w.name} {w.dtype} B={w.batch}: max |logit diff| = {worst:.3e} over {compared} rows x steps")
         assert worst < TOL[w.dtype], f"max |logit diff| {worst:.3e} above {TOL[w.dtype]}"
         assert not bad, f"argmax mismatches at margin > {MARGIN}: {bad[:5]}"
-        greedy_compare(dec, w, ref, rows)
+        n_tok, _ = greedy_compare(dec, w, ref, rows)
+        print(f"[parity] {label or w.name} {w.dtype}: {n_tok} greedy tokens compared")
+        if need_tokens:
+            assert n_tok > 0, "the greedy comparison covered no token"
     finally:
         dec.close()
     return worst
@@ -48,7 +55,7 @@ def test_ragged_multi_tile(dtype):
     """Lengths that span several attention chunks and GEMM row tiles with ragged tails, d_enc != d_model."""
     enc_lens = [1, 63, 64, 65, 130, 257, 5, 200] + [17] * 62      # 70 rows: more than one 64-row tile
     dec_lens = [1, 2, 70, 66, 5, 33, 64, 65] + [3] * 62
-    w = wl.make_custom(MID, enc_lens, dec_lens, dtype=dtype, seed=21)
+    w = wl.make_custom(MID, enc_lens, dec_lens, dtype=dtype, seed=21, out_std=0.3)
     _run_both(w, rows=[0, 1, 2, 3, 4, 5, 6, 7, 8, 69])
 
 
@@ -57,7 +64,7 @@ def test_ragged_multi_tile(dtype):
 def test_degenerate_shapes(dtype, shape):
     enc_lens, dec_lens = shape
     w = wl.make_custom(SMALL, list(enc_lens), list(dec_lens), dtype=dtype, seed=5)
-    _run_both(w)
+    _run_both(w, need_tokens=False)         # one or two tokens in all: the first may already be a near-tie
 
 
 def test_random_shapes_fp32():
@@ -66,7 +73,7 @@ def test_random_shapes_fp32():
         B = int(rng.integers(1, 10))
         w = wl.make_custom(SMALL, rng.integers(1, 71, size=B), rng.integers(1, 41, size=B), dtype="fp32",
                            seed=100 + case)
-        _run_both(w)
+        _run_both(w, need_tokens=False, label=f"random{case}")
 
 
 def test_batch_composition_invariance_on_gpu():
@@ -93,38 +100,106 @@ def test_batch_composition_invariance_on_gpu():
     np.testing.assert_allclose(outs[0], outs[2], atol=2e-6)
 
 
+def _eos_case(dtype):
+    """A seeded workload and an end-of-sequence id, found by the checker alone, such that some utterance stops
+    early and every token up to each utterance's stop is fixed by the checker (top-2 margin > MARGIN)."""
+    for seed in range(13, 60):
+        w = wl.make_custom(SMALL, [12, 20, 7, 33, 5], [10, 10, 1, 10, 2], dtype=dtype, seed=seed, out_std=0.3)
+        free = oracle_reference(w, want_logits=False)
+        for u, t in ((1, 3), (0, 2), (3, 5), (2, 1), (4, 6)):
+            eos = int(free["next"][u, t])
+            cut = oracle_reference(w, want_logits=False, eos=eos)
+            fixed = all(np.min(cut["margin"][v, :cut["lens"][v]]) > MARGIN for v in range(w.batch))
+            early = cut["lens"] < w.dec_lens
+            if fixed and np.any(early) and np.any(~early) and np.min(cut["lens"][early]) >= 3:
+                return w, eos, cut
+    raise AssertionError("no seeded case found")
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_eos_stops_an_utterance(dtype):
-    """With eos enabled an utterance retires right after emitting it; the others run on.  The expectation is
-    built from a run without eos of the same decoder: same tokens up to and including the first eos, then -1.
-    (Near-ties could flip a bf16 token between two runs; utterances whose checker margin is below 0.01
-    somewhere in the compared prefix are left out.)"""
+    """With eos enabled an utterance retires right after emitting it (the token is stored and counted) while the
+    others run on.  Expectation: the CPU checker's decode with the same end-of-sequence id."""
     b = _binding()
-    w = wl.make_custom(SMALL, [12, 20, 7, 33, 5], [10, 10, 10, 10, 10], dtype=dtype, seed=13)
-    ref = oracle_reference(w)
-    dec = b.decoder_for_workload(w)
-    enc = dec.upload_encoder(w.enc)
-    dec.precompute_cross_kv(enc, w.enc_lens)
-    free, _ = dec.greedy_decode(w.dec_lens)
-    free = free.cpu().numpy()
-    dec.close()
-    eos = int(free[1, 3])
+    w, eos, cut = _eos_case(dtype)
     dec = b.decoder_for_workload(w, eos_id=eos)
-    dec.precompute_cross_kv(enc, w.enc_lens)
+    dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
     toks, lens = dec.greedy_decode(w.dec_lens)
     toks, lens = toks.cpu().numpy(), lens.cpu().numpy()
     dec.close()
     stopped_early = 0
     for u in range(w.batch):
-        hits = [t for t in range(10) if free[u, t] == eos]
-        expect = hits[0] + 1 if hits else 10
-        if np.min(ref["margin"][u, :expect]) < 0.01:
-            continue
-        assert lens[u] == expect, (u, lens[u], expect)
-        assert np.array_equal(toks[u, :expect], free[u, :expect])
-        assert np.all(toks[u, expect:] == -1)
-        stopped_early += expect < 10
-    assert lens[1] <= 4
+        n = int(cut["lens"][u])
+        assert lens[u] == n, (u, lens[u], n)
+        assert np.array_equal(toks[u, :n], cut["next"][u, :n])
+        assert np.all(toks[u, n:] == -1)
+        if n < w.dec_lens[u]:
+            assert toks[u, n - 1] == eos
+            stopped_early += 1
+    assert stopped_early > 0
+
+
+def test_handle_reuse_across_batch_sizes():
+    """One handle and one pair of output buffers decode batches of 12, 7 and 12 utterances in turn (the step graphs
+    recorded for the first batch are replayed for the others): every batch against the checker."""
+    import torch
+    b = _binding()
+    rng = np.random.default_rng(3)
+    works = [wl.make_custom(MID, rng.integers(1, 90, size=n), rng.integers(2, 12, size=n), dtype="bf16", seed=71,
+                            out_std=0.3) for n in (12, 7, 12)]
+    dec = b.Decoder(MID, works[0].weights, "bf16", max_batch=12,
+                    max_total_enc_frames=max(int(w.enc_lens.sum()) for w in works),
+                    max_enc_len=max(int(w.enc_lens.max()) for w in works), max_dec_len=12)
+    toks = torch.empty((12, 12), dtype=torch.int32, device="cuda:0")
+    lens = torch.empty(12, dtype=torch.int32, device="cuda:0")
+    total = 0
+    try:
+        for w in works:
+            assert all(np.array_equal(a, c) for a, c in zip(w.weights["w_qkv"], works[0].weights["w_qkv"]))
+            ref = oracle_reference(w, want_logits=False)
+            dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
+            dec.greedy_decode(w.dec_lens, toks, lens)
+            got, got_lens = toks.cpu().numpy(), lens.cpu().numpy()
+            assert np.array_equal(got_lens[:w.batch], w.dec_lens)
+            for u in range(w.batch):
+                L = int(w.dec_lens[u])
+                assert np.all(got[u, L:] == -1)
+                for t in range(L):
+                    if ref["margin"][u, t] <= MARGIN:
+                        break
+                    assert got[u, t] == ref["next"][u, t], (w.batch, u, t)
+                    total += 1
+    finally:
+        dec.close()
+    assert total > 0
+
+
+LN_CASES = {
+    "small": (SMALL, [37, 5, 70, 9], [9, 12, 4, 6]),
+    "mid": (MID, [1, 63, 130, 17, 40, 8, 90], [3, 20, 7, 11, 2, 16, 5]),
+    "wide": (dict(n_layers=2, d_model=1024, n_heads=16, d_ffn=2048, vocab=900, d_enc=256), [50, 3, 140, 21, 77], [6, 9, 3, 8, 5]),
+}
+
+
+@pytest.mark.parametrize("offset", [0.0, 4.0])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("case", ["small", "mid", "wide"])
+def test_layernorm_parameters_output_bias_and_mean_offset(case, dtype, offset):
+    """LayerNorm gains and shifts drawn around 1 and 0 (N(1, 0.3), N(0, 0.3)), an output-projection bias, and
+    (offset 4) an embedding table shifted by a constant so that the residual stream's mean dwarfs its spread:
+    the folded LayerNorm rstd * ((gamma * x) W^T - mean * c1) + c2 has to survive that cancellation."""
+    model, enc_lens, dec_lens = LN_CASES[case]
+    w = wl.make_custom(model, enc_lens, dec_lens, dtype=dtype, seed=91, ln_std=0.3, out_bias_std=0.3,
+                       embed_offset=offset)
+    _run_both(w, need_tokens=False, label=f"ln-{case}-offset{offset:g}")
+
+
+def test_long_rows_bf16():
+    """Decodes far beyond 128 cached positions (the self-attention block loops over its warps' chunks more than
+    once) beside a short one, with encoder outputs of up to 500 frames at a batch small enough for the
+    cross-attention variant that overlaps its loads: every step of every row against the checker."""
+    w = wl.make_custom(MID, [300, 40, 500, 9, 77], [240, 145, 129, 128, 17], dtype="bf16", seed=33, out_std=0.3)
+    _run_both(w, label="long-rows")
 
 
 def test_error_codes():
@@ -190,7 +265,7 @@ def test_large_batches_bf16(batch):
     enc_lens = rng.integers(1, 90, size=batch)
     dec_lens = rng.integers(1, 9, size=batch)
     dec_lens[:3] = [12, 1, 7]
-    w = wl.make_custom(MID, enc_lens, dec_lens, dtype="bf16", seed=40 + batch)
+    w = wl.make_custom(MID, enc_lens, dec_lens, dtype="bf16", seed=40 + batch, out_std=0.3)
     rows = [0, 1, 2, batch // 2, batch - 2, batch - 1] + [int(r) for r in rng.choice(batch, size=6, replace=False)]
     _run_both(w, rows=sorted(set(rows)))
 
@@ -201,7 +276,8 @@ def test_projection_stage_ring_reuse(batch, monkeypatch):
     (4 k-blocks for d = 256, 8 for the FFN), so stages are refilled while earlier ones are still being read."""
     monkeypatch.setenv("AED_DEC_GEMM_CTAS", "1")
     rng = np.random.default_rng(batch)
-    w = wl.make_custom(MID, rng.integers(1, 90, size=batch), rng.integers(1, 7, size=batch), dtype="bf16", seed=batch)
+    w = wl.make_custom(MID, rng.integers(1, 90, size=batch), rng.integers(1, 7, size=batch), dtype="bf16", seed=batch,
+                       out_std=0.3)
     _run_both(w, rows=[0, 1, batch // 2, batch - 1])
 
 
@@ -223,6 +299,10 @@ def test_config4_shape_sampled_rows():
     rows = sorted({int(order[0]), int(order[5]), int(order[17]), int(np.argmin(w.enc_lens))})
     rows = [r for r in rows if w.dec_lens[r] <= 24][:4]
     assert rows
+    # plus one long row: more than 128 tokens (the looping part of self-attention) over more than 400 frames
+    long_rows = [int(r) for r in np.flatnonzero((w.dec_lens > 128) & (w.enc_lens > 400))]
+    assert long_rows
+    rows = sorted(set(rows + [min(long_rows, key=lambda r: int(w.dec_lens[r]))]))
     _run_both(w, rows=rows)
 
 
@@ -236,6 +316,7 @@ def test_config2_shape_sampled_rows(cluster, monkeypatch):
     rows = sorted({int(order[0]), int(order[len(order) // 2]), int(order[3]), int(np.argmin(w.enc_lens))})
     # keep the checker's work bounded: drop sampled rows longer than 40 tokens
     rows = [r for r in rows if w.dec_lens[r] <= 40][:4]
+    rows = sorted(set(rows + [int(np.argmax(w.dec_lens))]))     # and the longest decode of the batch (131 tokens)
     _run_both(w, rows=rows)
 
 
@@ -254,7 +335,7 @@ def test_cluster_path_row_counts(batch, monkeypatch):
     enc_lens = rng.integers(1, 150, size=batch)
     dec_lens = rng.integers(1, 24, size=batch)
     enc_lens[0], dec_lens[0] = 1, 40              # one frame; longer than two 16-position chunks of the self cache
-    w = wl.make_custom(CLUSTER_A, enc_lens, dec_lens, dtype="bf16", seed=300 + batch)
+    w = wl.make_custom(CLUSTER_A, enc_lens, dec_lens, dtype="bf16", seed=300 + batch, out_std=0.3)
     rows = sorted({0, batch - 1, batch // 2, int(np.argmax(enc_lens))})
     _run_both(w, rows=rows)
 
@@ -263,7 +344,8 @@ def test_cluster_path_d1024(monkeypatch):
     monkeypatch.setenv("AED_DEC_CLUSTER", "1")
     rng = np.random.default_rng(31)
     batch = 24
-    w = wl.make_custom(CLUSTER_B, rng.integers(1, 200, size=batch), rng.integers(1, 20, size=batch), dtype="bf16", seed=77)
+    w = wl.make_custom(CLUSTER_B, rng.integers(1, 200, size=batch), rng.integers(1, 20, size=batch), dtype="bf16", seed=77,
+                       out_std=0.3)
     _run_both(w, rows=[0, 5, 23])
 
 

@@ -17,7 +17,7 @@
 #include "step_kernels.cuh"
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
-#include "cluster_step.cuh"
+#include "mega_step.cuh"
 
 using namespace aed;
 
@@ -49,10 +49,10 @@ struct Layout {
     size_t self_layer_elems, cross_layer_elems;
     int max_chunks;
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
-    size_t actd_hi, actd_lo, actf_hi, actf_lo;
+    size_t actd_hi, actd_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
-    size_t x1, x2;                        // the other two buffers of the rotating residual stream (cluster path)
-    size_t cl_blocks, cl_maps;            // block descriptions and tensor maps of the persistent step kernel
+    size_t x1;                            // second buffer of the residual stream (persistent step kernel)
+    size_t mega_bars, mega_maps, mega_layers;   // arrival counters, weight tensor maps and per-layer arguments of that kernel
     size_t fold_layer_floats;
     int rows_cap;
 };
@@ -116,16 +116,14 @@ Layout make_layout(const aed_dec_config_t &c)
     if (c.dtype == AED_DTYPE_BF16) {
         L.actd_hi = take((size_t)L.rows_cap * d * 2);
         L.actd_lo = take((size_t)L.rows_cap * d * 2);
-        L.actf_hi = take((size_t)L.rows_cap * F * 2);
-        L.actf_lo = take((size_t)L.rows_cap * F * 2);
         L.fold_layer_floats = 2 * (3 * d + d + F);       // c1 | c2 for qkv, then for cross-q, then for ffn1
         L.fold_c = take(L.fold_layer_floats * c.n_layers * 4);
         L.ln_stats = take((size_t)3 * rows_bucket(c.max_batch) * 8);
         L.qc = take(B * d * 4);
         L.x1 = take(B * d * 4);
-        L.x2 = take(B * d * 4);
-        L.cl_blocks = take((size_t)3 * c.n_layers * sizeof(cl::ClusterParams));
-        L.cl_maps = take((size_t)6 * c.n_layers * sizeof(CUtensorMap));
+        L.mega_bars = take(((size_t)c.n_layers * mega::kStagesPerLayer + 1) * 4);
+        L.mega_maps = take((size_t)6 * c.n_layers * sizeof(CUtensorMap));
+        L.mega_layers = take((size_t)c.n_layers * sizeof(mega::LayerArgs));
     }
     L.total = off;
     return L;
@@ -158,23 +156,19 @@ struct aed_dec {
     size_t prof_used = 0;
     // bf16 mode: TMA descriptors of the weight matrices and of the activation planes (one per MMA N in 16..256)
     struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2, kvc; };
-    struct ClLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };      // boxes of 64 rows x 64 k
-    std::vector<ClLayerMaps> cl_layers;
-    bool use_cluster = false;             // head-parallel cluster kernels for steps of at most 64 rows
-    bool use_persistent = true;           // all blocks of a step in one launch with grid-wide arrivals between them
-    int cl_prefetch = 0;                  // bit 0: next block's weights, bit 1: next block's K/V rows (L2 prefetch)
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
-    CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]
+    CUtensorMap tc_actd[5][2];                    // [log2(N/16)][plane]: final LayerNorm output, operand of the vocabulary projection
     CUtensorMap tc_src_x[5], tc_src_att[5], tc_src_hid[5];   // fp32 sources of the fused projections, per MMA N
     int tc_kvc_box = 0;                           // rows of the w_kv_c box = MMA N of the precompute
     bool use_tc = false;
-    int act_planes = 2;
+    // persistent step kernel (bf16 mode): one launch per step for steps of at most mega_rows rows
+    bool use_mega = false;
+    int mega_rows = 0, mega_slots = 0;
     int sm_count = 148;
     int tc_target_ctas = 128;
     bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
     bool use_pdl = true;
-    bool use_fused = true;
     bool attn_pipe = true;
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
@@ -218,11 +212,10 @@ aed_status_t fail(aed_dec *d, aed_status_t code, const char *fmt, ...)
 
 enum KernelFamily { KF_BOOKKEEPING = 0, KF_EMBED, KF_LAYERNORM, KF_GEMM_QKV, KF_ATTN_SELF, KF_ATTN_COMBINE, KF_GEMM_O,
                     KF_GEMM_QC, KF_ATTN_CROSS, KF_GEMM_OC, KF_GEMM_FF1, KF_GEMM_FF2, KF_GEMM_VOCAB, KF_PRECOMPUTE,
-                    KF_BLOCK_SELF, KF_BLOCK_CROSS, KF_BLOCK_FFN, KF_COUNT };
+                    KF_STEP_LAYERS, KF_COUNT };
 const char *const kFamilyNames[KF_COUNT] = {"bookkeeping", "embed", "layernorm", "gemm_qkv", "attn_self", "attn_combine",
                                             "gemm_o", "gemm_qc", "attn_cross", "gemm_oc", "gemm_ff1", "gemm_ff2",
-                                            "gemm_vocab", "precompute_cross_kv", "block_self", "block_cross",
-                                            "block_ffn"};
+                                            "gemm_vocab", "precompute_cross_kv", "step_layers"};
 
 // Records an event before and after the launches issued while it is alive (profiling mode only).
 struct ProfScope {
@@ -280,8 +273,7 @@ aed_status_t launch_gemm(aed_dec *dec, int family, int rows_ub, int rows_fixed, 
 
 template <typename T, bool kCross, bool kAppend = false>
 aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float *q, int ldq, const T *cache,
-                              int seq_capacity, float *out, __nv_bfloat16 *out_hi = nullptr,
-                              __nv_bfloat16 *out_lo = nullptr)
+                              int seq_capacity, float *out)
 {
     const auto &c = dec->cfg;
     const int H = c.n_heads;
@@ -298,14 +290,9 @@ aed_status_t launch_attention(aed_dec *dec, int rows_ub, int len_ub, const float
     AED_LAUNCHED(dec);
     }
     ProfScope ps(dec, KF_ATTN_COMBINE);
-    if (out_hi)
-        attn_combine_planes_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
+    attn_combine_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
             dec->state(), dec->at<int32_t>(dec->lay.active_list), partials, H, dec->at<int32_t>(dec->lay.t_u),
-            dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out_hi, out_lo, c.d_model);
-    else
-        attn_combine_kernel<kCross><<<(rows_ub * H + 3) / 4, 128, 0, dec->stream>>>(
-            dec->state(), dec->at<int32_t>(dec->lay.active_list), partials, H, dec->at<int32_t>(dec->lay.t_u),
-            dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out, c.d_model);
+        dec->at<int32_t>(dec->lay.enc_len), dec->lay.max_chunks, out, c.d_model);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -446,7 +433,122 @@ bool encode_map(CUtensorMap *map, const void *base, size_t rows, size_t cols, in
 
 constexpr int kTcSmemBudget = 200 * 1024;
 
-cl::ClusterParams cluster_block_params(const aed_dec *dec, int l, int k);
+// ---- persistent step kernel (bf16 mode, small batches) ----------------------------------------------------------
+
+mega::MegaParams mega_params(const aed_dec *dec)
+{
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    mega::MegaParams p{};
+    p.n_layers = c.n_layers; p.d = c.d_model; p.n_heads = c.n_heads; p.d_ffn = c.d_ffn;
+    p.n_slots = dec->mega_slots;
+    p.self_capacity = c.max_dec_len; p.frame_capacity = c.max_total_enc_frames;
+    p.scale = 1.0f / sqrtf((float)kHeadDim); p.eps = c.ln_eps;
+    p.x0 = dec->at<float>(L.x); p.x1 = dec->at<float>(L.x1);
+    p.qkv = dec->at<float>(L.qkv); p.hid = dec->at<float>(L.hid);
+    p.stats1 = dec->at<float2>(L.ln_stats); p.stats3 = dec->at<float2>(L.ln_stats) + 2 * rows_bucket(c.max_batch);
+    p.row_info = dec->at<int4>(L.row_info);
+    p.state = dec->state();
+    p.bars = dec->at<int>(L.mega_bars);
+    p.maps = dec->at<CUtensorMap>(L.mega_maps);
+    p.layers = dec->at<mega::LayerArgs>(L.mega_layers);
+    return p;
+}
+
+// Decide whether the persistent step kernel can run on this device for this model, and stage what it reads.
+aed_status_t mega_setup(aed_dec *dec)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const size_t d = c.d_model, F = c.d_ffn;
+    const char *v = getenv("AED_DEC_PERSISTENT");
+    if (v && v[0] == '0') return AED_OK;                  // A/B runs and the tests of the kernel chain at small batches
+    const int G = dec->sm_count;
+    if (d < 128 || d > 1024 || F < 128 || c.n_heads > G || G < mega::kMaxRows) return AED_OK;
+    // ring depth: what fits beside the fixed regions
+    int slots = mega::kMaxSlots;
+    while (slots > 4 && mega::smem_layout(slots).total + 1024 > kTcSmemBudget + 20 * 1024) --slots;
+    const int smem = mega::smem_layout(slots).total + 1024;
+    cudaError_t e = cudaFuncSetAttribute(mega::mega_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    int per_sm = 0;
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mega::mega_step_kernel, mega::kThreads, smem);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return AED_OK; }
+    if (per_sm < 1) return AED_OK;
+    std::vector<CUtensorMap> maps(6 * c.n_layers);
+    std::vector<mega::LayerArgs> layers(c.n_layers);
+    bool ok = true;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        CUtensorMap *m = &maps[6 * l];
+        ok = ok && encode_map(m + 0, w.w_qkv, 3 * d, d, tc::kTileM) && encode_map(m + 1, w.w_o, d, d, tc::kTileM) &&
+             encode_map(m + 2, w.w_q_c, d, d, 64) && encode_map(m + 3, w.w_o_c, d, d, tc::kTileM) &&
+             encode_map(m + 4, w.w_ff1, F, d, tc::kTileM) && encode_map(m + 5, w.w_ff2, d, F, tc::kTileM);
+        const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
+        mega::LayerArgs &a = layers[l];
+        a.ln1_g = (const T *)w.ln1_g; a.ln2_g = (const T *)w.ln2_g; a.ln3_g = (const T *)w.ln3_g;
+        a.c1_qkv = fc; a.c2_qkv = fc + 3 * d; a.c1_qc = fc + 6 * d; a.c2_qc = fc + 7 * d; a.c1_ff = fc + 8 * d; a.c2_ff = fc + 8 * d + F;
+        a.b_o = (const T *)w.b_o; a.b_oc = (const T *)w.b_o_c; a.b_ff2 = (const T *)w.b_ff2;
+        a.self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
+        a.cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+    }
+    if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the persistent step kernel");
+    e = cudaMemcpyAsync(dec->ws + L.mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, dec->stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(dec->ws + L.mega_layers, layers.data(), layers.size() * sizeof(mega::LayerArgs), cudaMemcpyHostToDevice, dec->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(dec->stream);      // the host vectors go away
+    if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "persistent step kernel set-up: %s", cudaGetErrorString(e));
+    dec->mega_slots = slots;
+    dec->mega_rows = std::min(mega::kMaxRows, (G / c.n_heads) * mega::kUnitRows);
+    dec->use_mega = true;
+    return AED_OK;
+}
+
+aed_status_t launch_ln_planes(aed_dec *dec, int rows_ub, const float *x, const void *g, const void *b, float *zero_buf, int zero_cols);
+aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p);
+
+// One step through the persistent kernel: embedding, all layers in one cooperative launch, final LayerNorm,
+// vocabulary projection.
+aed_status_t forward_step_mega(aed_dec *dec, int rows_ub, const int32_t *tokens, float *logits_out)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const int d = c.d_model, V = c.vocab;
+    float *x0 = dec->at<float>(L.x), *x1 = dec->at<float>(L.x1);
+    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
+    {
+        ProfScope ps(dec, KF_EMBED);
+        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x0, dec->at<float>(L.qkv), 3 * d);
+        AED_LAUNCHED(dec);
+    }
+    {
+        ProfScope ps(dec, KF_STEP_LAYERS);
+        const mega::MegaParams p = mega_params(dec);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(dec->sm_count);
+        cfg.blockDim = dim3(mega::kThreads);
+        cfg.dynamicSmemBytes = (size_t)mega::smem_layout(dec->mega_slots).total + 1024;
+        cfg.stream = dec->stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;        // every block resident at once: they wait on one another
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, mega::mega_step_kernel, p);
+        if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "persistent step launch: %s", cudaGetErrorString(e));
+        AED_LAUNCHED(dec);
+    }
+    AED_TRY(launch_ln_planes(dec, rows_ub, (c.n_layers & 1) ? x1 : x0, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
+    tc::TcParams tp{};
+    tp.bias = (const T *)dec->b_out;
+    tp.logits_out = logits_out;
+    tp.keys = dec->at<unsigned long long>(L.keys);
+    tp.active_list = active_list;
+    AED_TRY(launch_vocab_gemm(dec, rows_ub, tp));
+    return AED_OK;
+}
 
 aed_status_t tc_setup(aed_dec *dec)
 {
@@ -470,16 +572,13 @@ aed_status_t tc_setup(aed_dec *dec)
         const int box = 16 << i;
         ok = ok && encode_map(&dec->tc_actd[i][0], dec->ws + L.actd_hi, L.rows_cap, d, box) &&
              encode_map(&dec->tc_actd[i][1], dec->ws + L.actd_lo, L.rows_cap, d, box) &&
-             encode_map(&dec->tc_actf[i][0], dec->ws + L.actf_hi, L.rows_cap, F, box) &&
-             encode_map(&dec->tc_actf[i][1], dec->ws + L.actf_lo, L.rows_cap, F, box) &&
              encode_map(&dec->tc_src_x[i], dec->ws + L.x, c.max_batch, d, box, true) &&
              encode_map(&dec->tc_src_att[i], dec->ws + L.act, c.max_batch, d, box, true) &&
              encode_map(&dec->tc_src_hid[i], dec->ws + L.hid, c.max_batch, F, box, true);
     }
     if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed (are all weight tensors 16-byte aligned?)");
     const int smem = kTcSmemBudget + 1024;
-    cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_CROSSKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     int dev = 0, sms = 0;
     if (e == cudaSuccess) e = cudaGetDevice(&dev);
@@ -510,96 +609,11 @@ aed_status_t tc_setup(aed_dec *dec)
         dec->use_pdl = !(v && v[0] == '1');
         v = getenv("AED_DEC_NO_ATTN_PIPE");
         dec->attn_pipe = !(v && v[0] == '1');
-        v = getenv("AED_DEC_NO_FUSED");
-        dec->use_fused = !(v && v[0] == '1');
     }
-    const char *planes = getenv("AED_DEC_ACT_PLANES");
-    dec->act_planes = (planes && planes[0] == '1') ? 1 : 2;
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
     if (ctas && atoi(ctas) > 0) { dec->tc_target_ctas = atoi(ctas); dec->tc_target_fixed = true; }
-    // head-parallel cluster path: shapes whose projections split evenly over 8 CTAs and 16 clusters
-    {
-        // opt-in until it beats the kernel-per-projection path at every row count
-        const char *v = getenv("AED_DEC_CLUSTER");
-        const bool want = v && v[0] == '1';
-        const bool shape_ok = (d == 512 || d == 1024) && c.n_heads <= cl::kClusters / 2 && F % 128 == 0 &&
-                              F / 128 <= (size_t)cl::kClusters;
-        if (want && shape_ok && dec->use_fused) {
-            dec->cl_layers.resize(c.n_layers);
-            bool ok2 = true;
-            for (int l = 0; l < c.n_layers; ++l) {
-                const LayerWeights &w = dec->layers[l];
-                aed_dec::ClLayerMaps &m = dec->cl_layers[l];
-                ok2 = ok2 && encode_map(&m.qkv, w.w_qkv, 3 * d, d, 64) && encode_map(&m.o, w.w_o, d, d, 64) &&
-                      encode_map(&m.qc, w.w_q_c, d, d, 64) && encode_map(&m.oc, w.w_o_c, d, d, 64) &&
-                      encode_map(&m.ff1, w.w_ff1, F, d, 64) && encode_map(&m.ff2, w.w_ff2, d, F, 64);
-            }
-            if (!ok2) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the cluster path");
-            const int kbs = (int)d / cl::kCS / tc::kBlockK;
-            auto max_smem = [&](int kind) {
-                int m = 0;
-                for (int n = 16; n <= cl::kMaxRows; n <<= 1) m = std::max(m, cl::cl_layout(kind, n, kbs).total + 1024);
-                return m;
-            };
-            cudaError_t e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_SELF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                  max_smem(cl::K_SELF));
-            if (e2 == cudaSuccess)
-                e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_CROSS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          max_smem(cl::K_CROSS));
-            if (e2 == cudaSuccess)
-                e2 = cudaFuncSetAttribute(cl::cluster_block_kernel<cl::K_FFN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          max_smem(cl::K_FFN));
-            if (e2 == cudaSuccess)
-                e2 = cudaFuncSetAttribute(cl::cluster_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          std::max(max_smem(cl::K_SELF), std::max(max_smem(cl::K_CROSS), max_smem(cl::K_FFN))));
-            if (e2 != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "cluster path set-up: %s", cudaGetErrorString(e2));
-            // All clusters of a launch must be resident at once, or the launch runs in two waves and loses more
-            // than the path gains: ask the device (the answer depends on how many SMs each GPC of this chip has).
-            bool resident = true;
-            for (int kind = 0; kind < 3 && resident; ++kind) {
-                cudaLaunchConfig_t cfg = {};
-                cfg.gridDim = dim3(cl::kClusters * cl::kCS);
-                cfg.blockDim = dim3(cl::kClThreads);
-                cfg.dynamicSmemBytes = (size_t)max_smem(kind);
-                cudaLaunchAttribute attr[1];
-                attr[0].id = cudaLaunchAttributeClusterDimension;
-                attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-                cfg.attrs = attr;
-                cfg.numAttrs = 1;
-                int n = 0;
-                cudaError_t e3 = kind == 0   ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_SELF>, &cfg)
-                                 : kind == 1 ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_CROSS>, &cfg)
-                                             : cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_FFN>, &cfg);
-                if (e3 != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-                resident = n >= cl::kClusters;
-            }
-            dec->use_cluster = resident;
-            if (resident) {
-                // block descriptions and tensor maps of the persistent step kernel, in the workspace
-                std::vector<cl::ClusterParams> blocks(3 * c.n_layers);
-                std::vector<CUtensorMap> maps(6 * c.n_layers);
-                const char *pf0 = getenv("AED_DEC_CL_PREFETCH");
-                if (pf0) dec->cl_prefetch = atoi(pf0);
-                for (int l = 0; l < c.n_layers; ++l) {
-                    for (int k = 0; k < 3; ++k) blocks[3 * l + k] = cluster_block_params(dec, l, k);
-                    const aed_dec::ClLayerMaps &m = dec->cl_layers[l];
-                    const CUtensorMap six[6] = {m.qkv, m.o, m.qc, m.oc, m.ff1, m.ff2};
-                    for (int i = 0; i < 6; ++i) maps[6 * l + i] = six[i];
-                }
-                cudaError_t e4 = cudaMemcpyAsync(dec->ws + L.cl_blocks, blocks.data(), blocks.size() * sizeof(cl::ClusterParams),
-                                                 cudaMemcpyHostToDevice, dec->stream);
-                if (e4 == cudaSuccess)
-                    e4 = cudaMemcpyAsync(dec->ws + L.cl_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice,
-                                         dec->stream);
-                if (e4 == cudaSuccess) e4 = cudaStreamSynchronize(dec->stream);      // the host vectors go away
-                if (e4 != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "cluster path set-up: %s", cudaGetErrorString(e4));
-                const char *pv = getenv("AED_DEC_NO_PERSIST");
-                dec->use_persistent = !(pv && pv[0] == '1');
-            }
-        }
-    }
     dec->use_tc = true;
-    return AED_OK;
+    return mega_setup(dec);
 }
 
 // MMA N for a step with at most rows_ub rows: the smallest of 16, 32, ..., 256 that covers them (or 256).
@@ -610,38 +624,28 @@ int tc_n_index(int rows_ub)
     return i;
 }
 
-// One projection of the step on tensor cores: out[r, o] += sum_k act[r, k] * W[o, k] (+ bias by the first k-split).
-template <int EPI>
-aed_status_t launch_tc_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, int M, int K, bool act_is_ffn,
-                            int rows_ub, tc::TcParams p)
+// The vocabulary projection on tensor cores: logits[r, v] = sum_k act[r, k] * Wout[v, k] (+ bias), argmax in the epilogue.
+aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p)
 {
-    ProfScope ps(dec, family);
+    ProfScope ps(dec, KF_GEMM_VOCAB);
+    const int M = dec->cfg.vocab, K = dec->cfg.d_model;
     const int ni = tc_n_index(rows_ub), n_tile = 16 << ni;
     const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
     const int k_blocks = K / tc::kBlockK;
-    int splits = 1;
-    if (EPI == tc::TC_EPI_ADD) {
-        // About 64 CTAs with deep TMA rings already pull the weights at HBM rate; more k-splits only multiply
-        // the red.global traffic of the epilogue (splits x rows x features x 4 bytes).
-        splits = dec->tc_target_ctas / (m_tiles * row_tiles);
-        if (splits < 1) splits = 1;
-        if (splits > k_blocks) splits = k_blocks;
-    }
     p.a_rows = M;
     p.n_tile = n_tile;
     p.k_blocks = k_blocks;
-    p.use_lo = dec->act_planes == 2;
+    p.use_lo = 1;
     p.rows_fixed = -1;
     p.state = dec->state();
-    const int stage_bytes = tc::kATileBytes + dec->act_planes * n_tile * tc::kBlockK * 2;
+    const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2;
     int stages = kTcSmemBudget / stage_bytes;
-    const int kb_per_split = (k_blocks + splits - 1) / splits;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
-    if (stages > kb_per_split) stages = kb_per_split;
-    const CUtensorMap *acts = act_is_ffn ? dec->tc_actf[ni] : dec->tc_actd[ni];
-    dim3 grid(m_tiles, splits, row_tiles);
-    tc::tc_gemm_kernel<EPI><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
-        map_w, acts[0], acts[1], p, stages);
+    if (stages > k_blocks) stages = k_blocks;
+    const CUtensorMap *acts = dec->tc_actd[ni];
+    dim3 grid(m_tiles, 1, row_tiles);
+    tc::tc_gemm_kernel<tc::TC_EPI_LOGITS><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
+        dec->tc_w_out, acts[0], acts[1], p, stages);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -657,69 +661,7 @@ aed_status_t launch_ln_planes(aed_dec *dec, int rows_ub, const float *x, const v
         dec->at<__nv_bfloat16>(L.actd_hi), dec->at<__nv_bfloat16>(L.actd_lo), zero_buf, zero_cols);
     AED_LAUNCHED(dec);
     return AED_OK;
-}
-
-aed_status_t forward_step_tc(aed_dec *dec, int rows_ub, int self_len_ub, const int32_t *tokens, float *logits_out)
-{
-    typedef __nv_bfloat16 T;
-    const auto &c = dec->cfg;
-    const Layout &L = dec->lay;
-    const int d = c.d_model, F = c.d_ffn, V = c.vocab;
-    float *x = dec->at<float>(L.x), *qkv = dec->at<float>(L.qkv), *hid = dec->at<float>(L.hid);
-    T *ad_hi = dec->at<T>(L.actd_hi), *ad_lo = dec->at<T>(L.actd_lo);
-    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
-    {
-        ProfScope ps(dec, KF_EMBED);
-        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x);
-        AED_LAUNCHED(dec);
-    }
-    tc::TcParams p{};
-    for (int l = 0; l < c.n_layers; ++l) {
-        const LayerWeights &w = dec->layers[l];
-        const aed_dec::TcLayerMaps &m = dec->tc_layers[l];
-        T *self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
-        const T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-        // masked self-attention: [q | k | v] rows accumulate in qkv, the attention kernel appends k, v to the cache
-        AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln1_g, w.ln1_b, qkv, 3 * d));
-        p.out = qkv; p.ldo = 3 * d; p.bias = (const T *)w.b_qkv;
-        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_QKV, m.qkv, 3 * d, d, false, rows_ub, p));
-        AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len,
-                                                        nullptr, ad_hi, ad_lo)));
-        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
-        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_O, m.o, d, d, false, rows_ub, p));
-        // cross-attention
-        AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln2_g, w.ln2_b, qkv, d));
-        p.out = qkv; p.ldo = d; p.bias = (const T *)w.b_q_c;
-        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_QC, m.qc, d, d, false, rows_ub, p));
-        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qkv, d, cross, c.max_total_enc_frames,
-                                                        nullptr, ad_hi, ad_lo)));
-        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
-        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_OC, m.oc, d, d, false, rows_ub, p));
-        // feed-forward
-        AED_TRY(launch_ln_planes(dec, rows_ub, x, w.ln3_g, w.ln3_b, hid, F));
-        p.out = hid; p.ldo = F; p.bias = (const T *)w.b_ff1;
-        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_FF1, m.ff1, F, d, false, rows_ub, p));
-        {
-            ProfScope ps(dec, KF_LAYERNORM);
-            dim3 grid((F / 4 + 255) / 256, rows_ub);
-            relu_planes_kernel<<<grid, 256, 0, dec->stream>>>(dec->state(), hid, F, dec->at<T>(L.actf_hi), dec->at<T>(L.actf_lo));
-            AED_LAUNCHED(dec);
-        }
-        p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
-        AED_TRY(launch_tc_gemm<tc::TC_EPI_ADD>(dec, KF_GEMM_FF2, m.ff2, d, F, true, rows_ub, p));
-    }
-    AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
-    p.out = nullptr; p.bias = (const T *)dec->b_out;
-    p.logits_out = logits_out;
-    p.keys = dec->at<unsigned long long>(L.keys);
-    p.active_list = active_list;
-    AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, p));
-    return AED_OK;
-}
-
-
-// ---- fused step (bf16 mode): 8 kernels per layer, chained with programmatic dependent launch -------------------
+}// ---- fused step (bf16 mode): 8 kernels per layer, chained with programmatic dependent launch -------------------
 
 struct FusedGemm {
     const CUtensorMap *map;
@@ -858,128 +800,7 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
     tp.logits_out = logits_out;
     tp.keys = dec->at<unsigned long long>(L.keys);
     tp.active_list = active_list;
-    AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, tp));
-    return AED_OK;
-}
-
-// ---- head-parallel cluster step (bf16 mode, at most 64 rows): 3 cluster kernels per layer ----------------------
-
-// Description of block k (0 self, 1 cross, 2 FFN) of layer l: buffers of the rotating residual stream, LayerNorm
-// fold constants, caches, and the static data of the following block to pull into L2.
-cl::ClusterParams cluster_block_params(const aed_dec *dec, int l, int k)
-{
-    typedef __nv_bfloat16 T;
-    const auto &c = dec->cfg;
-    const Layout &L = dec->lay;
-    const size_t d = c.d_model, F = c.d_ffn, e2 = sizeof(T);
-    float *xb[3] = {dec->at<float>(L.x), dec->at<float>(L.x1), dec->at<float>(L.x2)};
-    const LayerWeights &w = dec->layers[l];
-    const int ln = (l + 1) % c.n_layers;               // next layer (or layer 0 of the next step)
-    const LayerWeights &wn = dec->layers[ln];
-    const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
-    T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-    const int blk = 3 * l + k;
-    cl::ClusterParams p{};
-    p.d = c.d_model; p.n_heads = c.n_heads; p.d_ffn = c.d_ffn;
-    p.x_in = xb[blk % 3]; p.x_out = xb[(blk + 1) % 3]; p.x_zero = xb[(blk + 2) % 3];
-    p.row_info = dec->at<int4>(L.row_info);
-    p.scale = 1.0f / sqrtf((float)kHeadDim);
-    p.eps = c.ln_eps;
-    p.state = dec->state();
-    if (k == 0) {           // next: the cross-attention weights and this layer's encoder K/V
-        p.gamma = (const T *)w.ln1_g; p.c1 = fc; p.c2 = fc + 3 * d; p.bias2 = (const T *)w.b_o;
-        p.cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems; p.seq_capacity = c.max_dec_len;
-        p.pf_ptr[0] = w.w_q_c; p.pf_bytes[0] = d * d * e2; p.pf_ptr[1] = w.w_o_c; p.pf_bytes[1] = d * d * e2;
-        p.pf_cache = cross; p.pf_capacity = c.max_total_enc_frames; p.pf_cross = 1;
-    } else if (k == 1) {    // next: the feed-forward weights
-        p.gamma = (const T *)w.ln2_g; p.c1 = fc + 6 * d; p.c2 = fc + 7 * d; p.bias2 = (const T *)w.b_o_c;
-        p.cache = cross; p.seq_capacity = c.max_total_enc_frames;
-        p.pf_ptr[0] = w.w_ff1; p.pf_bytes[0] = F * d * e2; p.pf_ptr[1] = w.w_ff2; p.pf_bytes[1] = F * d * e2;
-    } else {                // next: the self-attention weights and cache of the next layer
-        p.gamma = (const T *)w.ln3_g; p.c1 = fc + 8 * d; p.c2 = fc + 8 * d + F; p.bias2 = (const T *)w.b_ff2;
-        p.pf_ptr[0] = wn.w_qkv; p.pf_bytes[0] = 3 * d * d * e2; p.pf_ptr[1] = wn.w_o; p.pf_bytes[1] = d * d * e2;
-        p.pf_cache = dec->at<T>(L.self_cache) + (size_t)ln * L.self_layer_elems; p.pf_capacity = c.max_dec_len; p.pf_cross = 0;
-    }
-    if (!(dec->cl_prefetch & 1)) p.pf_ptr[0] = p.pf_ptr[1] = nullptr;
-    if (!(dec->cl_prefetch & 2)) p.pf_cache = nullptr;
-    return p;
-}
-
-template <int KIND>
-aed_status_t launch_cluster_block(aed_dec *dec, int family, const CUtensorMap &map_w1, const CUtensorMap &map_w2,
-                                  int rows_ub, cl::ClusterParams p)
-{
-    ProfScope ps(dec, family);
-    p.n_tile = 16 << tc_n_index(rows_ub);
-    const int kbs = dec->cfg.d_model / cl::kCS / tc::kBlockK;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cl::kClusters * cl::kCS);
-    cfg.blockDim = dim3(cl::kClThreads);
-    cfg.dynamicSmemBytes = (size_t)cl::cl_layout(KIND, p.n_tile, kbs).total + 1024;
-    cfg.stream = dec->stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, cl::cluster_block_kernel<KIND>, map_w1, map_w2, p);
-    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "cluster block launch: %s", cudaGetErrorString(e));
-    AED_LAUNCHED(dec);
-    return AED_OK;
-}
-
-aed_status_t forward_step_cluster(aed_dec *dec, int rows_ub, const int32_t *tokens, float *logits_out)
-{
-    typedef __nv_bfloat16 T;
-    const auto &c = dec->cfg;
-    const Layout &L = dec->lay;
-    const int d = c.d_model, V = c.vocab;
-    float *x0 = dec->at<float>(L.x), *x1 = dec->at<float>(L.x1);
-    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
-    {
-        ProfScope ps(dec, KF_EMBED);
-        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x0, x1, d);
-        AED_LAUNCHED(dec);
-    }
-    if (dec->use_persistent && !dec->profiling) {
-        // every block of the step in one launch
-        ProfScope ps(dec, KF_BLOCK_SELF);
-        const int n_tile = 16 << tc_n_index(rows_ub), kbs = d / cl::kCS / tc::kBlockK;
-        size_t smem = 0;
-        for (int k = 0; k < 3; ++k) smem = std::max(smem, (size_t)cl::cl_layout(k, n_tile, kbs).total + 1024);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(cl::kClusters * cl::kCS);
-        cfg.blockDim = dim3(cl::kClThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = dec->stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, cl::cluster_step_kernel, (const cl::ClusterParams *)dec->at<cl::ClusterParams>(L.cl_blocks),
-                                           (const CUtensorMap *)dec->at<CUtensorMap>(L.cl_maps), 3 * c.n_layers, n_tile);
-        if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "cluster step launch: %s", cudaGetErrorString(e));
-        AED_LAUNCHED(dec);
-    } else {
-        for (int l = 0; l < c.n_layers; ++l) {
-            const aed_dec::ClLayerMaps &m = dec->cl_layers[l];
-            AED_TRY(launch_cluster_block<cl::K_SELF>(dec, KF_BLOCK_SELF, m.qkv, m.o, rows_ub, cluster_block_params(dec, l, 0)));
-            AED_TRY(launch_cluster_block<cl::K_CROSS>(dec, KF_BLOCK_CROSS, m.qc, m.oc, rows_ub, cluster_block_params(dec, l, 1)));
-            AED_TRY(launch_cluster_block<cl::K_FFN>(dec, KF_BLOCK_FFN, m.ff1, m.ff2, rows_ub, cluster_block_params(dec, l, 2)));
-        }
-    }
-    // 3 blocks per layer: the result is back in the first buffer
-    AED_TRY(launch_ln_planes(dec, rows_ub, x0, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
-    tc::TcParams tp{};
-    tp.bias = (const T *)dec->b_out;
-    tp.logits_out = logits_out;
-    tp.keys = dec->at<unsigned long long>(L.keys);
-    tp.active_list = active_list;
-    AED_TRY(launch_tc_gemm<tc::TC_EPI_LOGITS>(dec, KF_GEMM_VOCAB, dec->tc_w_out, V, d, false, rows_ub, tp));
+    AED_TRY(launch_vocab_gemm(dec, rows_ub, tp));
     return AED_OK;
 }
 
@@ -1007,7 +828,7 @@ aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
     int stages = kTcSmemBudget / stage_bytes;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     if (stages > p.k_blocks) stages = p.k_blocks;
-    dim3 grid((dec->total_frames + tc::kTileM - 1) / tc::kTileM, 1, 2 * c.d_model / p.n_tile);
+    dim3 grid((dec->total_frames + tc::kTileM - 1) / tc::kTileM, 1, (2 * c.d_model + p.n_tile - 1) / p.n_tile);
     for (int l = 0; l < c.n_layers; ++l) {
         ProfScope ps(dec, KF_PRECOMPUTE);
         p.cross_store = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
@@ -1045,7 +866,9 @@ aed_status_t launch_build_active(aed_dec *dec, const uint8_t *mask)
                                                      dec->at<int32_t>(L.active_list), dec->state(),
                                                      dec->at<int32_t>(L.enc_len), dec->at<int32_t>(L.enc_off),
                                                      dec->at<int4>(L.row_info), rows_bucket(dec->cfg.max_batch),
-                                                     dec->at<int32_t>(L.len_order));
+                                                     dec->at<int32_t>(L.len_order),
+                                                     dec->use_mega ? dec->at<int>(L.mega_bars) : nullptr,
+                                                     dec->use_mega ? dec->cfg.n_layers * mega::kStagesPerLayer + 1 : 0);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -1185,9 +1008,7 @@ extern "C" aed_status_t aed_dec_precompute_cross_kv(aed_dec_t *dec, const void *
     }
     AED_CUDA(dec, cudaMemsetAsync(dec->ws + L.keys, 0, L.enc_off - L.keys, dec->stream));   // keys, state, t_u, retired, lists
     AED_CUDA(dec, cudaMemcpyAsync(&dec->state()->batch, &dec->batch, sizeof(int32_t), cudaMemcpyHostToDevice, dec->stream));
-    aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed)
-                     : dec->cfg.dtype == AED_DTYPE_BF16 ? precompute_impl<__nv_bfloat16>(dec, enc_packed)
-                                                        : precompute_impl<float>(dec, enc_packed);
+    aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed) : precompute_impl<float>(dec, enc_packed);
     if (s != AED_OK) return s;
     dec->have_batch = true;
     dec->fresh_batch = true;
@@ -1207,11 +1028,9 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_build_active(dec, active));
     const int rows_ub = dec->batch;
     const int self_len_ub = dec->steps_issued + 1 < dec->cfg.max_dec_len ? dec->steps_issued + 1 : dec->cfg.max_dec_len;
-    aed_status_t s = (dec->use_cluster && rows_ub <= cl::kMaxRows) ? forward_step_cluster(dec, rows_ub, tokens_in, logits_out)
-                     : dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out) : forward_step_tc(dec, rows_ub, self_len_ub, tokens_in, logits_out))
-                     : dec->cfg.dtype == AED_DTYPE_BF16
-                         ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tokens_in, logits_out)
-                         : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
+    aed_status_t s = (dec->use_mega && rows_ub <= dec->mega_rows) ? forward_step_mega(dec, rows_ub, tokens_in, logits_out)
+                     : dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out)
+                                   : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
     if (s != AED_OK) return s;
     AED_TRY(launch_finish(dec, rows_ub, next_out, 0, nullptr, nullptr));
     dec->steps_issued++;
@@ -1283,10 +1102,9 @@ aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int
     if (self_len_ub > dec->cfg.max_dec_len) self_len_ub = dec->cfg.max_dec_len;
     AED_TRY(launch_build_active(dec, nullptr));
     const int32_t *tok = dec->at<int32_t>(L.cur_tok);
-    aed_status_t st = (dec->use_cluster && rows_ub <= cl::kMaxRows) ? forward_step_cluster(dec, rows_ub, tok, nullptr)
-                      : dec->use_tc ? (dec->use_fused ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr) : forward_step_tc(dec, rows_ub, self_len_ub, tok, nullptr))
-                      : dec->cfg.dtype == AED_DTYPE_BF16 ? forward_step<__nv_bfloat16>(dec, rows_ub, self_len_ub, tok, nullptr)
-                                                         : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
+    aed_status_t st = (dec->use_mega && rows_ub <= dec->mega_rows) ? forward_step_mega(dec, rows_ub, tok, nullptr)
+                      : dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr)
+                                    : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
     if (st != AED_OK) return st;
     return launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens);
 }
@@ -1345,7 +1163,10 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
         const int rows_ub = alive[s];
         if (dec->use_graphs && !dec->profiling) {
             // grids are sized for the bucket; kernels leave rows beyond the device-side row count alone
-            const int rows_b = rows_bucket(rows_ub), chunks = (s + 1 + kAttnChunk - 1) / kAttnChunk;
+            // (the persistent kernel reads the row count and every length on the device: one graph serves all its steps)
+            const bool mega_step = dec->use_mega && rows_ub <= dec->mega_rows;
+            const int rows_b = mega_step ? dec->mega_rows : rows_bucket(rows_ub);
+            const int chunks = mega_step ? 0 : (s + 1 + kAttnChunk - 1) / kAttnChunk;
             const aed_dec::GraphKey key(rows_b, chunks, tokens_out, out_lens);
             auto it = dec->graphs.find(key);
             if (it == dec->graphs.end()) {
@@ -1416,44 +1237,6 @@ extern "C" int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, co
     }
     return n;
 }
-
-#ifdef AED_TRACE
-// Debug builds only: how many clusters of a block kernel the device holds at once (row tile n_tile).
-extern "C" int32_t aed_dec_cluster_occupancy(aed_dec_t *dec, int32_t kind, int32_t n_tile)
-{
-    if (!dec || !dec->use_cluster) return -1;
-    const int kbs = dec->cfg.d_model / cl::kCS / tc::kBlockK;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cl::kClusters * cl::kCS);
-    cfg.blockDim = dim3(cl::kClThreads);
-    cfg.dynamicSmemBytes = (size_t)cl::cl_layout(kind, n_tile, kbs).total + 1024;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cl::kCS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int n = -1;
-    cudaError_t e = kind == 0   ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_SELF>, &cfg)
-                    : kind == 1 ? cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_CROSS>, &cfg)
-                                : cudaOccupancyMaxActiveClusters(&n, cl::cluster_block_kernel<cl::K_FFN>, &cfg);
-    return e == cudaSuccess ? n : -2;
-}
-
-// Debug builds only: copy out the device-side start-time trace (ids and nanosecond stamps) and clear it.
-extern "C" int32_t aed_dec_trace_read(aed_dec_t *dec, int32_t max_events, uint32_t *ids, unsigned long long *t_ns)
-{
-    if (!dec) return AED_ERR_INVALID_ARG;
-    if (cudaStreamSynchronize(dec->stream) != cudaSuccess) return AED_ERR_CUDA;
-    static TraceBuf host;
-    char *src = dec->ws + dec->lay.state + 256;
-    if (cudaMemcpy(&host, src, sizeof host, cudaMemcpyDeviceToHost) != cudaSuccess) return AED_ERR_CUDA;
-    cudaMemset(src, 0, 8);
-    int n = host.count < (1u << 16) ? (int)host.count : (1 << 16);
-    if (n > max_events) n = max_events;
-    for (int i = 0; i < n; ++i) { ids[i] = host.ev[i].id; t_ns[i] = host.ev[i].t_ns; }
-    return n;
-}
-#endif
 
 extern "C" int64_t aed_dec_launch_count(const aed_dec_t *dec) { return dec ? dec->launches : 0; }
 

@@ -19,7 +19,8 @@ __global__ void build_active_kernel(const uint8_t *__restrict__ mask, const int3
                                     const int32_t *__restrict__ t_u, int max_dec_len,
                                     int32_t *__restrict__ active_list, DecState *state,
                                     const int32_t *__restrict__ enc_len, const int32_t *__restrict__ enc_off,
-                                    int4 *__restrict__ row_info, int row_slots, const int32_t *__restrict__ order)
+                                    int4 *__restrict__ row_info, int row_slots, const int32_t *__restrict__ order,
+                                    int *__restrict__ step_counters, int n_step_counters)
 {
     AED_TRACE_BEGIN(state, 1);
     __shared__ int warp_counts[32];
@@ -57,6 +58,8 @@ __global__ void build_active_kernel(const uint8_t *__restrict__ mask, const int3
         __syncthreads();
     }
     if (threadIdx.x == 0) { state->n_active = base; state->grid_sync = 0; }
+    // arrival counters (and the abort word) of the persistent step kernel start every step at zero
+    for (int i = threadIdx.x; i < n_step_counters; i += blockDim.x) step_counters[i] = 0;
     for (int r = base + threadIdx.x; r < row_slots; r += blockDim.x) row_info[r] = make_int4(-1, 0, 0, 0);
 }
 
@@ -650,41 +653,6 @@ attn_combine_kernel(const DecState *state, const int32_t *__restrict__ active_li
     *reinterpret_cast<float2 *>(out + (size_t)r * ldo + h * kHeadDim + lane * 2) = o;
 }
 
-// Same merge, result written as a bf16 high plane and a bf16 low plane (value - high), the operand form of the
-// tensor-core projections.
-template <bool kCross>
-__global__ void __launch_bounds__(128)
-attn_combine_planes_kernel(const DecState *state, const int32_t *__restrict__ active_list,
-                           const float *__restrict__ partials, int n_heads, const int32_t *__restrict__ t_u,
-                           const int32_t *__restrict__ enc_len, int max_chunks, __nv_bfloat16 *__restrict__ out_hi,
-                           __nv_bfloat16 *__restrict__ out_lo, int ldo)
-{
-    const int rh = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    const int r = rh / n_heads, h = rh % n_heads;
-    if (r >= state->n_active) return;
-    const int u = active_list[r];
-    const int len = kCross ? enc_len[u] : t_u[u] + 1;
-    const int n_chunks = (len + kAttnChunk - 1) / kAttnChunk;
-    const float *src = partials + (size_t)rh * max_chunks * kPartialStride;
-    float m = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, src[(size_t)c * kPartialStride]);
-    float l = 0.f, a0 = 0.f, a1 = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
-        const float *p = src + (size_t)c * kPartialStride;
-        float w = expf(p[0] - m);
-        l = fmaf(p[1], w, l);
-        a0 = fmaf(p[2 + lane * 2], w, a0);
-        a1 = fmaf(p[3 + lane * 2], w, a1);
-    }
-    const float inv = 1.f / l;
-    const float o0 = a0 * inv, o1 = a1 * inv;
-    const __nv_bfloat16 h0 = __float2bfloat16_rn(o0), h1 = __float2bfloat16_rn(o1);
-    const size_t off = (size_t)r * ldo + h * kHeadDim + lane * 2;
-    *reinterpret_cast<__nv_bfloat162 *>(out_hi + off) = __halves2bfloat162(h0, h1);
-    *reinterpret_cast<__nv_bfloat162 *>(out_lo + off) =
-        __halves2bfloat162(__float2bfloat16_rn(o0 - __bfloat162float(h0)), __float2bfloat16_rn(o1 - __bfloat162float(h1)));
-}
-
 // LayerNorm whose result is written as bf16 high and low planes [row, d]; the same block also clears the fp32
 // rows that the following split-K projection accumulates into (zero_cols columns of zero_buf, if any).
 template <int kMaxPerThread>
@@ -739,29 +707,6 @@ __global__ void layernorm_planes_kernel(const DecState *state, const float *__re
         }
     }
     for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
-}
-
-// relu(hidden) as bf16 high and low planes [row, f]
-__global__ void relu_planes_kernel(const DecState *state, const float *__restrict__ hid, int f,
-                                   __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo)
-{
-    AED_TRACE_BEGIN(state, 5);
-    int r = blockIdx.y;
-    if (r >= state->n_active) return;
-    int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
-    if (i >= f) return;
-    float4 h = *reinterpret_cast<const float4 *>(hid + (size_t)r * f + i);
-    const float y[4] = {fmaxf(h.x, 0.f), fmaxf(h.y, 0.f), fmaxf(h.z, 0.f), fmaxf(h.w, 0.f)};
-    __nv_bfloat16 hi[4], lo[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        hi[j] = __float2bfloat16_rn(y[j]);
-        lo[j] = __float2bfloat16_rn(y[j] - __bfloat162float(hi[j]));
-    }
-    __nv_bfloat162 *ph = reinterpret_cast<__nv_bfloat162 *>(out_hi + (size_t)r * f + i);
-    __nv_bfloat162 *pl = reinterpret_cast<__nv_bfloat162 *>(out_lo + (size_t)r * f + i);
-    ph[0] = __halves2bfloat162(hi[0], hi[1]); ph[1] = __halves2bfloat162(hi[2], hi[3]);
-    pl[0] = __halves2bfloat162(lo[0], lo[1]); pl[1] = __halves2bfloat162(lo[2], lo[3]);
 }
 
 // ------------------------------------------------------------------------------------------------------------

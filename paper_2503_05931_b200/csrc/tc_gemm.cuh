@@ -9,9 +9,9 @@
 // 32*(w%4) .. +31) and run the epilogue.
 //
 // Two uses:
-//   * decode-step projections ("weights as A"): A = weight matrix [out_features, K], B = activations
-//     [rows, K] as a bf16 high plane and, optionally, a low (residual) plane accumulated into the same D, so
-//     that activations keep ~16 mantissa bits; split-K partials are added to an fp32 output with red.global.
+//   * vocabulary projection ("weights as A"): A = output matrix [vocab, K], B = the final LayerNorm output
+//     [rows, K] as a bf16 high plane and a low (residual) plane accumulated into the same D, so that
+//     activations keep ~16 mantissa bits; the greedy argmax is taken in the epilogue.
 //   * cross-K/V precompute ("frames as A"): A = packed encoder frames, B = [2d, d_enc] weights of a layer.
 //
 // Every wait on an mbarrier is bounded: on expiry the CTA raises the error word in the decode state, stops
@@ -124,7 +124,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-enum TcEpilogue { TC_EPI_ADD = 0, TC_EPI_LOGITS = 1, TC_EPI_CROSSKV = 2 };
+enum TcEpilogue { TC_EPI_LOGITS = 1, TC_EPI_CROSSKV = 2 };
 
 struct TcParams {
     int a_rows;          // valid rows of A (output features, or frames)
@@ -132,10 +132,7 @@ struct TcParams {
     int k_blocks;        // k-blocks over the whole K
     int use_lo;          // 1: accumulate the low activation plane as well
     int rows_fixed;      // >= 0: number of valid B rows; < 0: read it from the decode state
-    // TC_EPI_ADD: out[r * ldo + o] += D[o][r] (+ bias[o] from the CTA of k-split 0)
-    float *out;
-    int ldo;
-    const __nv_bfloat16 *bias;
+    const __nv_bfloat16 *bias;         // over the columns of D's first dimension (vocabulary / K-V features), may be null
     // TC_EPI_LOGITS
     float *logits_out;                 // [batch, vocab] by utterance or nullptr
     unsigned long long *keys;          // [rows]
@@ -251,18 +248,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int a_idx = a0 + quarter * 32 + lane;          // row of A this thread owns
             const bool a_ok = a_idx < p.a_rows;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-            if (EPI == TC_EPI_ADD) {
-                const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
-                for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + c0, v);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int r = row0 + c0 + j;
-                        if (a_ok && r < n_rows) atomicAdd(p.out + static_cast<size_t>(r) * p.ldo + a_idx, v[j] + bias);
-                    }
-                }
-            } else if (EPI == TC_EPI_LOGITS) {
+            if (EPI == TC_EPI_LOGITS) {
                 const float bias = (p.bias && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
                 for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
                     float v[16];

@@ -28,7 +28,8 @@ def _stale() -> bool:
 def build_trace() -> str:
     """Debug build with device-side start-time stamps in every step kernel (libaed_dec_trace.so)."""
     out = os.path.join(_HERE, "libaed_dec_trace.so")
-    subprocess.run([os.environ.get("NVCC", "nvcc")] + NVCC_FLAGS + ["-DAED_TRACE", "-o", out] + _sources(), check=True)
+    src = os.path.join(CSRC, "debug", "trace_exports.cu")
+    subprocess.run([os.environ.get("NVCC", "nvcc")] + NVCC_FLAGS + ["-DAED_TRACE", "-o", out, src], check=True)
     return out
 
 

@@ -17,7 +17,6 @@
 #include "step_kernels.cuh"
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
-#include "mega_step.cuh"
 
 using namespace aed;
 
@@ -51,8 +50,6 @@ struct Layout {
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
     size_t actd_hi, actd_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
-    size_t x1;                            // second buffer of the residual stream (persistent step kernel)
-    size_t mega_bars, mega_maps, mega_layers;   // arrival counters, weight tensor maps and per-layer arguments of that kernel
     size_t fold_layer_floats;
     int rows_cap;
 };
@@ -120,10 +117,6 @@ Layout make_layout(const aed_dec_config_t &c)
         L.fold_c = take(L.fold_layer_floats * c.n_layers * 4);
         L.ln_stats = take((size_t)3 * rows_bucket(c.max_batch) * 8);
         L.qc = take(B * d * 4);
-        L.x1 = take(B * d * 4);
-        L.mega_bars = take(((size_t)c.n_layers * mega::kStagesPerLayer + 1) * 4);
-        L.mega_maps = take((size_t)6 * c.n_layers * sizeof(CUtensorMap));
-        L.mega_layers = take((size_t)c.n_layers * sizeof(mega::LayerArgs));
     }
     L.total = off;
     return L;
@@ -162,9 +155,6 @@ struct aed_dec {
     CUtensorMap tc_src_x[5], tc_src_att[5], tc_src_hid[5];   // fp32 sources of the fused projections, per MMA N
     int tc_kvc_box = 0;                           // rows of the w_kv_c box = MMA N of the precompute
     bool use_tc = false;
-    // persistent step kernel (bf16 mode): one launch per step for steps of at most mega_rows rows
-    bool use_mega = false;
-    int mega_rows = 0, mega_slots = 0;
     int sm_count = 148;
     int tc_target_ctas = 128;
     bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
@@ -212,10 +202,10 @@ aed_status_t fail(aed_dec *d, aed_status_t code, const char *fmt, ...)
 
 enum KernelFamily { KF_BOOKKEEPING = 0, KF_EMBED, KF_LAYERNORM, KF_GEMM_QKV, KF_ATTN_SELF, KF_ATTN_COMBINE, KF_GEMM_O,
                     KF_GEMM_QC, KF_ATTN_CROSS, KF_GEMM_OC, KF_GEMM_FF1, KF_GEMM_FF2, KF_GEMM_VOCAB, KF_PRECOMPUTE,
-                    KF_STEP_LAYERS, KF_COUNT };
+                    KF_COUNT };
 const char *const kFamilyNames[KF_COUNT] = {"bookkeeping", "embed", "layernorm", "gemm_qkv", "attn_self", "attn_combine",
                                             "gemm_o", "gemm_qc", "attn_cross", "gemm_oc", "gemm_ff1", "gemm_ff2",
-                                            "gemm_vocab", "precompute_cross_kv", "step_layers"};
+                                            "gemm_vocab", "precompute_cross_kv"};
 
 // Records an event before and after the launches issued while it is alive (profiling mode only).
 struct ProfScope {
@@ -433,123 +423,6 @@ bool encode_map(CUtensorMap *map, const void *base, size_t rows, size_t cols, in
 
 constexpr int kTcSmemBudget = 200 * 1024;
 
-// ---- persistent step kernel (bf16 mode, small batches) ----------------------------------------------------------
-
-mega::MegaParams mega_params(const aed_dec *dec)
-{
-    const auto &c = dec->cfg;
-    const Layout &L = dec->lay;
-    mega::MegaParams p{};
-    p.n_layers = c.n_layers; p.d = c.d_model; p.n_heads = c.n_heads; p.d_ffn = c.d_ffn;
-    p.n_slots = dec->mega_slots;
-    p.self_capacity = c.max_dec_len; p.frame_capacity = c.max_total_enc_frames;
-    p.scale = 1.0f / sqrtf((float)kHeadDim); p.eps = c.ln_eps;
-    p.x0 = dec->at<float>(L.x); p.x1 = dec->at<float>(L.x1);
-    p.qkv = dec->at<float>(L.qkv); p.hid = dec->at<float>(L.hid);
-    p.stats1 = dec->at<float2>(L.ln_stats); p.stats3 = dec->at<float2>(L.ln_stats) + 2 * rows_bucket(c.max_batch);
-    p.row_info = dec->at<int4>(L.row_info);
-    p.state = dec->state();
-    p.bars = dec->at<int>(L.mega_bars);
-    p.maps = dec->at<CUtensorMap>(L.mega_maps);
-    p.layers = dec->at<mega::LayerArgs>(L.mega_layers);
-    return p;
-}
-
-// Decide whether the persistent step kernel can run on this device for this model, and stage what it reads.
-aed_status_t mega_setup(aed_dec *dec)
-{
-    typedef __nv_bfloat16 T;
-    const auto &c = dec->cfg;
-    const Layout &L = dec->lay;
-    const size_t d = c.d_model, F = c.d_ffn;
-    const char *v = getenv("AED_DEC_PERSISTENT");
-    if (v && v[0] == '0') return AED_OK;                  // A/B runs and the tests of the kernel chain at small batches
-    const int G = dec->sm_count;
-    if (d < 128 || d > 1024 || F < 128 || c.n_heads > G || G < mega::kMaxRows) return AED_OK;
-    // ring depth: what fits beside the fixed regions
-    int slots = mega::kMaxSlots;
-    while (slots > 4 && mega::smem_layout(slots).total + 1024 > kTcSmemBudget + 20 * 1024) --slots;
-    const int smem = mega::smem_layout(slots).total + 1024;
-    cudaError_t e = cudaFuncSetAttribute(mega::mega_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    int per_sm = 0;
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mega::mega_step_kernel, mega::kThreads, smem);
-    if (e != cudaSuccess) { (void)cudaGetLastError(); return AED_OK; }
-    if (per_sm < 1) return AED_OK;
-    std::vector<CUtensorMap> maps(6 * c.n_layers);
-    std::vector<mega::LayerArgs> layers(c.n_layers);
-    bool ok = true;
-    for (int l = 0; l < c.n_layers; ++l) {
-        const LayerWeights &w = dec->layers[l];
-        CUtensorMap *m = &maps[6 * l];
-        ok = ok && encode_map(m + 0, w.w_qkv, 3 * d, d, tc::kTileM) && encode_map(m + 1, w.w_o, d, d, tc::kTileM) &&
-             encode_map(m + 2, w.w_q_c, d, d, 64) && encode_map(m + 3, w.w_o_c, d, d, tc::kTileM) &&
-             encode_map(m + 4, w.w_ff1, F, d, tc::kTileM) && encode_map(m + 5, w.w_ff2, d, F, tc::kTileM);
-        const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
-        mega::LayerArgs &a = layers[l];
-        a.ln1_g = (const T *)w.ln1_g; a.ln2_g = (const T *)w.ln2_g; a.ln3_g = (const T *)w.ln3_g;
-        a.c1_qkv = fc; a.c2_qkv = fc + 3 * d; a.c1_qc = fc + 6 * d; a.c2_qc = fc + 7 * d; a.c1_ff = fc + 8 * d; a.c2_ff = fc + 8 * d + F;
-        a.b_o = (const T *)w.b_o; a.b_oc = (const T *)w.b_o_c; a.b_ff2 = (const T *)w.b_ff2;
-        a.self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
-        a.cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-    }
-    if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the persistent step kernel");
-    e = cudaMemcpyAsync(dec->ws + L.mega_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, dec->stream);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(dec->ws + L.mega_layers, layers.data(), layers.size() * sizeof(mega::LayerArgs), cudaMemcpyHostToDevice, dec->stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(dec->stream);      // the host vectors go away
-    if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "persistent step kernel set-up: %s", cudaGetErrorString(e));
-    dec->mega_slots = slots;
-    dec->mega_rows = std::min(mega::kMaxRows, (G / c.n_heads) * mega::kUnitRows);
-    dec->use_mega = true;
-    return AED_OK;
-}
-
-aed_status_t launch_ln_planes(aed_dec *dec, int rows_ub, const float *x, const void *g, const void *b, float *zero_buf, int zero_cols);
-aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p);
-
-// One step through the persistent kernel: embedding, all layers in one cooperative launch, final LayerNorm,
-// vocabulary projection.
-aed_status_t forward_step_mega(aed_dec *dec, int rows_ub, const int32_t *tokens, float *logits_out)
-{
-    typedef __nv_bfloat16 T;
-    const auto &c = dec->cfg;
-    const Layout &L = dec->lay;
-    const int d = c.d_model, V = c.vocab;
-    float *x0 = dec->at<float>(L.x), *x1 = dec->at<float>(L.x1);
-    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
-    {
-        ProfScope ps(dec, KF_EMBED);
-        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x0, dec->at<float>(L.qkv), 3 * d);
-        AED_LAUNCHED(dec);
-    }
-    {
-        ProfScope ps(dec, KF_STEP_LAYERS);
-        const mega::MegaParams p = mega_params(dec);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(dec->sm_count);
-        cfg.blockDim = dim3(mega::kThreads);
-        cfg.dynamicSmemBytes = (size_t)mega::smem_layout(dec->mega_slots).total + 1024;
-        cfg.stream = dec->stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeCooperative;        // every block resident at once: they wait on one another
-        attr[0].val.cooperative = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, mega::mega_step_kernel, p);
-        if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "persistent step launch: %s", cudaGetErrorString(e));
-        AED_LAUNCHED(dec);
-    }
-    AED_TRY(launch_ln_planes(dec, rows_ub, (c.n_layers & 1) ? x1 : x0, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
-    tc::TcParams tp{};
-    tp.bias = (const T *)dec->b_out;
-    tp.logits_out = logits_out;
-    tp.keys = dec->at<unsigned long long>(L.keys);
-    tp.active_list = active_list;
-    AED_TRY(launch_vocab_gemm(dec, rows_ub, tp));
-    return AED_OK;
-}
-
 aed_status_t tc_setup(aed_dec *dec)
 {
     const auto &c = dec->cfg;
@@ -613,7 +486,7 @@ aed_status_t tc_setup(aed_dec *dec)
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
     if (ctas && atoi(ctas) > 0) { dec->tc_target_ctas = atoi(ctas); dec->tc_target_fixed = true; }
     dec->use_tc = true;
-    return mega_setup(dec);
+    return AED_OK;
 }
 
 // MMA N for a step with at most rows_ub rows: the smallest of 16, 32, ..., 256 that covers them (or 256).
@@ -866,9 +739,7 @@ aed_status_t launch_build_active(aed_dec *dec, const uint8_t *mask)
                                                      dec->at<int32_t>(L.active_list), dec->state(),
                                                      dec->at<int32_t>(L.enc_len), dec->at<int32_t>(L.enc_off),
                                                      dec->at<int4>(L.row_info), rows_bucket(dec->cfg.max_batch),
-                                                     dec->at<int32_t>(L.len_order),
-                                                     dec->use_mega ? dec->at<int>(L.mega_bars) : nullptr,
-                                                     dec->use_mega ? dec->cfg.n_layers * mega::kStagesPerLayer + 1 : 0);
+                                                     dec->at<int32_t>(L.len_order));
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -1028,9 +899,8 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_build_active(dec, active));
     const int rows_ub = dec->batch;
     const int self_len_ub = dec->steps_issued + 1 < dec->cfg.max_dec_len ? dec->steps_issued + 1 : dec->cfg.max_dec_len;
-    aed_status_t s = (dec->use_mega && rows_ub <= dec->mega_rows) ? forward_step_mega(dec, rows_ub, tokens_in, logits_out)
-                     : dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out)
-                                   : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
+    aed_status_t s = dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out)
+                                 : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
     if (s != AED_OK) return s;
     AED_TRY(launch_finish(dec, rows_ub, next_out, 0, nullptr, nullptr));
     dec->steps_issued++;
@@ -1102,9 +972,8 @@ aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int
     if (self_len_ub > dec->cfg.max_dec_len) self_len_ub = dec->cfg.max_dec_len;
     AED_TRY(launch_build_active(dec, nullptr));
     const int32_t *tok = dec->at<int32_t>(L.cur_tok);
-    aed_status_t st = (dec->use_mega && rows_ub <= dec->mega_rows) ? forward_step_mega(dec, rows_ub, tok, nullptr)
-                      : dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr)
-                                    : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
+    aed_status_t st = dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr)
+                                  : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
     if (st != AED_OK) return st;
     return launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens);
 }
@@ -1163,10 +1032,7 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
         const int rows_ub = alive[s];
         if (dec->use_graphs && !dec->profiling) {
             // grids are sized for the bucket; kernels leave rows beyond the device-side row count alone
-            // (the persistent kernel reads the row count and every length on the device: one graph serves all its steps)
-            const bool mega_step = dec->use_mega && rows_ub <= dec->mega_rows;
-            const int rows_b = mega_step ? dec->mega_rows : rows_bucket(rows_ub);
-            const int chunks = mega_step ? 0 : (s + 1 + kAttnChunk - 1) / kAttnChunk;
+            const int rows_b = rows_bucket(rows_ub), chunks = (s + 1 + kAttnChunk - 1) / kAttnChunk;
             const aed_dec::GraphKey key(rows_b, chunks, tokens_out, out_lens);
             auto it = dec->graphs.find(key);
             if (it == dec->graphs.end()) {

@@ -19,8 +19,7 @@ __global__ void build_active_kernel(const uint8_t *__restrict__ mask, const int3
                                     const int32_t *__restrict__ t_u, int max_dec_len,
                                     int32_t *__restrict__ active_list, DecState *state,
                                     const int32_t *__restrict__ enc_len, const int32_t *__restrict__ enc_off,
-                                    int4 *__restrict__ row_info, int row_slots, const int32_t *__restrict__ order,
-                                    int *__restrict__ step_counters, int n_step_counters)
+                                    int4 *__restrict__ row_info, int row_slots, const int32_t *__restrict__ order)
 {
     AED_TRACE_BEGIN(state, 1);
     __shared__ int warp_counts[32];
@@ -58,8 +57,6 @@ __global__ void build_active_kernel(const uint8_t *__restrict__ mask, const int3
         __syncthreads();
     }
     if (threadIdx.x == 0) { state->n_active = base; state->grid_sync = 0; }
-    // arrival counters (and the abort word) of the persistent step kernel start every step at zero
-    for (int i = threadIdx.x; i < n_step_counters; i += blockDim.x) step_counters[i] = 0;
     for (int r = base + threadIdx.x; r < row_slots; r += blockDim.x) row_info[r] = make_int4(-1, 0, 0, 0);
 }
 
@@ -472,30 +469,35 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             }
         }
     }
+    // The LayerNorm-fold constants of this block's columns are static as well (read once per step and layer, so
+    // they come from DRAM): requested here, before the dependency wait.
+    const int new_chunk = (len - 1) / kFusedChunk;
+    const bool owns_new = kAppend && !kCross && warp == new_chunk % n_warps;
+    const int d_model = n_heads * kHeadDim;
+    const int qcol = h * kHeadDim + dg * 8;
+    float qc1[8], qc2[8], kc1[8], kc2[8], vc1[8], vc2[8];
+    if (ln_stats) {
+        load8(ln_c1 + qcol, qc1); load8(ln_c2 + qcol, qc2);
+        if (owns_new) {
+            load8(ln_c1 + d_model + qcol, kc1); load8(ln_c2 + d_model + qcol, kc2);
+            load8(ln_c1 + 2 * d_model + qcol, vc1); load8(ln_c2 + 2 * d_model + qcol, vc2);
+        }
+    }
     AED_TRACE_RESERVE(tcur, state, (threadIdx.x == 0 && blockIdx.x == 0) ? 4u : 0u);
     AED_TRACE_PUT(state, tcur, 8 + (kCross ? 1 : 0));      // resident, first chunk requested
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     AED_TRACE_PUT(state, tcur, 3);                          // dependency resolved
     // Everything this block needs from earlier kernels is requested in one round: statistics, query, and (in the
-    // warp that owns the new position) the new key and value, with the LayerNorm-fold constants of their columns.
-    // When the projection ran on gamma*x, its raw output y becomes rstd*(y - mean*c1) + c2 here.
-    const int new_chunk = (len - 1) / kFusedChunk;
-    const bool owns_new = kAppend && !kCross && warp == new_chunk % n_warps;
-    const int d_model = n_heads * kHeadDim;
-    const int qcol = h * kHeadDim + dg * 8;
+    // warp that owns the new position) the new key and value.  When the projection ran on gamma*x, its raw output
+    // y becomes rstd*(y - mean*c1) + c2 here.
     float2 st = make_float2(0.f, 1.f);
-    float qv[8], qc1[8], qc2[8], kn[8], vn[8], kc1[8], kc2[8], vc1[8], vc2[8];
+    float qv[8], kn[8], vn[8];
     if (ln_stats) st = ln_stats[r];
     load8(q + (size_t)r * ldq + qcol, qv);
-    if (ln_stats) { load8(ln_c1 + qcol, qc1); load8(ln_c2 + qcol, qc2); }
     if (owns_new) {
         load8(q + (size_t)r * ldq + d_model + qcol, kn);
         load8(q + (size_t)r * ldq + 2 * d_model + qcol, vn);
-        if (ln_stats) {
-            load8(ln_c1 + d_model + qcol, kc1); load8(ln_c2 + d_model + qcol, kc2);
-            load8(ln_c1 + 2 * d_model + qcol, vc1); load8(ln_c2 + 2 * d_model + qcol, vc2);
-        }
     }
     if (ln_stats) {
 #pragma unroll

@@ -54,9 +54,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false if the phase did not complete in time or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+// (The polling loop is kept out of line: the common case is that the phase has already completed.)
+__device__ __noinline__ bool mbar_wait_poll(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
     return bounded_poll([&] { return mbar_try_wait(bar, parity); }, [] { return clock64(); }, kWaitCycles, abort_flag);
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_poll(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c_inner, int c_outer, uint64_t *bar)

@@ -21,14 +21,6 @@ def _binding():
     return binding
 
 
-@pytest.fixture(params=["persistent", "chain"])
-def small_batch_path(request, monkeypatch):
-    """bf16 steps of at most 64 rows run in the persistent step kernel by default; AED_DEC_PERSISTENT=0 (read when a
-    handle is created) sends them through the kernel-per-projection chain that larger steps always take."""
-    monkeypatch.setenv("AED_DEC_PERSISTENT", "1" if request.param == "persistent" else "0")
-    return request.param
-
-
 def _run_both(w, rows=None, need_tokens=True, label=""):
     """Teacher-forced logits and argmax at every step (this comparison carries the weight: it never stops at a
     near-tie), then the free-running greedy decode up to each utterance's first near-tie.  ``need_tokens``: demand
@@ -69,7 +61,7 @@ def test_ragged_multi_tile(dtype):
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("shape", [((1,), (1,)), ((1,), (5,)), ((7,), (1,)), ((3, 1, 2), (2, 4, 1))])
-def test_degenerate_shapes(dtype, shape, small_batch_path):
+def test_degenerate_shapes(dtype, shape):
     enc_lens, dec_lens = shape
     w = wl.make_custom(SMALL, list(enc_lens), list(dec_lens), dtype=dtype, seed=5)
     _run_both(w, need_tokens=False)         # one or two tokens in all: the first may already be a near-tie
@@ -125,7 +117,7 @@ def _eos_case(dtype):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-def test_eos_stops_an_utterance(dtype, small_batch_path):
+def test_eos_stops_an_utterance(dtype):
     """With eos enabled an utterance retires right after emitting it (the token is stored and counted) while the
     others run on.  Expectation: the CPU checker's decode with the same end-of-sequence id."""
     b = _binding()
@@ -147,7 +139,7 @@ def test_eos_stops_an_utterance(dtype, small_batch_path):
     assert stopped_early > 0
 
 
-def test_handle_reuse_across_batch_sizes(small_batch_path):
+def test_handle_reuse_across_batch_sizes():
     """One handle and one pair of output buffers decode batches of 12, 7 and 12 utterances in turn (the step graphs
     recorded for the first batch are replayed for the others): every batch against the checker."""
     import torch
@@ -195,19 +187,17 @@ LN_CASES = {
 @pytest.mark.parametrize("offset", [0.0, 4.0])
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("case", ["small", "mid", "wide"])
-def test_layernorm_parameters_output_bias_and_mean_offset(case, dtype, offset, small_batch_path):
+def test_layernorm_parameters_output_bias_and_mean_offset(case, dtype, offset):
     """LayerNorm gains and shifts drawn around 1 and 0 (N(1, 0.3), N(0, 0.3)), an output-projection bias, and
     (offset 4) an embedding table shifted by a constant so that the residual stream's mean dwarfs its spread:
     the folded LayerNorm rstd * ((gamma * x) W^T - mean * c1) + c2 has to survive that cancellation."""
-    if dtype == "fp32" and small_batch_path == "chain":
-        pytest.skip("the switch only exists in bf16 mode")
     model, enc_lens, dec_lens = LN_CASES[case]
     w = wl.make_custom(model, enc_lens, dec_lens, dtype=dtype, seed=91, ln_std=0.3, out_bias_std=0.3,
                        embed_offset=offset)
     _run_both(w, need_tokens=False, label=f"ln-{case}-offset{offset:g}")
 
 
-def test_long_rows_bf16(small_batch_path):
+def test_long_rows_bf16():
     """Decodes far beyond 128 cached positions (the self-attention block loops over its warps' chunks more than
     once) beside a short one, with encoder outputs of up to 500 frames at a batch small enough for the
     cross-attention variant that overlaps its loads: every step of every row against the checker."""
@@ -319,7 +309,7 @@ def test_config4_shape_sampled_rows():
     _run_both(w, rows=rows)
 
 
-def test_config2_shape_sampled_rows(small_batch_path):
+def test_config2_shape_sampled_rows():
     """24-layer d=1024 bf16 decoder at batch 64 (the benchmark configuration, on both launch paths): a sample of
     utterances is decoded one by one by the checker and compared with the GPU's full-batch run."""
     w = wl.make_workload("cfg2")
@@ -331,16 +321,16 @@ def test_config2_shape_sampled_rows(small_batch_path):
     _run_both(w, rows=rows)
 
 
-# ---- persistent step kernel (bf16, at most 64 rows per step) --------------------------------------------------------
+# ---- small batches: every row-tile width of the step projections ------------------------------------------------------
 
-WIDE_A = dict(n_layers=2, d_model=512, n_heads=8, d_ffn=1024, vocab=600, d_enc=256)      # 18 row blocks per head
-WIDE_B = dict(n_layers=1, d_model=1024, n_heads=16, d_ffn=768, vocab=520, d_enc=128)     # 9 row blocks per head
+WIDE_A = dict(n_layers=2, d_model=512, n_heads=8, d_ffn=1024, vocab=600, d_enc=256)
+WIDE_B = dict(n_layers=1, d_model=1024, n_heads=16, d_ffn=768, vocab=520, d_enc=128)
 ODD = dict(n_layers=3, d_model=192, n_heads=3, d_ffn=320, vocab=333, d_enc=64)           # 3 k-blocks, partial feature tiles
 
 
 @pytest.mark.parametrize("batch", [1, 7, 16, 17, 40, 64])
-def test_small_batch_row_counts(batch, small_batch_path):
-    """One to four 16-row MMA tiles with partly filled tiles, units holding 1 to 8 rows, ragged encoder lengths from
+def test_small_batch_row_counts(batch):
+    """Row-tile widths 16, 32 and 64 of the step projections with partly filled tiles, ragged encoder lengths from
     1 frame to several attention chunks, and rows retiring at different steps."""
     rng = np.random.default_rng(900 + batch)
     enc_lens = rng.integers(1, 150, size=batch)
@@ -352,38 +342,12 @@ def test_small_batch_row_counts(batch, small_batch_path):
 
 
 @pytest.mark.parametrize("model", ["wide_b", "odd"])
-def test_small_batch_model_shapes(model, small_batch_path):
-    """d_model 1024 with 16 heads (eight rows per unit at 64 rows) and a model whose widths are not multiples of
-    128 (an odd number of k-blocks, feature tiles that end inside a tile)."""
+def test_small_batch_model_shapes(model):
+    """d_model 1024 with 16 heads at 64 rows, and a model whose widths are not multiples of 128 (an odd number of
+    k-blocks, feature tiles that end inside a tile, a cross-K/V feature count that is not a multiple of 256)."""
     rng = np.random.default_rng(31)
     batch = 64 if model == "wide_b" else 23
     m = WIDE_B if model == "wide_b" else ODD
     w = wl.make_custom(m, rng.integers(1, 200, size=batch), rng.integers(1, 20, size=batch), dtype="bf16", seed=77,
                        out_std=0.1, ln_std=0.2, out_bias_std=0.1)
     _run_both(w, rows=[0, 5, batch // 2, batch - 1])
-
-
-def test_persistent_kernel_matches_kernel_chain(monkeypatch):
-    """Both launch paths compute the same step: their logits agree far inside the tolerance against the checker
-    (both keep two bf16 planes of every activation)."""
-    import torch
-    b = _binding()
-    rng = np.random.default_rng(5)
-    batch = 33
-    w = wl.make_custom(WIDE_A, rng.integers(1, 120, size=batch), [6] * batch, dtype="bf16", seed=9)
-    outs = []
-    for persistent in ("1", "0"):
-        monkeypatch.setenv("AED_DEC_PERSISTENT", persistent)
-        dec = b.decoder_for_workload(w)
-        dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
-        logits = torch.zeros((batch, WIDE_A["vocab"]), dtype=torch.float32, device="cuda:0")
-        toks = torch.full((batch,), 1, dtype=torch.int32, device="cuda:0")
-        rec = []
-        for t in range(6):
-            dec.step(toks, None, logits, None)
-            toks.fill_(2 + t)
-            rec.append(logits.cpu().numpy().copy())
-        dec.sync_status()
-        dec.close()
-        outs.append(np.stack(rec))
-    assert np.max(np.abs(outs[0] - outs[1])) < 2e-3

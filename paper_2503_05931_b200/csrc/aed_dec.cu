@@ -17,6 +17,7 @@
 #include "step_kernels.cuh"
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
+#include "crosskv_gemm.cuh"
 
 using namespace aed;
 
@@ -50,6 +51,7 @@ struct Layout {
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
     size_t actd_hi, actd_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
+    size_t ckv_maps, ckv_bias;            // per-layer tensor maps and bias pointers of the cross-K/V weights
     size_t fold_layer_floats;
     int rows_cap;
 };
@@ -117,6 +119,8 @@ Layout make_layout(const aed_dec_config_t &c)
         L.fold_c = take(L.fold_layer_floats * c.n_layers * 4);
         L.ln_stats = take((size_t)3 * rows_bucket(c.max_batch) * 8);
         L.qc = take(B * d * 4);
+        L.ckv_maps = take((size_t)c.n_layers * sizeof(CUtensorMap));
+        L.ckv_bias = take((size_t)c.n_layers * sizeof(void *));
     }
     L.total = off;
     return L;
@@ -148,12 +152,11 @@ struct aed_dec {
     std::vector<int> prof_family;                  // family of each recorded launch
     size_t prof_used = 0;
     // bf16 mode: TMA descriptors of the weight matrices and of the activation planes (one per MMA N in 16..256)
-    struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2, kvc; };
+    struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
     CUtensorMap tc_actd[5][2];                    // [log2(N/16)][plane]: final LayerNorm output, operand of the vocabulary projection
     CUtensorMap tc_src_x[5], tc_src_att[5], tc_src_hid[5];   // fp32 sources of the fused projections, per MMA N
-    int tc_kvc_box = 0;                           // rows of the w_kv_c box = MMA N of the precompute
     bool use_tc = false;
     int sm_count = 148;
     int tc_target_ctas = 128;
@@ -431,14 +434,16 @@ aed_status_t tc_setup(aed_dec *dec)
     if (!encode_tiled_fn()) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     bool ok = true;
     dec->tc_layers.resize(c.n_layers);
-    dec->tc_kvc_box = 2 * d >= 256 ? 256 : (int)(2 * d);
+    std::vector<CUtensorMap> kvc_maps(c.n_layers);
+    std::vector<const void *> kvc_bias(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerWeights &w = dec->layers[l];
         aed_dec::TcLayerMaps &m = dec->tc_layers[l];
         ok = ok && encode_map(&m.qkv, w.w_qkv, 3 * d, d, tc::kTileM) && encode_map(&m.o, w.w_o, d, d, tc::kTileM) &&
              encode_map(&m.qc, w.w_q_c, d, d, tc::kTileM) && encode_map(&m.oc, w.w_o_c, d, d, tc::kTileM) &&
              encode_map(&m.ff1, w.w_ff1, F, d, tc::kTileM) && encode_map(&m.ff2, w.w_ff2, d, F, tc::kTileM) &&
-             encode_map(&m.kvc, w.w_kv_c, 2 * d, c.d_enc, dec->tc_kvc_box);
+             encode_map(&kvc_maps[l], w.w_kv_c, 2 * d, c.d_enc, ckv::kTileN);
+        kvc_bias[l] = w.b_kv_c;
     }
     ok = ok && encode_map(&dec->tc_w_out, dec->w_out, c.vocab, d, tc::kTileM);
     for (int i = 0; i < 5; ++i) {
@@ -452,7 +457,11 @@ aed_status_t tc_setup(aed_dec *dec)
     if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed (are all weight tensors 16-byte aligned?)");
     const int smem = kTcSmemBudget + 1024;
     cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_CROSSKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv::crosskv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ckv::kStages * ckv::kStageBytes + 1024);
+    // tensor maps and bias pointers of the cross-K/V weights: read by the precompute kernel from the workspace
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dec->ws + L.ckv_maps, kvc_maps.data(), kvc_maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, dec->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dec->ws + L.ckv_bias, kvc_bias.data(), kvc_bias.size() * sizeof(void *), cudaMemcpyHostToDevice, dec->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(dec->stream);       // the host vectors go away
     int dev = 0, sms = 0;
     if (e == cudaSuccess) e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -515,10 +524,13 @@ aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p)
     int stages = kTcSmemBudget / stage_bytes;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     if (stages > k_blocks) stages = k_blocks;
+    // every ring stage belongs to one issuing thread: stages is a multiple of the number of producers
+    const int producers = stages >= tc::kProducerWarps ? tc::kProducerWarps : stages;
+    stages -= stages % producers;
     const CUtensorMap *acts = dec->tc_actd[ni];
     dim3 grid(m_tiles, 1, row_tiles);
     tc::tc_gemm_kernel<tc::TC_EPI_LOGITS><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
-        dec->tc_w_out, acts[0], acts[1], p, stages);
+        dec->tc_w_out, acts[0], acts[1], p, stages, producers);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -677,7 +689,7 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
     return AED_OK;
 }
 
-// Cross K/V of every layer on tensor cores: D[frame, feature] = enc[frame, :] . w_kv_c[feature, :]
+// Cross K/V of every layer on tensor cores, one persistent launch: D[frame, feature] = enc[frame, :] . w_kv_c[feature, :]
 aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
 {
     typedef __nv_bfloat16 T;
@@ -687,29 +699,21 @@ aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
     CUtensorMap map_enc;
     if (!encode_map(&map_enc, enc_packed, dec->total_frames, c.d_enc, tc::kTileM))
         return fail(dec, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the encoder states");
-    tc::TcParams p{};
-    p.a_rows = dec->total_frames;
-    p.n_tile = dec->tc_kvc_box;
-    p.k_blocks = c.d_enc / tc::kBlockK;
-    p.use_lo = 0;
-    p.rows_fixed = 0;
+    ckv::CkvParams p{};
+    p.total_frames = dec->total_frames;
     p.frame_capacity = c.max_total_enc_frames;
-    p.d_model = c.d_model;
-    p.n_heads = c.n_heads;
+    p.d_model = c.d_model; p.n_heads = c.n_heads; p.d_enc = c.d_enc;
+    p.n_layers = c.n_layers;
+    p.store = dec->at<T>(L.cross_store);
+    p.layer_elems = L.cross_layer_elems;
+    p.bias = dec->at<const T *>(L.ckv_bias);
     p.state = dec->state();
-    const int stage_bytes = tc::kATileBytes + p.n_tile * tc::kBlockK * 2;
-    int stages = kTcSmemBudget / stage_bytes;
-    if (stages > tc::kMaxStages) stages = tc::kMaxStages;
-    if (stages > p.k_blocks) stages = p.k_blocks;
-    dim3 grid((dec->total_frames + tc::kTileM - 1) / tc::kTileM, 1, (2 * c.d_model + p.n_tile - 1) / p.n_tile);
-    for (int l = 0; l < c.n_layers; ++l) {
-        ProfScope ps(dec, KF_PRECOMPUTE);
-        p.cross_store = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-        p.bias = (const T *)dec->layers[l].b_kv_c;
-        tc::tc_gemm_kernel<tc::TC_EPI_CROSSKV><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
-            map_enc, dec->tc_layers[l].kvc, dec->tc_layers[l].kvc, p, stages);
-        AED_LAUNCHED(dec);
-    }
+    const long long tiles = (long long)((dec->total_frames + tc::kTileM - 1) / tc::kTileM) * c.n_layers *
+                            ((2 * c.d_model + ckv::kTileN - 1) / ckv::kTileN);
+    ProfScope ps(dec, KF_PRECOMPUTE);
+    ckv::crosskv_gemm_kernel<<<(unsigned)std::min<long long>(tiles, dec->sm_count), ckv::kCkvThreads, ckv::kStages * ckv::kStageBytes + 1024, dec->stream>>>(
+        map_enc, dec->at<CUtensorMap>(L.ckv_maps), p);
+    AED_LAUNCHED(dec);
     return AED_OK;
 }
 

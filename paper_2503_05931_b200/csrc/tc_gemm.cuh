@@ -4,9 +4,10 @@
 //
 // Both operands are K-major bf16 in global memory and arrive in shared memory through
 // cp.async.bulk.tensor (no multicast) with the 128-byte swizzle the MMA descriptors name.
-// One CTA = one (128-row tile of A, N-row tile of B, k-split).  Warp roles: warp 0 issues TMA, warp 1 owns
-// the TMEM allocation and issues the MMAs, warps 2..5 drain the accumulator (warp w reads TMEM lanes
-// 32*(w%4) .. +31) and run the epilogue.
+// One CTA = one (128-row tile of A, N-row tile of B, k-split).  Warp roles: warps 0..3 issue TMA (a thread's
+// copies complete one after the other, about a third of a microsecond each, so the k-blocks are shared out round
+// robin over four issuing threads), warp 4 owns the TMEM allocation and issues the MMAs, warps 5..8 drain the
+// accumulator (warp w reads TMEM lanes 32*(w%4) .. +31) and run the epilogue.
 //
 // Two uses:
 //   * vocabulary projection ("weights as A"): A = output matrix [vocab, K], B = the final LayerNorm output
@@ -29,7 +30,8 @@ constexpr int kBlockK = 64;                    // bf16 elements per k-block = on
 constexpr int kTileM = 128;
 constexpr int kATileBytes = kTileM * kBlockK * 2;
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 192;
+constexpr int kThreads = 288;                    // 4 producer warps, 1 MMA warp, 4 epilogue warps
+constexpr int kProducerWarps = 4;
 constexpr long long kWaitCycles = 2000000000ll;   // about a second at B200 clocks
 constexpr int kErrTimeout = 2;
 
@@ -130,7 +132,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-enum TcEpilogue { TC_EPI_LOGITS = 1, TC_EPI_CROSSKV = 2 };
+enum TcEpilogue { TC_EPI_LOGITS = 1 };
 
 struct TcParams {
     int a_rows;          // valid rows of A (output features, or frames)
@@ -143,9 +145,6 @@ struct TcParams {
     float *logits_out;                 // [batch, vocab] by utterance or nullptr
     unsigned long long *keys;          // [rows]
     const int32_t *active_list;
-    // TC_EPI_CROSSKV: D[frame][feature] -> store [2][H][frame_capacity][64]; bias over features
-    __nv_bfloat16 *cross_store;
-    int frame_capacity, d_model, n_heads;
     DecState *state;
 };
 
@@ -153,8 +152,10 @@ struct TcParams {
 template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_b_lo, TcParams p, int stages)
+               const __grid_constant__ CUtensorMap map_b_lo, TcParams p, int stages, int producers)
 {
+    // `stages` is a multiple of `producers` (1..kProducerWarps): every ring stage is refilled by one thread only, so
+    // a producer is never more than one phase ahead of the barrier it waits on (a parity wait cannot tell more).
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t bar_full[kMaxStages];
     __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
@@ -167,7 +168,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int row0 = blockIdx.z * p.n_tile;
     // Only row tiles after the first can be empty; the first one skips this read so that set-up and the first
     // loads do not wait on it (the epilogue reads the row count when it needs it).
-    if (EPI != TC_EPI_CROSSKV && blockIdx.z > 0 && row0 >= (p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active)) return;
+    if (blockIdx.z > 0 && row0 >= (p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active)) return;
     const int a0 = blockIdx.x * kTileM;
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
@@ -187,20 +188,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(&tmem_slot, tmem_cols);
+    if (warp == kProducerWarps) tmem_alloc(&tmem_slot, tmem_cols);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     if (threadIdx.x == 0) AED_TRACE_MARK(p.state, 32);      // set-up done
 
-    if (warp == 0) {
-        if (lane == 0) {
+    if (warp < kProducerWarps) {
+        if (lane == 0 && warp < producers) {
             prefetch_tensormap(&map_a);
             prefetch_tensormap(&map_b);
             if (p.use_lo) prefetch_tensormap(&map_b_lo);
             int issued = 0;
-            for (int i = 0; i < n_kb; ++i) {
+            for (int i = warp; i < n_kb; i += producers) {
                 const int s = i % stages;
                 if (i >= stages && !mbar_wait(&bar_empty[s], ((i / stages) - 1) & 1, &abort_flag)) break;
                 uint8_t *st = tiles + static_cast<size_t>(s) * stage_bytes;
@@ -211,15 +212,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (p.use_lo) tma_load_2d(st + kATileBytes + b_bytes, &map_b_lo, kc, row0, &bar_full[s]);
                 issued = i + 1;
             }
-            if (abort_flag) {
-                // give copies that are still in flight a bounded chance to land before the CTA's memory goes away
-                for (int i = (issued > stages ? issued - stages : 0); i < issued; ++i) {
-                    const long long start = clock64();
-                    while (!mbar_try_wait(&bar_full[i % stages], (i / stages) & 1) && clock64() - start < kWaitCycles / 8) {}
-                }
+            if (abort_flag && issued > 0) {
+                // give this thread's last copies a bounded chance to land before the CTA's memory goes away
+                const int i = issued - 1;
+                const long long start = clock64();
+                while (!mbar_try_wait(&bar_full[i % stages], (i / stages) & 1) && clock64() - start < kWaitCycles / 8) {}
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == kProducerWarps) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(p.n_tile);
             bool ok = true;
@@ -249,7 +249,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int n_rows = p.rows_fixed >= 0 ? p.rows_fixed : p.state->n_active;
         const bool ok = mbar_wait(&bar_done, 0, &abort_flag);
         tc_fence_after_sync();
-        if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 34);  // accumulator complete
+        if (threadIdx.x == (kProducerWarps + 1) * 32) AED_TRACE_MARK(p.state, 34);  // accumulator complete
         if (ok) {
             const int a_idx = a0 + quarter * 32 + lane;          // row of A this thread owns
             const bool a_ok = a_idx < p.a_rows;
@@ -275,33 +275,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (lane == 0 && key != 0ull) atomicMax(p.keys + r, key);
                     }
                 }
-            } else {   // TC_EPI_CROSSKV: this thread owns frame a_idx; columns are features row0 + c
-                for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + c0, v);
-                    const int o = row0 + c0;                         // 16 consecutive features inside one head
-                    if (!a_ok || o >= 2 * p.d_model) continue;
-                    const int kv = o / p.d_model, c = o % p.d_model, h = c / kHeadDim, e = c % kHeadDim;
-                    uint32_t packed[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float lo = v[2 * j] + (p.bias ? to_f32(p.bias[o + 2 * j]) : 0.f);
-                        const float hi = v[2 * j + 1] + (p.bias ? to_f32(p.bias[o + 2 * j + 1]) : 0.f);
-                        __nv_bfloat162 pair = __floats2bfloat162_rn(lo, hi);
-                        packed[j] = *reinterpret_cast<uint32_t *>(&pair);
-                    }
-                    __nv_bfloat16 *dst = p.cross_store +
-                        ((static_cast<size_t>(kv) * p.n_heads + h) * p.frame_capacity + a_idx) * kHeadDim + e;
-                    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    reinterpret_cast<uint4 *>(dst)[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
-                }
             }
         }
     }
-    if (threadIdx.x == 64) AED_TRACE_MARK(p.state, 35);      // epilogue issued
+    if (threadIdx.x == (kProducerWarps + 1) * 32) AED_TRACE_MARK(p.state, 35);      // epilogue issued
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kProducerWarps) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, tmem_cols);
     }

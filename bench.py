@@ -235,8 +235,16 @@ def run_stream(args):
     w = wl.make_workload("cfg5")
     peaks = load_peaks()
     rng = np.random.default_rng(5)
+    # the paper's configuration: 30 duration bins of equal cumulative duration x 2 token sub-bins, estimated on a
+    # separate sample of the same law, flexible allocation (nothing that fits any bucket is dropped)
+    _, est_enc, est_dec = wl.draw_lengths(np.random.default_rng(wl.BASE_SEED + 500), 20000, "lognormal")
+    dur_bounds, tok_bounds = bucketing.estimate_bins_2d(est_enc, est_dec, 30, 2)
+    sizes = bucketing.bucket_batch_sizes(dur_bounds, tok_bounds)
+    paper_batches, dropped = bucketing.bucket_batches(w.enc_lens, w.dec_lens, dur_bounds, tok_bounds, sizes, "flexible")
+    paper_batches += [dropped[i:i + 128] for i in range(0, len(dropped), 128)]      # every arm decodes all utterances
     arms = {"random128": bucketing.random_batches(w.batch, 128, rng),
-            "bucketed8x4": bucketing.bucket_batches_2d(w.enc_lens, w.dec_lens)}
+            "bucketed8x4": bucketing.bucket_batches_2d(w.enc_lens, w.dec_lens),
+            "bucketed30x2": paper_batches}
     all_batches = [b for bs in arms.values() for b in bs]
     dec = binding.Decoder(w.model, w.weights, w.dtype, max_batch=max(len(b) for b in all_batches),
                           max_total_enc_frames=max(int(w.enc_lens[b].sum()) for b in all_batches),

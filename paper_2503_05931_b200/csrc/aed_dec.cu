@@ -18,7 +18,6 @@
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
 #include "crosskv_gemm.cuh"
-#include "attn_stream.cuh"
 
 using namespace aed;
 
@@ -164,7 +163,6 @@ struct aed_dec {
     bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
     bool use_pdl = true;
     bool attn_pipe = true;
-    int attn_stream_rows = 128;           // steps with more rows use the streaming attention kernel
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
     struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -327,37 +325,6 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     return AED_OK;
 }
 
-// Attention for steps with many rows: persistent blocks that stream the K/V runs through shared memory.
-template <bool kCross>
-aed_status_t launch_attention_stream(aed_dec *dec, int rows_ub, const float *q, int ldq, __nv_bfloat16 *cache, int seq_capacity,
-                                     float *out, const float2 *ln_stats, const float *ln_c1, const float *ln_c2, bool pdl)
-{
-    ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
-    as::AttnStreamParams p{};
-    p.state = dec->state(); p.err_state = dec->state();
-    p.row_info = dec->at<int4>(dec->lay.row_info);
-    p.q = q; p.ldq = ldq;
-    p.cache = cache;
-    p.n_heads = dec->cfg.n_heads; p.seq_capacity = seq_capacity;
-    p.scale = 1.0f / sqrtf((float)kHeadDim);
-    p.out = out; p.ldo = dec->cfg.d_model;
-    p.ln_stats = ln_stats; p.ln_c1 = ln_c1; p.ln_c2 = ln_c2;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(std::min(rows_ub * dec->cfg.n_heads, dec->sm_count));
-    cfg.blockDim = dim3(as::kAsThreads);
-    cfg.dynamicSmemBytes = (size_t)as::kStages * as::kStageBytes + 1024;
-    cfg.stream = dec->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, as::attn_stream_kernel<kCross>, p);
-    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
-    AED_LAUNCHED(dec);
-    return AED_OK;
-}
-
 #define AED_TRY(expr)                        \
     do {                                     \
         aed_status_t s__ = (expr);           \
@@ -500,8 +467,6 @@ aed_status_t tc_setup(aed_dec *dec)
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
     dec->sm_count = sms > 0 ? sms : 148;
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(as::attn_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, as::kStages * as::kStageBytes + 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(as::attn_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, as::kStages * as::kStageBytes + 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_GAMMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_LN_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -526,8 +491,7 @@ aed_status_t tc_setup(aed_dec *dec)
         dec->use_pdl = !(v && v[0] == '1');
         v = getenv("AED_DEC_NO_ATTN_PIPE");
         dec->attn_pipe = !(v && v[0] == '1');
-        v = getenv("AED_DEC_ATTN_STREAM_ROWS");
-        if (v && atoi(v) > 0) dec->attn_stream_rows = atoi(v);
+
     }
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
     if (ctas && atoi(ctas) > 0) { dec->tc_target_ctas = atoi(ctas); dec->tc_target_fixed = true; }
@@ -676,11 +640,8 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.prefetch_ptr = wn.w_qkv; p.prefetch_bytes = (size_t)3 * d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p));
         // 2. self-attention (applies LN1 to q, k, v; appends k, v)
-        if (rows_ub > dec->attn_stream_rows)
-            AED_TRY(launch_attention_stream<false>(dec, rows_ub, qkv, 3 * d, self_cache, c.max_dec_len, att, stats, c1_qkv, c2_qkv, pdl));
-        else
-            AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
-                                                            nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
+        AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
+                                                        nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
         // 3. x += att Wo^T + bo ; side: clear the FFN hidden rows
         p = sg::StepGemmParams{};
         p.src = att; p.ld_src = d;
@@ -696,12 +657,8 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.prefetch_ptr = wn.w_q_c; p.prefetch_bytes = (size_t)d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QC, m.qc, dec->tc_src_x, d, d, rows_ub, p));
         // 5. cross-attention
-        if (rows_ub > dec->attn_stream_rows)
-            AED_TRY(launch_attention_stream<true>(dec, rows_ub, qc, d, const_cast<T *>(cross), c.max_total_enc_frames, att,
-                                                  stats + stats_stride, c1_qc, c2_qc, pdl));
-        else
-            AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
-                                                            nullptr, nullptr, stats + stats_stride, c1_qc, c2_qc, pdl)));
+        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
+                                                        nullptr, nullptr, stats + stats_stride, c1_qc, c2_qc, pdl)));
         // 6. x += att Woc^T + boc ; side: clear the [q | k | v] rows for the next layer
         p = sg::StepGemmParams{};
         p.src = att; p.ld_src = d;

@@ -83,11 +83,20 @@ def family_bytes(family, w):
     return None
 
 
-# DRAM bytes per algorithmic byte of a kernel family, from the ncu capture summarised in
-# profiles/step_kernels_cfg2_clip2_ncu.txt (dram__bytes_read.sum + dram__bytes_write.sum of one launch over the
-# family's algorithmic bytes of that launch; traffic grows in proportion to the rows' frames).  An entry is removed
-# when its kernel changes, which turns the reported traffic back into null.
-NCU_TRAFFIC_RATIO = {"attn_cross": 30.789888 / 30.490624}
+# Which kernel a launch family runs (the library times launches per call site; the six projections of a layer are
+# six call sites of one kernel).
+KERNEL_OF_FAMILY = {
+    "gemm_qkv": "step_gemm_kernel", "gemm_o": "step_gemm_kernel", "gemm_qc": "step_gemm_kernel",
+    "gemm_oc": "step_gemm_kernel", "gemm_ff1": "step_gemm_kernel", "gemm_ff2": "step_gemm_kernel",
+    "attn_self": "attn_fused_kernel", "attn_cross": "attn_fused_kernel", "attn_combine": "attn_combine_kernel",
+    "gemm_vocab": "tc_gemm_kernel", "precompute_cross_kv": "crosskv_gemm_kernel", "layernorm": "layernorm_planes_kernel",
+    "embed": "embed_kernel", "bookkeeping": "build_active/finish_step",
+}
+
+# DRAM bytes per algorithmic byte of a kernel, from the ncu captures summarised under profiles/ (dram__bytes_read.sum +
+# dram__bytes_write.sum of the captured launches over their algorithmic bytes).  An entry is removed when its kernel
+# changes, which turns the reported traffic back into null.
+NCU_TRAFFIC_RATIO = {}
 
 
 def roofline_seconds(w, peaks):
@@ -413,7 +422,7 @@ def main():
             "clocks": clocks,
         }
         if not args.no_profile:
-            line["roofline"] = profile_dominant_kernel(dec, w, one_pass, peaks)
+            line["roofline"] = profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step)
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(w)
         print(json.dumps(line), flush=True)
@@ -423,25 +432,41 @@ def main():
         dist.destroy_process_group()
 
 
-def profile_dominant_kernel(dec, w, one_pass, peaks):
-    """Per-kernel device time of one more pass, taken with CUDA events around every launch on the library's
-    stream, and the roofline figure of the kernel family that takes the largest share."""
+def profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step):
+    """Roofline figure of the kernel that takes the largest share of device time.
+
+    Shares come from one extra pass with CUDA events around every launch on the library's stream (no graph replay in
+    that pass), summed per kernel, not per call site.  The kernel's time inside the measured (graphed, overlapped)
+    pass is taken as share x measured pass time: launches overlap under programmatic dependent launch, so a per-launch
+    duration of the measured configuration only exists in that sense.  ``avg_us_ungraphed`` is the plain event
+    figure of the extra pass, which includes the host launch gap."""
     prof = dec.profile_pass(one_pass)
     if not prof:
         return None
-    top = max(prof, key=lambda k: prof[k]["ms"])
-    info = prof[top]
-    bytes_total = family_bytes(top, w)
-    achieved = bytes_total / (info["ms"] * 1e-3) / 1e9 if bytes_total else None
-    ratio = NCU_TRAFFIC_RATIO.get(top) if w.name == "cfg2" else None
-    traffic = ratio * bytes_total / max(info["launches"], 1) if (ratio and bytes_total) else None
-    return {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": traffic,
-            "traffic_unit": "bytes per launch (ncu capture of a 64-row launch, scaled by frames)",
-            "algorithmic_bytes_per_launch": (bytes_total / max(info["launches"], 1)) if bytes_total else None,
-            "launches": info["launches"], "avg_us": 1e3 * info["ms"] / max(info["launches"], 1),
+    total = sum(v["ms"] for v in prof.values())
+    kernels = {}
+    for fam, v in prof.items():
+        k = kernels.setdefault(KERNEL_OF_FAMILY.get(fam, fam), {"ms": 0.0, "launches": 0, "bytes": 0.0, "families": []})
+        k["ms"] += v["ms"]; k["launches"] += v["launches"]; k["families"].append(fam)
+        k["bytes"] += family_bytes(fam, w) or 0.0
+    top = max(kernels, key=lambda k: kernels[k]["ms"])
+    info = kernels[top]
+    share = info["ms"] / total
+    in_graph_ms = share * ms_per_step
+    per_launch = info["bytes"] / max(info["launches"], 1)
+    achieved = info["bytes"] / (in_graph_ms * 1e-3) / 1e9 if info["bytes"] else None
+    ratio = NCU_TRAFFIC_RATIO.get(top)
+    return {"bound": "hbm", "kernel": top, "families": sorted(info["families"]), "achieved": achieved,
+            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
+            "traffic": ratio * per_launch if (ratio and per_launch) else None,
+            "traffic_unit": "bytes per launch (ncu capture of one layer's launches, scaled by algorithmic bytes)",
+            "algorithmic_bytes_per_launch": per_launch or None,
+            "launches": info["launches"], "share_of_device_time": round(share, 4),
+            "avg_us": 1e3 * in_graph_ms / max(info["launches"], 1),
+            "avg_us_ungraphed": 1e3 * info["ms"] / max(info["launches"], 1),
             "peak_source": peaks["source"],
-            "shares": {k: round(v["ms"] / sum(x["ms"] for x in prof.values()), 4) for k, v in prof.items()}}
+            "shares": {k: round(v["ms"] / total, 4) for k, v in sorted(kernels.items(), key=lambda kv: -kv[1]["ms"])},
+            "family_shares": {k: round(v["ms"] / total, 4) for k, v in prof.items()}}
 
 
 if __name__ == "__main__":

@@ -49,7 +49,7 @@ struct Layout {
     size_t self_layer_elems, cross_layer_elems;
     int max_chunks;
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
-    size_t actd_hi, actd_lo;
+    size_t actd_hi, actd_lo, actf_hi, actf_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
     size_t ckv_maps, ckv_bias;            // per-layer tensor maps and bias pointers of the cross-K/V weights
     size_t fold_layer_floats;
@@ -115,6 +115,8 @@ Layout make_layout(const aed_dec_config_t &c)
     if (c.dtype == AED_DTYPE_BF16) {
         L.actd_hi = take((size_t)L.rows_cap * d * 2);
         L.actd_lo = take((size_t)L.rows_cap * d * 2);
+        L.actf_hi = take((size_t)L.rows_cap * F * 2);        // FFN hidden layer as planes (steps with many rows)
+        L.actf_lo = take((size_t)L.rows_cap * F * 2);
         L.fold_layer_floats = 2 * (3 * d + d + F);       // c1 | c2 for qkv, then for cross-q, then for ffn1
         L.fold_c = take(L.fold_layer_floats * c.n_layers * 4);
         L.ln_stats = take((size_t)3 * rows_bucket(c.max_batch) * 8);
@@ -155,7 +157,7 @@ struct aed_dec {
     struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
-    CUtensorMap tc_actd[5][2];                    // [log2(N/16)][plane]: final LayerNorm output, operand of the vocabulary projection
+    CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]: activation planes [rows, d] and [rows, F]
     CUtensorMap tc_src_x[5], tc_src_att[5], tc_src_hid[5];   // fp32 sources of the fused projections, per MMA N
     bool use_tc = false;
     int sm_count = 148;
@@ -163,6 +165,7 @@ struct aed_dec {
     bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
     bool use_pdl = true;
     bool attn_pipe = true;
+    int planes_rows = 128;                // steps with more rows make their activation planes once per projection input
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
     struct GraphEntry { cudaGraphExec_t exec; int64_t nodes; };
@@ -450,6 +453,8 @@ aed_status_t tc_setup(aed_dec *dec)
         const int box = 16 << i;
         ok = ok && encode_map(&dec->tc_actd[i][0], dec->ws + L.actd_hi, L.rows_cap, d, box) &&
              encode_map(&dec->tc_actd[i][1], dec->ws + L.actd_lo, L.rows_cap, d, box) &&
+             encode_map(&dec->tc_actf[i][0], dec->ws + L.actf_hi, L.rows_cap, F, box) &&
+             encode_map(&dec->tc_actf[i][1], dec->ws + L.actf_lo, L.rows_cap, F, box) &&
              encode_map(&dec->tc_src_x[i], dec->ws + L.x, c.max_batch, d, box, true) &&
              encode_map(&dec->tc_src_att[i], dec->ws + L.act, c.max_batch, d, box, true) &&
              encode_map(&dec->tc_src_hid[i], dec->ws + L.hid, c.max_batch, F, box, true);
@@ -470,6 +475,7 @@ aed_status_t tc_setup(aed_dec *dec)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_GAMMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_LN_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
     // LayerNorm-fold constants of every layer
     for (int l = 0; l < c.n_layers; ++l) {
@@ -491,6 +497,8 @@ aed_status_t tc_setup(aed_dec *dec)
         dec->use_pdl = !(v && v[0] == '1');
         v = getenv("AED_DEC_NO_ATTN_PIPE");
         dec->attn_pipe = !(v && v[0] == '1');
+        v = getenv("AED_DEC_PLANES_ROWS");
+        if (v && atoi(v) > 0) dec->planes_rows = atoi(v);
 
     }
     const char *ctas = getenv("AED_DEC_GEMM_CTAS");
@@ -556,8 +564,9 @@ struct FusedGemm {
 
 template <int MODE>
 aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, const CUtensorMap *src_maps, int M,
-                              int K, int rows_ub, sg::StepGemmParams p)
+                              int K, int rows_ub, sg::StepGemmParams p, const CUtensorMap (*plane_maps)[2] = nullptr)
 {
+    // plane_maps (B_PLANES only): [log2(N/16)][high, low] tensor maps of the ready-made activation planes
     ProfScope ps(dec, family);
     // Rows per CTA tile: up to 128 (two ring stages still fit beside the transposition buffer); more rows are
     // covered by row tiles that re-read the weight tile from L2.
@@ -566,7 +575,7 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     const int n_tile = 16 << ni;
     const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
     const int k_blocks = K / tc::kBlockK;
-    const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2 + n_tile * tc::kBlockK * 4;
+    const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2 + (MODE == sg::B_PLANES ? 0 : n_tile * tc::kBlockK * 4);
     int stages = kTcSmemBudget / stage_bytes;
     if (stages > sg::kMaxKb) stages = sg::kMaxKb;
     // k-splits: every split adds rows x features x 4 bytes of red.global traffic, so large batches stop at about
@@ -597,7 +606,12 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     attr[0].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, src_maps[ni], p);
+    // the accumulator is transposed through the ring's memory before it leaves: n_tile rows of 132 floats
+    if (MODE == sg::B_PLANES && (size_t)stages * stage_bytes < (size_t)n_tile * (tc::kTileM + 4) * 4)
+        cfg.dynamicSmemBytes = (size_t)n_tile * (tc::kTileM + 4) * 4 + 1024;
+    cudaError_t e = MODE == sg::B_PLANES
+                        ? cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, plane_maps[ni][0], plane_maps[ni][1], p)
+                        : cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, src_maps[ni], src_maps[ni], p);
     if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "projection launch: %s", cudaGetErrorString(e));
     AED_LAUNCHED(dec);
     return AED_OK;
@@ -679,6 +693,106 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
         p.prefetch_ptr = wn.w_ff2; p.prefetch_bytes = (size_t)F * d * e2;
         AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, dec->tc_src_hid, d, F, rows_ub, p));
+    }
+    AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
+    tc::TcParams tp{};
+    tp.bias = (const T *)dec->b_out;
+    tp.logits_out = logits_out;
+    tp.keys = dec->at<unsigned long long>(L.keys);
+    tp.active_list = active_list;
+    AED_TRY(launch_vocab_gemm(dec, rows_ub, tp));
+    return AED_OK;
+}
+
+// ---- steps with many rows (bf16 mode): activation planes made once per projection input, 12 kernels per layer -------
+// With hundreds of rows every feature tile of the fused projections would convert the same activation rows again
+// (24 times for the QKV projection) and that conversion, not the tensor cores, would set the pace.  Here a small kernel
+// writes gamma * x (with the row statistics) or the ReLU of the corrected hidden layer as bf16 planes once, attention
+// writes its output as planes, and the projections fetch both operands by TMA.
+
+template <typename K, typename... Args>
+aed_status_t launch_pdl(aed_dec *dec, K kernel, dim3 grid, dim3 block, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = dec->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, args...);
+    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
+aed_status_t forward_step_planes(aed_dec *dec, int rows_ub, int self_len_ub, const int32_t *tokens, float *logits_out)
+{
+    typedef __nv_bfloat16 T;
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const int d = c.d_model, F = c.d_ffn, V = c.vocab;
+    float *x = dec->at<float>(L.x), *qkv = dec->at<float>(L.qkv), *hid = dec->at<float>(L.hid), *qc = dec->at<float>(L.qc);
+    T *ad_hi = dec->at<T>(L.actd_hi), *ad_lo = dec->at<T>(L.actd_lo), *af_hi = dec->at<T>(L.actf_hi), *af_lo = dec->at<T>(L.actf_lo);
+    float2 *stats = dec->at<float2>(L.ln_stats);
+    const int stats_stride = rows_bucket(c.max_batch);
+    const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
+    {
+        ProfScope ps(dec, KF_EMBED);
+        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
+        AED_LAUNCHED(dec);
+    }
+    const bool pdl = dec->use_pdl;
+    const dim3 ln_block(d <= 2048 ? 256 : 1024);
+    auto gamma_planes = [&](const void *g, float2 *st, float *zero_buf, int zero_cols) -> aed_status_t {
+        ProfScope ps(dec, KF_LAYERNORM);
+        return launch_pdl(dec, gamma_planes_kernel<8>, dim3(rows_ub), ln_block, (const DecState *)dec->state(), (const float *)x,
+                          (const T *)g, d, c.ln_eps, st, ad_hi, ad_lo, zero_buf, zero_cols);
+    };
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerWeights &w = dec->layers[l];
+        const aed_dec::TcLayerMaps &m = dec->tc_layers[l];
+        T *self_cache = dec->at<T>(L.self_cache) + (size_t)l * L.self_layer_elems;
+        const T *cross = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+        const float *fc = dec->at<float>(L.fold_c) + (size_t)l * L.fold_layer_floats;
+        const float *c1_qkv = fc, *c2_qkv = fc + 3 * d, *c1_qc = fc + 6 * d, *c2_qc = fc + 7 * d, *c1_ff = fc + 8 * d,
+                    *c2_ff = fc + 8 * d + F;
+        sg::StepGemmParams p{};
+        // self-attention block
+        AED_TRY(gamma_planes(w.ln1_g, stats, qc, d));
+        p.out = qkv; p.ldo = 3 * d;
+        AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_QKV, m.qkv, nullptr, 3 * d, d, rows_ub, p, dec->tc_actd));
+        AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, nullptr,
+                                                        ad_hi, ad_lo, stats, c1_qkv, c2_qkv, pdl)));
+        p = sg::StepGemmParams{};
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
+        AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_O, m.o, nullptr, d, d, rows_ub, p, dec->tc_actd));
+        // cross-attention block
+        AED_TRY(gamma_planes(w.ln2_g, stats + stats_stride, hid, F));
+        p = sg::StepGemmParams{};
+        p.out = qc; p.ldo = d;
+        AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_QC, m.qc, nullptr, d, d, rows_ub, p, dec->tc_actd));
+        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, nullptr,
+                                                        ad_hi, ad_lo, stats + stats_stride, c1_qc, c2_qc, pdl)));
+        p = sg::StepGemmParams{};
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
+        AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_OC, m.oc, nullptr, d, d, rows_ub, p, dec->tc_actd));
+        // feed-forward block
+        AED_TRY(gamma_planes(w.ln3_g, stats + 2 * stats_stride, qkv, 3 * d));
+        p = sg::StepGemmParams{};
+        p.out = hid; p.ldo = F;
+        AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_FF1, m.ff1, nullptr, F, d, rows_ub, p, dec->tc_actd));
+        {
+            ProfScope ps(dec, KF_LAYERNORM);
+            AED_TRY(launch_pdl(dec, lnrelu_planes_kernel, dim3((F / 4 + 255) / 256, rows_ub), dim3(256), (const DecState *)dec->state(),
+                               (const float *)hid, F, (const float2 *)(stats + 2 * stats_stride), c1_ff, c2_ff, af_hi, af_lo));
+        }
+        p = sg::StepGemmParams{};
+        p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
+        AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_FF2, m.ff2, nullptr, d, F, rows_ub, p, dec->tc_actf));
     }
     AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
     tc::TcParams tp{};
@@ -904,8 +1018,9 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_build_active(dec, active));
     const int rows_ub = dec->batch;
     const int self_len_ub = dec->steps_issued + 1 < dec->cfg.max_dec_len ? dec->steps_issued + 1 : dec->cfg.max_dec_len;
-    aed_status_t s = dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out)
-                                 : forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out);
+    aed_status_t s = !dec->use_tc ? forward_step<float>(dec, rows_ub, self_len_ub, tokens_in, logits_out)
+                     : rows_ub > dec->planes_rows ? forward_step_planes(dec, rows_ub, self_len_ub, tokens_in, logits_out)
+                                                  : forward_step_fused(dec, rows_ub, self_len_ub, tokens_in, logits_out);
     if (s != AED_OK) return s;
     AED_TRY(launch_finish(dec, rows_ub, next_out, 0, nullptr, nullptr));
     dec->steps_issued++;
@@ -977,8 +1092,9 @@ aed_status_t enqueue_greedy_step(aed_dec *dec, int rows_ub, int self_len_ub, int
     if (self_len_ub > dec->cfg.max_dec_len) self_len_ub = dec->cfg.max_dec_len;
     AED_TRY(launch_build_active(dec, nullptr));
     const int32_t *tok = dec->at<int32_t>(L.cur_tok);
-    aed_status_t st = dec->use_tc ? forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr)
-                                  : forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr);
+    aed_status_t st = !dec->use_tc ? forward_step<float>(dec, rows_ub, self_len_ub, tok, nullptr)
+                      : rows_ub > dec->planes_rows ? forward_step_planes(dec, rows_ub, self_len_ub, tok, nullptr)
+                                                   : forward_step_fused(dec, rows_ub, self_len_ub, tok, nullptr);
     if (st != AED_OK) return st;
     return launch_finish(dec, rows_ub, nullptr, 1, tokens_out, out_lens);
 }

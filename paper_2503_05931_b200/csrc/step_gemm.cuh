@@ -9,6 +9,9 @@
 //   B_PLAIN    B = src                                   (attention output -> output projection)
 //   B_GAMMA    B = gamma[k] * src                        (LayerNorm folded into the projection, see below)
 //   B_LN_RELU  B = relu(rstd_r * (src - mean_r * c1[k]) + c2[k])   (FFN hidden layer from the folded first GEMM)
+//   B_PLANES   B arrives ready-made: bf16 high and low planes in global memory, fetched by TMA.  Steps with many rows
+//              take this form: there every feature tile would otherwise convert the same activation rows again, and
+//              the conversion, not the tensor cores, would set the pace.
 //
 // LayerNorm folding: LN(x) W^T = rstd * ((gamma*x) W^T - mean * c1) + c2 with c1[o] = sum_k gamma_k W[o,k] and
 // c2[o] = sum_k beta_k W[o,k] + b[o].  The GEMM therefore runs on gamma*x without knowing the row statistics;
@@ -29,7 +32,7 @@ using namespace tc;
 constexpr int kMaxKb = 4;             // ring stages per CTA
 constexpr int kSgThreads = 384;       // warp 0 TMA, warp 1 MMA, warps 2..9 activation tiles and epilogue, warps 10..11 side jobs
 
-enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2 };
+enum BMode { B_PLAIN = 0, B_GAMMA = 1, B_LN_RELU = 2, B_PLANES = 3 };
 
 struct StepGemmParams {
     int a_rows;                // output features M
@@ -96,8 +99,10 @@ __device__ __forceinline__ void red_add_v4(float *addr, float4 v)
 // (n_tile x 256 B, filled by TMA, later reused to transpose the accumulator); plus 1024 for alignment.
 template <int MODE>
 __global__ void __launch_bounds__(kSgThreads, 2)
-step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_src, StepGemmParams p)
+step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_src,
+                 const __grid_constant__ CUtensorMap map_lo, StepGemmParams p)
 {
+    // map_src: fp32 source tiles (B_PLAIN, B_GAMMA, B_LN_RELU) or the high plane (B_PLANES); map_lo: the low plane.
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t bar_a[kMaxKb];
     __shared__ __align__(8) uint64_t bar_s[kMaxKb];
@@ -120,11 +125,11 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     const int S = p.stages;
     // Small tiles (at most 32 rows, one or two k-blocks): the producer threads read their 8 source values per k-block
     // straight from global memory right after the dependency wait instead of waiting for a TMA copy into shared memory.
-    const bool direct = p.n_tile <= 32 && n_kb <= 2;
+    const bool direct = MODE != B_PLANES && p.n_tile <= 32 && n_kb <= 2;
 
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
     const int plane_bytes = p.n_tile * kBlockK * 2;
-    const int src_bytes = p.n_tile * kBlockK * 4;
+    const int src_bytes = MODE == B_PLANES ? 0 : p.n_tile * kBlockK * 4;
     const int stage_bytes = kATileBytes + 2 * plane_bytes + src_bytes;
     uint32_t tmem_cols = 32;
     while (tmem_cols < static_cast<uint32_t>(p.n_tile)) tmem_cols <<= 1;
@@ -164,7 +169,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                     tma_load_2d(stage, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[s]);
                 }
                 // fp32 activation source, written by the previous kernels
-                if (!direct) {
+                if (MODE != B_PLANES && !direct) {
                     mbar_expect_tx(&bar_s[s], src_bytes);
                     tma_load_2d(stage + kATileBytes + 2 * plane_bytes, &map_src, (kb_begin + i) * kBlockK, row0, &bar_s[s]);
                 }
@@ -178,7 +183,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             for (int i = 0; i < n_kb && ok; ++i) {
                 const int s = i % S;
                 const uint32_t par = (i / S) & 1;
-                ok = mbar_wait(&bar_b[s], par, &abort_flag) && mbar_wait(&bar_a[s], par, &abort_flag);
+                ok = mbar_wait(MODE == B_PLANES ? &bar_s[s] : &bar_b[s], par, &abort_flag) && mbar_wait(&bar_a[s], par, &abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t sa = smem_u32(tiles + static_cast<size_t>(s) * stage_bytes);
@@ -212,6 +217,23 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + i * 4096), "r"(4096) : "memory");
         }
         pdl_wait();
+        if (MODE == B_PLANES) {
+            // the activation planes of every k-block, by the first lane of these two warps (a thread's copies complete
+            // one after the other); each ring stage is refilled by one of them only
+            if (lane == 0) {
+                const int loaders = (S % 2 == 0) ? 2 : 1, me = warp - 10;
+                if (me < loaders) {
+                    for (int i = me; i < n_kb; i += loaders) {
+                        const int s = i % S;
+                        if (i >= S && !mbar_wait(&bar_e[s], ((i / S) - 1) & 1, &abort_flag)) break;
+                        uint8_t *stage = tiles + static_cast<size_t>(s) * stage_bytes;
+                        mbar_expect_tx(&bar_s[s], 2 * plane_bytes);
+                        tma_load_2d(stage + kATileBytes, &map_src, (kb_begin + i) * kBlockK, row0, &bar_s[s]);
+                        tma_load_2d(stage + kATileBytes + plane_bytes, &map_lo, (kb_begin + i) * kBlockK, row0, &bar_s[s]);
+                    }
+                }
+            }
+        }
         const int n_rows = p.state->n_active;
         if (p.zero_buf) {
             const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
@@ -266,7 +288,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 if (i < n_kb) load8(p.src + static_cast<size_t>(rs) * p.ld_src + (kb_begin + i) * kBlockK + c * 8, dv[i]);
         }
         bool ok = true;
-        for (int i = 0; i < n_kb && ok; ++i) {
+        for (int i = 0; MODE != B_PLANES && i < n_kb && ok; ++i) {
             const int s = i % S;
             uint8_t *stage = tiles + static_cast<size_t>(s) * stage_bytes;
             uint8_t *hi_tile = stage + kATileBytes, *lo_tile = hi_tile + plane_bytes;
@@ -319,7 +341,8 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         constexpr int kPitch = kTileM + 4;
         const int rows_here = min(p.n_tile, max(n_rows - row0, 0));
         const int second = warp >= 6 ? 1 : 0;
-        const bool fits = static_cast<size_t>(p.n_tile) * kPitch * 4 <= static_cast<size_t>(n_kb < S ? n_kb : S) * stage_bytes;
+        // (B_PLANES: the launch reserves at least the transposition buffer, whatever the ring needs)
+        const bool fits = MODE == B_PLANES || static_cast<size_t>(p.n_tile) * kPitch * 4 <= static_cast<size_t>(n_kb < S ? n_kb : S) * stage_bytes;
         if (ok && fits) {
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             for (int c0 = 16 * second; c0 < rows_here; c0 += 32) {

@@ -712,6 +712,102 @@ __global__ void layernorm_planes_kernel(const DecState *state, const float *__re
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// Activation planes for steps with many rows.  There the projections fetch their activation operand ready-made
+// (bf16 high plane + bf16 low plane = value - high) instead of converting it in every feature tile.
+// Both kernels start with a programmatic-dependency wait and may be launched ahead of their predecessor's end.
+// ------------------------------------------------------------------------------------------------------------
+// planes of gamma * x, the LayerNorm statistics (mean, rstd) of every row, and the clearing of the fp32 rows a later
+// split-K projection accumulates into (zero_cols columns of zero_buf, if any).  One block per row.
+template <int kMaxPerThread>
+__global__ void gamma_planes_kernel(const DecState *state, const float *__restrict__ x, const __nv_bfloat16 *__restrict__ g,
+                                    int d, float eps, float2 *__restrict__ stats_out, __nv_bfloat16 *__restrict__ out_hi,
+                                    __nv_bfloat16 *__restrict__ out_lo, float *__restrict__ zero_buf, int zero_cols)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int r = blockIdx.x;
+    if (r >= state->n_active) return;
+    __shared__ float red[32];
+    __shared__ float stat;
+    float v[kMaxPerThread];
+    const float *xr = x + (size_t)r * d;
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        const int i = threadIdx.x + j * blockDim.x;
+        v[j] = (i < d) ? xr[i] : 0.f;
+        s += v[j];
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    s = warp_sum(s);
+    if (lane == 0) red[warp] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) { float t = 0.f; for (int w = 0; w < n_warps; ++w) t += red[w]; stat = t / d; }
+    __syncthreads();
+    const float mean = stat;
+    float q = 0.f;
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        const int i = threadIdx.x + j * blockDim.x;
+        const float c = (i < d) ? v[j] - mean : 0.f;
+        q += c * c;
+    }
+    q = warp_sum(q);
+    __syncthreads();
+    if (lane == 0) red[warp] = q;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < n_warps; ++w) t += red[w];
+        stats_out[r] = make_float2(mean, rsqrtf(t / d + eps));
+    }
+#pragma unroll
+    for (int j = 0; j < kMaxPerThread; ++j) {
+        const int i = threadIdx.x + j * blockDim.x;
+        if (i < d) {
+            const float y = to_f32(g[i]) * v[j];
+            const __nv_bfloat16 hi = __float2bfloat16_rn(y);
+            out_hi[(size_t)r * d + i] = hi;
+            out_lo[(size_t)r * d + i] = __float2bfloat16_rn(y - __bfloat162float(hi));
+        }
+    }
+    for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
+}
+
+// planes of relu(rstd * (hidden_raw - mean * c1) + c2): the FFN hidden layer after the folded first projection.
+// grid: x = blocks of 1024 hidden features, y = rows.
+__global__ void lnrelu_planes_kernel(const DecState *state, const float *__restrict__ hid, int f,
+                                     const float2 *__restrict__ stats, const float *__restrict__ c1,
+                                     const float *__restrict__ c2, __nv_bfloat16 *__restrict__ out_hi,
+                                     __nv_bfloat16 *__restrict__ out_lo)
+{
+    const int r = blockIdx.y;
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (i < f) {                       // static operands before the dependency wait
+        a = *reinterpret_cast<const float4 *>(c1 + i);
+        b = *reinterpret_cast<const float4 *>(c2 + i);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (r >= state->n_active || i >= f) return;
+    const float2 st = stats[r];
+    const float4 h = *reinterpret_cast<const float4 *>(hid + (size_t)r * f + i);
+    const float y[4] = {fmaxf(fmaf(st.y, h.x - st.x * a.x, b.x), 0.f), fmaxf(fmaf(st.y, h.y - st.x * a.y, b.y), 0.f),
+                        fmaxf(fmaf(st.y, h.z - st.x * a.z, b.z), 0.f), fmaxf(fmaf(st.y, h.w - st.x * a.w, b.w), 0.f)};
+    __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        hi[j] = __float2bfloat16_rn(y[j]);
+        lo[j] = __float2bfloat16_rn(y[j] - __bfloat162float(hi[j]));
+    }
+    __nv_bfloat162 *ph = reinterpret_cast<__nv_bfloat162 *>(out_hi + (size_t)r * f + i);
+    __nv_bfloat162 *pl = reinterpret_cast<__nv_bfloat162 *>(out_lo + (size_t)r * f + i);
+    ph[0] = __halves2bfloat162(hi[0], hi[1]); ph[1] = __halves2bfloat162(hi[2], hi[3]);
+    pl[0] = __halves2bfloat162(lo[0], lo[1]); pl[1] = __halves2bfloat162(lo[2], lo[3]);
+}
+
+// ------------------------------------------------------------------------------------------------------------
 // End of a step: decode the argmax keys, hand the choice out by utterance id, advance t_u, and (greedy mode)
 // record the token, feed it back and retire finished utterances.
 // ------------------------------------------------------------------------------------------------------------

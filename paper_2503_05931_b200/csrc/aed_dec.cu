@@ -328,6 +328,26 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     return AED_OK;
 }
 
+// A launch that may start before its predecessor in the stream has ended (programmatic stream serialization): the
+// kernel itself waits (griddepcontrol.wait) before it touches what the predecessor wrote.
+aed_status_t launch_pdl_impl(aed_dec *dec, const void *kernel, dim3 grid, dim3 block, size_t smem, void **args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = dec->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelExC(&cfg, kernel, args);
+    if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+    AED_LAUNCHED(dec);
+    return AED_OK;
+}
+
 #define AED_TRY(expr)                        \
     do {                                     \
         aed_status_t s__ = (expr);           \
@@ -533,29 +553,35 @@ aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p)
     int stages = kTcSmemBudget / stage_bytes;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     if (stages > k_blocks) stages = k_blocks;
-    // every ring stage belongs to one issuing thread: stages is a multiple of the number of producers
-    const int producers = stages >= tc::kProducerWarps ? tc::kProducerWarps : stages;
+    // every ring stage belongs to one issuing thread: stages is a multiple of the number of producers (prefer the
+    // deeper ring: 6 stages with 3 producers rather than 4 with 4)
+    int producers = stages >= tc::kProducerWarps ? tc::kProducerWarps : stages;
+    if (stages > tc::kProducerWarps && stages % tc::kProducerWarps && stages % (tc::kProducerWarps - 1) == 0) producers = tc::kProducerWarps - 1;
     stages -= stages % producers;
     const CUtensorMap *acts = dec->tc_actd[ni];
     dim3 grid(m_tiles, 1, row_tiles);
-    tc::tc_gemm_kernel<tc::TC_EPI_LOGITS><<<grid, tc::kThreads, (size_t)stages * stage_bytes + 1024, dec->stream>>>(
-        dec->tc_w_out, acts[0], acts[1], p, stages, producers);
-    AED_LAUNCHED(dec);
-    return AED_OK;
+    void *args[] = {(void *)&dec->tc_w_out, (void *)&acts[0], (void *)&acts[1], &p, &stages, (void *)&producers};
+    return launch_pdl_impl(dec, (const void *)tc::tc_gemm_kernel<tc::TC_EPI_LOGITS>, grid, dim3(tc::kThreads),
+                           (size_t)stages * stage_bytes + 1024, args);
 }
+
+aed_status_t launch_pdl_impl(aed_dec *dec, const void *kernel, dim3 grid, dim3 block, size_t smem, void **args);
 
 aed_status_t launch_ln_planes(aed_dec *dec, int rows_ub, const float *x, const void *g, const void *b, float *zero_buf,
                               int zero_cols)
 {
     ProfScope ps(dec, KF_LAYERNORM);
-    const int d = dec->cfg.d_model;
+    int d = dec->cfg.d_model;
+    float eps = dec->cfg.ln_eps;
     const Layout &L = dec->lay;
-    layernorm_planes_kernel<8><<<rows_ub, d <= 2048 ? 256 : 1024, 0, dec->stream>>>(
-        dec->state(), x, (const __nv_bfloat16 *)g, (const __nv_bfloat16 *)b, d, dec->cfg.ln_eps,
-        dec->at<__nv_bfloat16>(L.actd_hi), dec->at<__nv_bfloat16>(L.actd_lo), zero_buf, zero_cols);
-    AED_LAUNCHED(dec);
-    return AED_OK;
-}// ---- fused step (bf16 mode): 8 kernels per layer, chained with programmatic dependent launch -------------------
+    const DecState *state = dec->state();
+    const __nv_bfloat16 *gp = (const __nv_bfloat16 *)g, *bp = (const __nv_bfloat16 *)b;
+    __nv_bfloat16 *hi = dec->at<__nv_bfloat16>(L.actd_hi), *lo = dec->at<__nv_bfloat16>(L.actd_lo);
+    void *args[] = {&state, &x, &gp, &bp, &d, &eps, &hi, &lo, &zero_buf, &zero_cols};
+    return launch_pdl_impl(dec, (const void *)layernorm_planes_kernel<8>, dim3(rows_ub), dim3(d <= 2048 ? 256 : 1024), 0, args);
+}
+
+// ---- fused step (bf16 mode): 8 kernels per layer, chained with programmatic dependent launch -------------------
 
 struct FusedGemm {
     const CUtensorMap *map;
@@ -686,6 +712,7 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.out = hid; p.ldo = F;
         p.stats_src = x; p.stats_out = stats + 2 * stats_stride; p.stats_d = d;
         p.prefetch_ptr = wn.w_ff1; p.prefetch_bytes = (size_t)F * d * e2;
+        if (l == c.n_layers - 1) { p.prefetch2_ptr = dec->w_out; p.prefetch2_bytes = (size_t)V * d * e2; }    // the vocabulary projection is next
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, dec->tc_src_x, F, d, rows_ub, p));
         // 8. x += relu(LN3-corrected hidden) W2^T + b2
         p = sg::StepGemmParams{};
@@ -868,12 +895,14 @@ aed_status_t launch_finish(aed_dec *dec, int rows_ub, int32_t *next_out, int gre
 {
     const Layout &L = dec->lay;
     ProfScope ps(dec, KF_BOOKKEEPING);
-    finish_step_kernel<<<(rows_ub + 127) / 128, 128, 0, dec->stream>>>(
-        dec->state(), dec->at<int32_t>(L.active_list), dec->at<unsigned long long>(L.keys), dec->at<int32_t>(L.t_u),
-        next_out, greedy, dec->at<int32_t>(L.cur_tok), dec->at<int32_t>(L.retired), dec->at<int32_t>(L.max_len),
-        dec->cfg.eos_id, tokens_out, dec->cfg.max_dec_len, out_lens);
-    AED_LAUNCHED(dec);
-    return AED_OK;
+    DecState *state = dec->state();
+    const int32_t *active_list = dec->at<int32_t>(L.active_list);
+    unsigned long long *keys = dec->at<unsigned long long>(L.keys);
+    int32_t *t_u = dec->at<int32_t>(L.t_u), *cur_tok = dec->at<int32_t>(L.cur_tok), *retired = dec->at<int32_t>(L.retired);
+    const int32_t *max_len = dec->at<int32_t>(L.max_len);
+    int eos = dec->cfg.eos_id, ld = dec->cfg.max_dec_len;
+    void *args[] = {&state, &active_list, &keys, &t_u, &next_out, &greedy, &cur_tok, &retired, &max_len, &eos, &tokens_out, &ld, &out_lens};
+    return launch_pdl_impl(dec, (const void *)finish_step_kernel, dim3((rows_ub + 127) / 128), dim3(128), 0, args);
 }
 
 aed_status_t fill_i32(aed_dec *dec, int32_t *p, int32_t v, size_t n)

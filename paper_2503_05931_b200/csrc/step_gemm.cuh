@@ -59,8 +59,8 @@ struct StepGemmParams {
     float *zero_buf;
     int zero_cols;
     // side job 3: pull a byte range that a later kernel streams (next layer's weights) into L2
-    const void *prefetch_ptr;
-    size_t prefetch_bytes;
+    const void *prefetch_ptr, *prefetch2_ptr;      // (the second range: the output matrix, from the last layer)
+    size_t prefetch_bytes, prefetch2_bytes;
     DecState *state;
 };
 
@@ -209,10 +209,11 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const int st = threadIdx.x - 320;                 // 0..63
         const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
         const int n_cta = gridDim.x * gridDim.y * gridDim.z;
-        if (p.prefetch_ptr) {
+        for (int range = 0; range < 2; ++range) {
             // static data: no need to wait for the previous kernel.  4 KB pieces, spread over all CTAs and threads.
-            const size_t pieces = p.prefetch_bytes / 4096;
-            const char *base = static_cast<const char *>(p.prefetch_ptr);
+            const char *base = static_cast<const char *>(range ? p.prefetch2_ptr : p.prefetch_ptr);
+            if (!base) continue;
+            const size_t pieces = (range ? p.prefetch2_bytes : p.prefetch_bytes) / 4096;
             for (size_t i = static_cast<size_t>(cta) * 64 + st; i < pieces; i += static_cast<size_t>(n_cta) * 64)
                 asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + i * 4096), "r"(4096) : "memory");
         }

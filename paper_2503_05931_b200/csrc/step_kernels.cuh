@@ -664,6 +664,9 @@ __global__ void layernorm_planes_kernel(const DecState *state, const float *__re
                                         float *__restrict__ zero_buf, int zero_cols)
 {
     AED_TRACE_BEGIN(state, 4);
+    // launched with programmatic stream serialization: nothing of the previous kernel is touched before this wait
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int r = blockIdx.x;
     if (r >= state->n_active) return;
     __shared__ float red[32];
@@ -819,6 +822,7 @@ __global__ void finish_step_kernel(DecState *state, const int32_t *__restrict__ 
                                    int32_t *__restrict__ tokens_out, int tokens_ld, int32_t *__restrict__ out_lens)
 {
     AED_TRACE_BEGIN(state, 6);
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // launched with programmatic stream serialization
     int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= state->n_active) return;
     int u = active_list[r];

@@ -194,6 +194,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     if (threadIdx.x == 0) AED_TRACE_MARK(p.state, 32);      // set-up done
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp < kProducerWarps) {
         if (lane == 0 && warp < producers) {
@@ -201,6 +202,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             prefetch_tensormap(&map_b);
             if (p.use_lo) prefetch_tensormap(&map_b_lo);
             int issued = 0;
+            bool waited = false;
             for (int i = warp; i < n_kb; i += producers) {
                 const int s = i % stages;
                 if (i >= stages && !mbar_wait(&bar_empty[s], ((i / stages) - 1) & 1, &abort_flag)) break;
@@ -208,6 +210,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 mbar_expect_tx(&bar_full[s], stage_bytes);
                 const int kc = (kb_begin + i) * kBlockK;
                 tma_load_2d(st, &map_a, kc, a0, &bar_full[s]);
+                // A is static (a weight matrix): its first tile is requested while the previous kernel still runs;
+                // B is that kernel's output
+                if (!waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited = true; }
                 tma_load_2d(st + kATileBytes, &map_b, kc, row0, &bar_full[s]);
                 if (p.use_lo) tma_load_2d(st + kATileBytes + b_bytes, &map_b_lo, kc, row0, &bar_full[s]);
                 issued = i + 1;

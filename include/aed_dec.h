@@ -143,6 +143,23 @@ aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, const uint8_
                           int32_t *next_out);
 
 /*
+ * Feed a fixed-length prompt in one pass instead of prompt_len single steps (the paper's decoder is fed a
+ * fixed-length task / language prompt before the transcript: caption of Fig. "tpsdist").  Every utterance of the
+ * batch consumes prompt[u][0 .. prompt_len-1] at positions 0 .. prompt_len-1: one batched causal pass in which the
+ * step weights are streamed once for all positions (in chunks of floor(max_batch / batch) positions, because the
+ * (utterance, position) rows share the step's row buffers; size max_batch >= batch * prompt_len for a single pass).
+ * The result is what prompt_len calls of aed_dec_step would leave: the self-attention caches hold prompt_len
+ * positions, t_u = prompt_len, and logits_out / next_out describe the last prompt position.
+ *   prompt      DEVICE int32 [batch, prompt_len], row-major by utterance
+ *   logits_out  DEVICE float [batch, vocab] or NULL
+ *   next_out    DEVICE int32 [batch] or NULL: greedy choice after the whole prompt
+ * Must directly follow aed_dec_precompute_cross_kv (AED_ERR_STATE otherwise); continue with aed_dec_step.
+ * AED_ERR_CAPACITY if prompt_len > max_dec_len; AED_ERR_UNSUPPORTED in the fp32 configuration.
+ */
+aed_status_t aed_dec_prefill(aed_dec_t *dec, const int32_t *prompt, int32_t prompt_len, float *logits_out,
+                             int32_t *next_out);
+
+/*
  * aed_dec_step for callers that cannot allocate device memory (the paper has no counterpart; this is a
  * deployment aid).  Some hosts of this library run where cudaMalloc is off limits: a serving process whose
  * device memory pool was sized and frozen at start-up, a real-time thread that may not block in the driver,

@@ -23,7 +23,7 @@ EXPORTED_SYMBOLS = [
     "aed_dec_workspace_bytes", "aed_dec_create", "aed_dec_precompute_cross_kv", "aed_dec_step",
     "aed_dec_greedy_decode", "aed_dec_sync_status", "aed_dec_launch_count", "aed_dec_destroy",
     "aed_dec_last_error", "aed_dec_create_error", "aed_dec_profile_enable", "aed_dec_profile_read",
-    "aed_dec_step_static_scratch", "aed_dec_static_scratch_bytes", "aed_dec_status_of_error_word",
+    "aed_dec_step_static_scratch", "aed_dec_static_scratch_bytes", "aed_dec_status_of_error_word", "aed_dec_prefill",
 ]
 
 _GLOBAL_FIELDS = ["embed", "final_ln_g", "final_ln_b", "w_out", "b_out"]
@@ -70,6 +70,8 @@ def load_library() -> C.CDLL:
     lib.aed_dec_precompute_cross_kv.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32), C.c_int32]
     lib.aed_dec_step.restype = C.c_int
     lib.aed_dec_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.aed_dec_prefill.restype = C.c_int
+    lib.aed_dec_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     lib.aed_dec_step_static_scratch.restype = C.c_int
     lib.aed_dec_step_static_scratch.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.aed_dec_static_scratch_bytes.restype = C.c_size_t
@@ -187,6 +189,12 @@ class Decoder:
         logits_out float32 [B, V] or None, next_out int32 [B] or None."""
         ptr = lambda t: t.data_ptr() if t is not None else None
         self._check(self.lib.aed_dec_step(self.handle, ptr(tokens_in), ptr(active), ptr(logits_out), ptr(next_out)))
+
+    def prefill(self, prompt, logits_out=None, next_out=None) -> None:
+        """prompt: device int32 tensor [batch, prompt_len]; logits_out / next_out describe the last prompt position."""
+        assert prompt.is_cuda and prompt.dtype == self._torch.int32 and prompt.is_contiguous() and prompt.dim() == 2
+        ptr = lambda t: t.data_ptr() if t is not None else None
+        self._check(self.lib.aed_dec_prefill(self.handle, prompt.data_ptr(), int(prompt.shape[1]), ptr(logits_out), ptr(next_out)))
 
     def step_static_scratch(self, tokens_in, active=None, logits_out=None, next_out=None) -> None:
         """``step`` with the attention scratch in the library's built-in device array (for callers that

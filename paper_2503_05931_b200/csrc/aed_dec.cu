@@ -45,7 +45,7 @@ struct LayerWeights {
 // Byte offsets of every region of the caller's workspace.
 struct Layout {
     size_t self_cache, cross_store, x, act, qkv, hid, partials, pe, keys, state;
-    size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, row_info, len_order, total;
+    size_t t_u, retired, active_list, cur_tok, enc_off, enc_len, max_len, row_info, row_tok, len_order, total;
     size_t self_layer_elems, cross_layer_elems;
     int max_chunks;
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
@@ -110,6 +110,7 @@ Layout make_layout(const aed_dec_config_t &c)
     L.enc_len = take(B * 4);
     L.max_len = take(B * 4);
     L.row_info = take((size_t)rows_bucket(c.max_batch) * 16);      // grids are sized for the bucket
+    L.row_tok = take((size_t)rows_bucket(c.max_batch) * 4);        // prefill: the token of every (utterance, position) row
     L.len_order = take(B * 4);                                     // utterances by decreasing encoder length
     L.rows_cap = (int)align_up(B, 16);
     if (c.dtype == AED_DTYPE_BF16) {
@@ -536,7 +537,7 @@ int tc_n_index(int rows_ub)
 }
 
 // The vocabulary projection on tensor cores: logits[r, v] = sum_k act[r, k] * Wout[v, k] (+ bias), argmax in the epilogue.
-aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p)
+aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p, int rows_fixed = -1)
 {
     ProfScope ps(dec, KF_GEMM_VOCAB);
     const int M = dec->cfg.vocab, K = dec->cfg.d_model;
@@ -547,7 +548,7 @@ aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p)
     p.n_tile = n_tile;
     p.k_blocks = k_blocks;
     p.use_lo = 1;
-    p.rows_fixed = -1;
+    p.rows_fixed = rows_fixed;          // >= 0: only that many rows (a prefill pass projects its last-position rows only)
     p.state = dec->state();
     const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2;
     int stages = kTcSmemBudget / stage_bytes;
@@ -643,7 +644,13 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     return AED_OK;
 }
 
-aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, const int32_t *tokens, float *logits_out)
+// A prefill pass (several prompt positions per utterance, rows = (utterance, position) pairs): the row table and the
+// rows' tokens are already in place; keys and values are appended by a kernel of their own before any row attends; only
+// the last chunk projects to the vocabulary, and only for the rows of the last position (rows 0 .. batch - 1).
+struct PrefillPass { bool last_chunk; int batch; };
+
+aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, const int32_t *tokens, float *logits_out,
+                                const PrefillPass *pf = nullptr)
 {
     typedef __nv_bfloat16 T;
     const auto &c = dec->cfg;
@@ -656,8 +663,12 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
     const int32_t *active_list = dec->at<int32_t>(L.active_list), *t_u = dec->at<int32_t>(L.t_u);
     {
         ProfScope ps(dec, KF_EMBED);
-        embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                          dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
+        if (pf)
+            embed_rows_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), dec->at<int4>(L.row_info), dec->at<int32_t>(L.row_tok),
+                                                                   (const T *)dec->embed, dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
+        else
+            embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
+                                                              dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
         AED_LAUNCHED(dec);
     }
     const bool pdl = dec->use_pdl;
@@ -680,8 +691,23 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.prefetch_ptr = wn.w_qkv; p.prefetch_bytes = (size_t)3 * d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p));
         // 2. self-attention (applies LN1 to q, k, v; appends k, v)
-        AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
-                                                        nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
+        if (pf) {
+            {
+                ProfScope ps(dec, KF_ATTN_SELF);
+                const DecState *state = dec->state();
+                const int4 *ri = dec->at<int4>(L.row_info);
+                const float *qp = qkv;
+                int ldq = 3 * d, heads = c.n_heads, cap = c.max_dec_len;
+                const float2 *stp = stats;
+                void *args[] = {&state, &ri, &qp, &ldq, &self_cache, &heads, &cap, &stp, &c1_qkv, &c2_qkv};
+                AED_TRY(launch_pdl_impl(dec, (const void *)append_kv_kernel<T>, dim3(rows_ub, c.n_heads), dim3(kHeadDim), 0, args));
+            }
+            AED_TRY((launch_attention_fused<T, false, false>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
+                                                             nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
+        } else {
+            AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
+                                                            nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
+        }
         // 3. x += att Wo^T + bo ; side: clear the FFN hidden rows
         p = sg::StepGemmParams{};
         p.src = att; p.ld_src = d;
@@ -721,13 +747,14 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.prefetch_ptr = wn.w_ff2; p.prefetch_bytes = (size_t)F * d * e2;
         AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, dec->tc_src_hid, d, F, rows_ub, p));
     }
+    if (pf && !pf->last_chunk) return AED_OK;
     AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
     tc::TcParams tp{};
     tp.bias = (const T *)dec->b_out;
     tp.logits_out = logits_out;
     tp.keys = dec->at<unsigned long long>(L.keys);
     tp.active_list = active_list;
-    AED_TRY(launch_vocab_gemm(dec, rows_ub, tp));
+    AED_TRY(launch_vocab_gemm(dec, pf ? pf->batch : rows_ub, tp, pf ? pf->batch : -1));
     return AED_OK;
 }
 
@@ -1054,6 +1081,53 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     AED_TRY(launch_finish(dec, rows_ub, next_out, 0, nullptr, nullptr));
     dec->steps_issued++;
     if (!active) dec->full_steps++;
+    dec->fresh_batch = false;
+    return AED_OK;
+}
+
+// ---- prompt prefill: several positions per utterance in one pass ---------------------------------------------------
+extern "C" aed_status_t aed_dec_prefill(aed_dec_t *dec, const int32_t *prompt, int32_t prompt_len, float *logits_out,
+                                        int32_t *next_out)
+{
+    if (!dec) return AED_ERR_INVALID_ARG;
+    if (!prompt) return fail(dec, AED_ERR_INVALID_ARG, "prompt must not be NULL");
+    if (prompt_len < 1) return fail(dec, AED_ERR_INVALID_ARG, "prompt_len must be at least 1");
+    if (!dec->have_batch) return fail(dec, AED_ERR_STATE, "aed_dec_prefill needs a batch: call aed_dec_precompute_cross_kv first");
+    if (!dec->fresh_batch) return fail(dec, AED_ERR_STATE, "aed_dec_prefill must directly follow aed_dec_precompute_cross_kv");
+    if (prompt_len > dec->cfg.max_dec_len)
+        return fail(dec, AED_ERR_CAPACITY, "prompt_len %d exceeds max_dec_len %d", prompt_len, dec->cfg.max_dec_len);
+    if (!dec->use_tc) return fail(dec, AED_ERR_UNSUPPORTED, "aed_dec_prefill needs the bf16 configuration (feed the prompt with aed_dec_step in fp32 mode)");
+    const Layout &L = dec->lay;
+    const int B = dec->batch;
+    // (utterance, position) rows share the step's row buffers: max_batch rows per pass
+    const int chunk_max = std::max(1, dec->cfg.max_batch / B);
+    for (int j0 = 0; j0 < prompt_len; j0 += chunk_max) {
+        const int chunk = std::min(chunk_max, prompt_len - j0), rows = B * chunk;
+        const bool last = j0 + chunk == prompt_len;
+        {
+            ProfScope ps(dec, KF_BOOKKEEPING);
+            const int slots = rows_bucket(dec->cfg.max_batch);
+            build_prefill_rows_kernel<<<(slots + 255) / 256, 256, 0, dec->stream>>>(
+                dec->state(), chunk, j0, prompt_len, prompt, dec->at<int32_t>(L.t_u), dec->at<int32_t>(L.enc_len),
+                dec->at<int32_t>(L.enc_off), dec->at<int32_t>(L.len_order), dec->at<int32_t>(L.active_list),
+                dec->at<int4>(L.row_info), dec->at<int32_t>(L.row_tok), slots);
+            AED_LAUNCHED(dec);
+        }
+        PrefillPass pf{last, B};
+        AED_TRY(forward_step_fused(dec, rows, j0 + chunk, nullptr, logits_out, &pf));
+        {
+            ProfScope ps(dec, KF_BOOKKEEPING);
+            DecState *state = dec->state();
+            const int32_t *active_list = dec->at<int32_t>(L.active_list);
+            unsigned long long *keys = dec->at<unsigned long long>(L.keys);
+            int32_t *t_u = dec->at<int32_t>(L.t_u), *cur_tok = dec->at<int32_t>(L.cur_tok);
+            int chunk_arg = chunk, last_arg = last ? 1 : 0;
+            void *args[] = {&state, &active_list, &keys, &t_u, &chunk_arg, &last_arg, &next_out, &cur_tok};
+            AED_TRY(launch_pdl_impl(dec, (const void *)prefill_finish_kernel, dim3((B + 127) / 128), dim3(128), 0, args));
+        }
+    }
+    dec->steps_issued = prompt_len;
+    dec->full_steps = prompt_len;
     dec->fresh_batch = false;
     return AED_OK;
 }

@@ -444,6 +444,9 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     const int len_static = (kAppend && !kCross) ? len - 1 : len;
     const int dg = lane & 7, pg = lane >> 3;
     Raw8<CT> rk[4], rv[4];
+    // Self-attention without an append of its own (prefill pass): the cache positions it reads are written by the
+    // kernel before it, so nothing is loaded ahead of the dependency wait.
+    if (!kCross && !kAppend) asm volatile("griddepcontrol.wait;" ::: "memory");
     {
         // This warp's first chunk starts streaming while the kernel that produces the query is still running.
         const int p0 = warp * kFusedChunk;
@@ -808,6 +811,89 @@ __global__ void lnrelu_planes_kernel(const DecState *state, const float *__restr
     __nv_bfloat162 *pl = reinterpret_cast<__nv_bfloat162 *>(out_lo + (size_t)r * f + i);
     ph[0] = __halves2bfloat162(hi[0], hi[1]); ph[1] = __halves2bfloat162(hi[2], hi[3]);
     pl[0] = __halves2bfloat162(lo[0], lo[1]); pl[1] = __halves2bfloat162(lo[2], lo[3]);
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Prompt prefill: several positions of every utterance in one pass.  A compact row is an (utterance, position)
+// pair; a chunk covers `chunk` consecutive positions of every utterance of the batch.  Rows are ordered position
+// major with the chunk's last position first (row = (chunk - 1 - j) * batch + i), so that the rows of the last
+// position, the only ones whose logits matter, are rows 0 .. batch - 1.
+// ------------------------------------------------------------------------------------------------------------
+__global__ void build_prefill_rows_kernel(DecState *state, int chunk, int j0, int prompt_len, const int32_t *__restrict__ prompt,
+                                          const int32_t *__restrict__ t_u, const int32_t *__restrict__ enc_len,
+                                          const int32_t *__restrict__ enc_off, const int32_t *__restrict__ order,
+                                          int32_t *__restrict__ active_list, int4 *__restrict__ row_info,
+                                          int32_t *__restrict__ row_tok, int row_slots)
+{
+    const int batch = state->batch, rows = batch * chunk;
+    for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < row_slots; r += gridDim.x * blockDim.x) {
+        if (r < rows) {
+            const int u = order[r % batch], j = chunk - 1 - r / batch;
+            active_list[r] = u;
+            row_info[r] = make_int4(u, t_u[u] + j, enc_len[u], enc_off[u]);
+            row_tok[r] = prompt[(size_t)u * prompt_len + j0 + j];
+        } else {
+            row_info[r] = make_int4(-1, 0, 0, 0);
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { state->n_active = rows; state->grid_sync = 0; }
+}
+
+// x[r] = E[token of the row] * sqrt(d) + PE[position of the row]
+template <typename T>
+__global__ void embed_rows_kernel(const DecState *state, const int4 *__restrict__ row_info, const int32_t *__restrict__ row_tok,
+                                  const T *__restrict__ embed, const float *__restrict__ pe, int d, int vocab, float scale,
+                                  float *__restrict__ x, float *__restrict__ zero_buf, int zero_cols)
+{
+    const int r = blockIdx.x;
+    if (r >= state->n_active) return;
+    const int tok = min(max(row_tok[r], 0), vocab - 1), t = row_info[r].y;
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+        x[(size_t)r * d + i] = to_f32(embed[(size_t)tok * d + i]) * scale + pe[(size_t)t * d + i];
+    for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
+}
+
+// Keys and values of every row into the self-attention cache (raw projection output with the LayerNorm fold applied,
+// rounded as the cache stores it), before any row attends: in a prefill pass a row reads positions that other rows of
+// the same pass append.  grid: (rows, heads), 64 threads.
+template <typename CT>
+__global__ void append_kv_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ qkv, int ldq,
+                                 CT *__restrict__ cache, int n_heads, int seq_capacity, const float2 *__restrict__ ln_stats,
+                                 const float *__restrict__ ln_c1, const float *__restrict__ ln_c2)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int r = blockIdx.x, h = blockIdx.y, dim = threadIdx.x;
+    const int4 ri = row_info[r];
+    if (ri.x < 0) return;
+    const int d_model = n_heads * kHeadDim;
+    const float2 st = ln_stats ? ln_stats[r] : make_float2(0.f, 1.f);
+#pragma unroll
+    for (int kv = 0; kv < 2; ++kv) {
+        const int col = (1 + kv) * d_model + h * kHeadDim + dim;
+        float y = qkv[(size_t)r * ldq + col];
+        if (ln_stats) y = fmaf(st.y, y - st.x * ln_c1[col], ln_c2[col]);
+        cache[((((size_t)ri.x * 2 + kv) * n_heads + h) * (size_t)seq_capacity + ri.y) * kHeadDim + dim] = from_f32<CT>(y);
+    }
+}
+
+// End of a prefill chunk: every utterance has `chunk` more positions cached; after the last chunk the argmax of the
+// last prompt position (rows 0 .. batch - 1) is handed out and becomes the utterance's current token.
+__global__ void prefill_finish_kernel(DecState *state, const int32_t *__restrict__ active_list,
+                                      unsigned long long *__restrict__ keys, int32_t *__restrict__ t_u, int chunk, int last,
+                                      int32_t *__restrict__ next_out, int32_t *__restrict__ cur_tok)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= state->batch) return;
+    const int u = active_list[r];
+    t_u[u] += chunk;
+    if (last) {
+        const int32_t tok = argmax_key_index(keys[r]);
+        keys[r] = 0ull;
+        cur_tok[u] = tok;
+        if (next_out) next_out[u] = tok;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------------------

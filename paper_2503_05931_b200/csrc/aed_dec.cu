@@ -175,6 +175,10 @@ struct aed_dec {
     bool use_graphs = true;
     // set only while aed_dec_step_static_scratch runs: attention partials go here instead of the workspace
     float *partials_override = nullptr;
+    // greedy decoding with an end-of-sequence id: the retired count of recent steps, copied to pinned host memory
+    static constexpr int kProbeSlots = 16;
+    int32_t *probe_host = nullptr;
+    cudaEvent_t probe_event[kProbeSlots] = {};
 
     template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
     DecState *state() const { return at<DecState>(lay.state); }
@@ -1252,7 +1256,21 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
     AED_TRY(fill_i32(dec, dec->at<int32_t>(L.cur_tok), dec->cfg.bos_id, B));
     AED_TRY(fill_i32(dec, tokens_out, -1, (size_t)B * dec->cfg.max_dec_len));
     AED_TRY(fill_i32(dec, out_lens, 0, B));
+    // With an end-of-sequence id the forced lengths are only upper bounds.  The host then stays at most kWindow steps
+    // ahead of the device: before it issues step s it looks at the retired count that step s - kWindow left behind
+    // (an asynchronous copy into pinned memory followed by an event) and stops once every utterance has retired.
+    const bool probe = dec->cfg.eos_id >= 0;
+    constexpr int kWindow = 8;
+    if (probe && !dec->probe_host) {
+        AED_CUDA(dec, cudaHostAlloc(reinterpret_cast<void **>(&dec->probe_host), aed_dec::kProbeSlots * sizeof(int32_t), cudaHostAllocDefault));
+        for (int i = 0; i < aed_dec::kProbeSlots; ++i) AED_CUDA(dec, cudaEventCreateWithFlags(&dec->probe_event[i], cudaEventDisableTiming));
+    }
     for (int s = 0; s < longest; ++s) {
+        if (probe && s >= kWindow) {
+            const int slot = (s - kWindow) % aed_dec::kProbeSlots;
+            AED_CUDA(dec, cudaEventSynchronize(dec->probe_event[slot]));
+            if (dec->probe_host[slot] >= B) break;           // everything retired kWindow steps ago: the steps in between did nothing
+        }
         const int rows_ub = alive[s];
         if (dec->use_graphs && !dec->profiling) {
             // grids are sized for the bucket; kernels leave rows beyond the device-side row count alone
@@ -1270,6 +1288,11 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
             AED_TRY(enqueue_greedy_step(dec, rows_ub, s + 1, tokens_out, out_lens));
         }
         dec->steps_issued = s + 1;
+        if (probe) {
+            const int slot = s % aed_dec::kProbeSlots;
+            AED_CUDA(dec, cudaMemcpyAsync(&dec->probe_host[slot], &dec->state()->n_retired, sizeof(int32_t), cudaMemcpyDeviceToHost, dec->stream));
+            AED_CUDA(dec, cudaEventRecord(dec->probe_event[slot], dec->stream));
+        }
     }
     dec->full_steps = dec->cfg.max_dec_len;   // every utterance is retired: further steps are refused
     return aed_dec_sync_status(dec);
@@ -1336,6 +1359,8 @@ extern "C" void aed_dec_destroy(aed_dec_t *dec)
     for (cudaEvent_t e : dec->prof_events) cudaEventDestroy(e);
     for (auto &g : dec->graphs) cudaGraphExecDestroy(g.second.exec);
     if (dec->capture_stream) cudaStreamDestroy(dec->capture_stream);
+    for (cudaEvent_t e : dec->probe_event) if (e) cudaEventDestroy(e);
+    if (dec->probe_host) cudaFreeHost(dec->probe_host);
     delete dec;
 }
 

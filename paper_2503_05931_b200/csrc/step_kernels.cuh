@@ -923,6 +923,7 @@ __global__ void finish_step_kernel(DecState *state, const int32_t *__restrict__ 
         if (t + 1 >= max_len[u] || (eos_id >= 0 && tok == eos_id)) {
             retired[u] = 1;
             out_lens[u] = t + 1;
+            atomicAdd(&state->n_retired, 1);          // the host polls this to stop issuing steps once every utterance is done
         }
     }
 }

@@ -139,6 +139,37 @@ def test_eos_stops_an_utterance(dtype):
     assert stopped_early > 0
 
 
+def test_eos_ends_the_decode_early():
+    """When every utterance has emitted the end-of-sequence id, the greedy loop stops issuing steps (the host follows
+    the device's retired count a few steps behind) instead of replaying all max_len of them."""
+    b = _binding()
+    for seed in range(13, 80):
+        w = wl.make_custom(SMALL, [12, 20, 7, 33, 5], [200] * 5, dtype="bf16", seed=seed, out_std=0.3)
+        probe = wl.make_custom(SMALL, [12, 20, 7, 33, 5], [8] * 5, dtype="bf16", seed=seed, out_std=0.3)
+        free = oracle_reference(probe, want_logits=False)
+        eos = int(free["next"][0, 3])
+        cut = oracle_reference(probe, want_logits=False, eos=eos)
+        if np.all(cut["lens"] < 8) and all(np.min(cut["margin"][u, :cut["lens"][u]]) > MARGIN for u in range(5)):
+            break
+    else:
+        raise AssertionError("no seeded case found")
+    dec = b.decoder_for_workload(w, eos_id=eos)
+    try:
+        dec.precompute_cross_kv(dec.upload_encoder(w.enc), w.enc_lens)
+        before = dec.launch_count()
+        toks, lens = dec.greedy_decode(w.dec_lens)
+        issued = dec.launch_count() - before
+        toks, lens = toks.cpu().numpy(), lens.cpu().numpy()
+    finally:
+        dec.close()
+    assert np.array_equal(lens, cut["lens"])
+    for u in range(5):
+        n = int(lens[u])
+        assert np.array_equal(toks[u, :n], cut["next"][u, :n]) and np.all(toks[u, n:] == -1)
+    per_step = 8 * SMALL["n_layers"] + 5
+    assert issued < 30 * per_step, issued          # 200 steps would be 4200 launches
+
+
 def test_handle_reuse_across_batch_sizes():
     """One handle and one pair of output buffers decode batches of 12, 7 and 12 utterances in turn (the step graphs
     recorded for the first batch are replayed for the others): every batch against the checker."""

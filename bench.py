@@ -83,8 +83,8 @@ def family_bytes(family, w):
     return None
 
 
-# Which kernel a launch family runs (the library times launches per call site; the six projections of a layer are
-# six call sites of one kernel).
+# Which kernel a launch family runs (the library times launches per call site; the projections of a layer are
+# five or six call sites of one kernel).
 KERNEL_OF_FAMILY = {
     "gemm_qkv": "step_gemm_kernel", "gemm_o": "step_gemm_kernel", "gemm_qc": "step_gemm_kernel",
     "gemm_oc": "step_gemm_kernel", "gemm_ff1": "step_gemm_kernel", "gemm_ff2": "step_gemm_kernel",
@@ -459,6 +459,9 @@ def profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step):
         k = kernels.setdefault(KERNEL_OF_FAMILY.get(fam, fam), {"ms": 0.0, "launches": 0, "bytes": 0.0, "families": []})
         k["ms"] += v["ms"]; k["launches"] += v["launches"]; k["families"].append(fam)
         k["bytes"] += family_bytes(fam, w) or 0.0
+    if "gemm_qkv" in prof and "gemm_qc" not in prof:
+        # steps of at most 128 rows: the cross-attention query matrix is read by the launch that reads Wqkv
+        kernels["step_gemm_kernel"]["bytes"] += family_bytes("gemm_qc", w) or 0.0
     top = max(kernels, key=lambda k: kernels[k]["ms"])
     info = kernels[top]
     share = info["ms"] / total

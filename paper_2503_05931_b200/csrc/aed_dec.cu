@@ -51,6 +51,7 @@ struct Layout {
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
     size_t actd_hi, actd_lo, actf_hi, actf_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
+    size_t comp_w, comp_b;                // per layer: Wqc diag(gamma2) Wo as bf16 [d, d], and Wqc (gamma2 * bo) as fp32 [d]
     size_t ckv_maps, ckv_bias;            // per-layer tensor maps and bias pointers of the cross-K/V weights
     size_t fold_layer_floats;
     int rows_cap;
@@ -124,6 +125,8 @@ Layout make_layout(const aed_dec_config_t &c)
         L.qc = take(B * d * 4);
         L.ckv_maps = take((size_t)c.n_layers * sizeof(CUtensorMap));
         L.ckv_bias = take((size_t)c.n_layers * sizeof(void *));
+        L.comp_w = take((size_t)c.n_layers * d * d * 2);
+        L.comp_b = take((size_t)c.n_layers * d * 4);
     }
     L.total = off;
     return L;
@@ -155,7 +158,7 @@ struct aed_dec {
     std::vector<int> prof_family;                  // family of each recorded launch
     size_t prof_used = 0;
     // bf16 mode: TMA descriptors of the weight matrices and of the activation planes (one per MMA N in 16..256)
-    struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2; };
+    struct TcLayerMaps { CUtensorMap qkv, o, qc, oc, ff1, ff2, o_qc; };      // o_qc: the composite Wqc diag(gamma2) Wo
     std::vector<TcLayerMaps> tc_layers;
     CUtensorMap tc_w_out;
     CUtensorMap tc_actd[5][2], tc_actf[5][2];     // [log2(N/16)][plane]: activation planes [rows, d] and [rows, F]
@@ -304,7 +307,7 @@ template <typename T, bool kCross, bool kAppend>
 aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const float *q, int ldq, const T *cache,
                                     int seq_capacity, float *out, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo,
                                     const float2 *ln_stats = nullptr, const float *ln_c1 = nullptr,
-                                    const float *ln_c2 = nullptr, bool pdl = false)
+                                    const float *ln_c2 = nullptr, bool pdl = false, const float *stats_x = nullptr)
 {
     ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
     int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
@@ -324,10 +327,13 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
     // Few blocks with long rows (late steps): the software-pipelined variant, two blocks per SM hold the whole grid.
     const bool pipe = kCross && !kAppend && rows_ub * dec->cfg.n_heads <= 2 * dec->sm_count && dec->attn_pipe;
     auto kernel = pipe ? attn_fused_kernel<T, kCross, kAppend, kCross && !kAppend> : attn_fused_kernel<T, kCross, kAppend, false>;
+    if constexpr (kCross && !kAppend) {
+        if (stats_x) kernel = pipe ? attn_fused_kernel<T, true, false, true, true> : attn_fused_kernel<T, true, false, false, true>;
+    }
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, (const DecState *)dec->state(),
                                        (const int4 *)dec->at<int4>(dec->lay.row_info), q, ldq, const_cast<T *>(cache),
                                        dec->cfg.n_heads, seq_capacity, 1.0f / sqrtf((float)kHeadDim), out, out_hi, out_lo,
-                                       dec->cfg.d_model, ln_stats, ln_c1, ln_c2);
+                                       dec->cfg.d_model, ln_stats, ln_c1, ln_c2, stats_x, dec->cfg.ln_eps);
     if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
     AED_LAUNCHED(dec);
     return AED_OK;
@@ -470,7 +476,8 @@ aed_status_t tc_setup(aed_dec *dec)
         ok = ok && encode_map(&m.qkv, w.w_qkv, 3 * d, d, tc::kTileM) && encode_map(&m.o, w.w_o, d, d, tc::kTileM) &&
              encode_map(&m.qc, w.w_q_c, d, d, tc::kTileM) && encode_map(&m.oc, w.w_o_c, d, d, tc::kTileM) &&
              encode_map(&m.ff1, w.w_ff1, F, d, tc::kTileM) && encode_map(&m.ff2, w.w_ff2, d, F, tc::kTileM) &&
-             encode_map(&kvc_maps[l], w.w_kv_c, 2 * d, c.d_enc, ckv::kTileN);
+             encode_map(&kvc_maps[l], w.w_kv_c, 2 * d, c.d_enc, ckv::kTileN) &&
+             encode_map(&m.o_qc, dec->ws + L.comp_w + (size_t)l * d * d * 2, d, d, tc::kTileM);
         kvc_bias[l] = w.b_kv_c;
     }
     ok = ok && encode_map(&dec->tc_w_out, dec->w_out, c.vocab, d, tc::kTileM);
@@ -513,7 +520,14 @@ aed_status_t tc_setup(aed_dec *dec)
                                                                            (const T *)w.b_q_c, (int)d, (int)d, fc + 6 * d, fc + 7 * d);
         sg::ln_fold_constants_kernel<<<(F + 7) / 8, 256, 0, dec->stream>>>((const T *)w.w_ff1, (const T *)w.ln3_g, (const T *)w.ln3_b,
                                                                            (const T *)w.b_ff1, (int)F, (int)d, fc + 8 * d, fc + 8 * d + F);
-        dec->launches += 3;
+        // The self-attention output projection and the cross-attention query projection meet without a nonlinearity:
+        // their composite lets one launch run both (see forward_step_fused).
+        T *cw = dec->at<T>(L.comp_w) + (size_t)l * d * d;
+        float *cb = dec->at<float>(L.comp_b) + (size_t)l * d;
+        sg::compose_weights_kernel<<<dim3((unsigned)((d + 15) / 16), (unsigned)((d + 15) / 16)), 256, 0, dec->stream>>>(
+            (const T *)w.w_q_c, (const T *)w.ln2_g, (const T *)w.w_o, (int)d, cw);
+        sg::compose_bias_kernel<<<(d + 7) / 8, 256, 0, dec->stream>>>((const T *)w.w_q_c, (const T *)w.ln2_g, (const T *)w.b_o, (int)d, cb);
+        dec->launches += 5;
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "fold constants: %s", cudaGetErrorString(e));
@@ -586,7 +600,7 @@ aed_status_t launch_ln_planes(aed_dec *dec, int rows_ub, const float *x, const v
     return launch_pdl_impl(dec, (const void *)layernorm_planes_kernel<8>, dim3(rows_ub), dim3(d <= 2048 ? 256 : 1024), 0, args);
 }
 
-// ---- fused step (bf16 mode): 8 kernels per layer, chained with programmatic dependent launch -------------------
+// ---- fused step (bf16 mode): 7 kernels per layer, chained with programmatic dependent launch -------------------
 
 struct FusedGemm {
     const CUtensorMap *map;
@@ -595,8 +609,10 @@ struct FusedGemm {
 
 template <int MODE>
 aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w, const CUtensorMap *src_maps, int M,
-                              int K, int rows_ub, sg::StepGemmParams p, const CUtensorMap (*plane_maps)[2] = nullptr)
+                              int K, int rows_ub, sg::StepGemmParams p, const CUtensorMap (*plane_maps)[2] = nullptr,
+                              const CUtensorMap *map_w2 = nullptr, int M2 = 0)
 {
+    // map_w2, M2: a second weight matrix [M2, K] over the same rows (its output, gamma and bias are in p)
     // plane_maps (B_PLANES only): [log2(N/16)][high, low] tensor maps of the ready-made activation planes
     ProfScope ps(dec, family);
     // Rows per CTA tile: up to 128 (two ring stages still fit beside the transposition buffer); more rows are
@@ -604,7 +620,10 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     int ni = tc_n_index(rows_ub);
     if (ni > 3) ni = 3;
     const int n_tile = 16 << ni;
-    const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = (M + tc::kTileM - 1) / tc::kTileM;
+    const int m_tiles1 = (M + tc::kTileM - 1) / tc::kTileM;
+    const int row_tiles = (rows_ub + n_tile - 1) / n_tile, m_tiles = m_tiles1 + (map_w2 ? (M2 + tc::kTileM - 1) / tc::kTileM : 0);
+    p.tiles_first = map_w2 ? m_tiles1 : 0;
+    p.a_rows2 = M2;
     const int k_blocks = K / tc::kBlockK;
     const int stage_bytes = tc::kATileBytes + 2 * n_tile * tc::kBlockK * 2 + (MODE == sg::B_PLANES ? 0 : n_tile * tc::kBlockK * 4);
     int stages = kTcSmemBudget / stage_bytes;
@@ -642,7 +661,7 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
         cfg.dynamicSmemBytes = (size_t)n_tile * (tc::kTileM + 4) * 4 + 1024;
     cudaError_t e = MODE == sg::B_PLANES
                         ? cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, plane_maps[ni][0], plane_maps[ni][1], p)
-                        : cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, src_maps[ni], src_maps[ni], p);
+                        : cudaLaunchKernelEx(&cfg, sg::step_gemm_kernel<MODE>, map_w, src_maps[ni], map_w2 ? *map_w2 : src_maps[ni], p);
     if (e != cudaSuccess) return fail(dec, AED_ERR_CUDA, "projection launch: %s", cudaGetErrorString(e));
     AED_LAUNCHED(dec);
     return AED_OK;
@@ -669,10 +688,11 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         ProfScope ps(dec, KF_EMBED);
         if (pf)
             embed_rows_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), dec->at<int4>(L.row_info), dec->at<int32_t>(L.row_tok),
-                                                                   (const T *)dec->embed, dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
+                                                                   (const T *)dec->embed, dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d,
+                                                                   qc, d);
         else
             embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                              dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d);
+                                                              dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d, qc, d);
         AED_LAUNCHED(dec);
     }
     const bool pdl = dec->use_pdl;
@@ -687,13 +707,15 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         const LayerWeights &wn = dec->layers[(l + 1) % c.n_layers];     // next layer (or layer 0 of the next step)
         const size_t e2 = sizeof(T);
         sg::StepGemmParams p{};
-        // 1. [q | k | v] raw = (gamma1 * x) Wqkv^T ; side: LN1 statistics of x, clear the cross-query rows
+        // 1. [q | k | v] raw = (gamma1 * x) Wqkv^T, and the part of the cross-attention query that this layer's input
+        //    already fixes, q'A raw = (gamma2 * x) Wqc^T (the rest follows in 3) ; side: LN1 statistics of x
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln1_g;
         p.out = qkv; p.ldo = 3 * d; p.bias = nullptr;
+        p.gamma2 = (const T *)w.ln2_g; p.out2 = qc; p.ldo2 = d; p.bias2 = nullptr;
         p.stats_src = x; p.stats_out = stats; p.stats_d = d;
-        p.zero_buf = qc; p.zero_cols = d;
         p.prefetch_ptr = wn.w_qkv; p.prefetch_bytes = (size_t)3 * d * d * e2;
-        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p));
+        p.prefetch2_ptr = wn.w_q_c; p.prefetch2_bytes = (size_t)d * d * e2;
+        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p, nullptr, &m.qc, d));
         // 2. self-attention (applies LN1 to q, k, v; appends k, v)
         if (pf) {
             {
@@ -712,31 +734,28 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
             AED_TRY((launch_attention_fused<T, false, true>(dec, rows_ub, self_len_ub, qkv, 3 * d, self_cache, c.max_dec_len, att,
                                                             nullptr, nullptr, stats, c1_qkv, c2_qkv, pdl)));
         }
-        // 3. x += att Wo^T + bo ; side: clear the FFN hidden rows
+        // 3. x += att Wo^T + bo, and in the same launch the rest of the cross-attention query:
+        //    (gamma2 * x_new) Wqc^T = q'A + att (Wqc diag(gamma2) Wo)^T + Wqc (gamma2 * bo), so the query projection does
+        //    not wait for the sum over all features of x_new ; side: clear the FFN hidden rows
         p = sg::StepGemmParams{};
         p.src = att; p.ld_src = d;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o;
+        p.out2 = qc; p.ldo2 = d; p.bias2 = dec->at<float>(L.comp_b) + (size_t)l * d;
         p.zero_buf = hid; p.zero_cols = F;
         p.prefetch_ptr = wn.w_o; p.prefetch_bytes = (size_t)d * d * e2;
-        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, dec->tc_src_att, d, d, rows_ub, p));
-        // 4. q' raw = (gamma2 * x) Wqc^T ; side: LN2 statistics
-        p = sg::StepGemmParams{};
-        p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln2_g;
-        p.out = qc; p.ldo = d;
-        p.stats_src = x; p.stats_out = stats + stats_stride; p.stats_d = d;
-        p.prefetch_ptr = wn.w_q_c; p.prefetch_bytes = (size_t)d * d * e2;
-        AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QC, m.qc, dec->tc_src_x, d, d, rows_ub, p));
-        // 5. cross-attention
+        p.prefetch2_ptr = dec->at<T>(L.comp_w) + (size_t)((l + 1) % c.n_layers) * d * d; p.prefetch2_bytes = (size_t)d * d * e2;
+        AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, dec->tc_src_att, d, d, rows_ub, p, nullptr, &m.o_qc, d));
+        // 4. cross-attention; every block computes the LN2 statistics of its row of x_new itself
         AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
-                                                        nullptr, nullptr, stats + stats_stride, c1_qc, c2_qc, pdl)));
-        // 6. x += att Woc^T + boc ; side: clear the [q | k | v] rows for the next layer
+                                                        nullptr, nullptr, nullptr, c1_qc, c2_qc, pdl, x)));
+        // 5. x += att Woc^T + boc ; side: clear the [q | k | v] rows for the next layer
         p = sg::StepGemmParams{};
         p.src = att; p.ld_src = d;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
         p.zero_buf = qkv; p.zero_cols = 3 * d;
         p.prefetch_ptr = wn.w_o_c; p.prefetch_bytes = (size_t)d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_OC, m.oc, dec->tc_src_att, d, d, rows_ub, p));
-        // 7. hidden raw = (gamma3 * x) W1^T ; side: LN3 statistics
+        // 6. hidden raw = (gamma3 * x) W1^T ; side: LN3 statistics
         p = sg::StepGemmParams{};
         p.src = x; p.ld_src = d; p.gamma = (const T *)w.ln3_g;
         p.out = hid; p.ldo = F;
@@ -744,10 +763,11 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.prefetch_ptr = wn.w_ff1; p.prefetch_bytes = (size_t)F * d * e2;
         if (l == c.n_layers - 1) { p.prefetch2_ptr = dec->w_out; p.prefetch2_bytes = (size_t)V * d * e2; }    // the vocabulary projection is next
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, dec->tc_src_x, F, d, rows_ub, p));
-        // 8. x += relu(LN3-corrected hidden) W2^T + b2
+        // 7. x += relu(LN3-corrected hidden) W2^T + b2 ; side: clear the cross-query rows
         p = sg::StepGemmParams{};
         p.src = hid; p.ld_src = F; p.c1 = c1_ff; p.c2 = c2_ff; p.stats_in = stats + 2 * stats_stride;
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_ff2;
+        p.zero_buf = qc; p.zero_cols = d;          // the next layer's first launch accumulates into it
         p.prefetch_ptr = wn.w_ff2; p.prefetch_bytes = (size_t)F * d * e2;
         AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, dec->tc_src_hid, d, F, rows_ub, p));
     }

@@ -61,13 +61,17 @@ __device__ __forceinline__ TraceCursor trace_reserve(const DecState *state, uint
     }
     return c;
 }
+// The SM's cycle counter (low 32 bits) goes with every mark; the global nanosecond timer, which costs a few hundred
+// nanoseconds to read, only where asked for (the first mark of a kernel, to place it on the common axis).
+template <bool kWallClock>
 __device__ __forceinline__ void trace_put(const DecState *state, TraceCursor &c, uint32_t id)
 {
     if (c.next < c.end) {
         TraceBuf *tb = reinterpret_cast<TraceBuf *>(reinterpret_cast<char *>(const_cast<DecState *>(state)) + 256);
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        unsigned long long t = 0;
+        if (kWallClock) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         tb->ev[c.next].id = id;
+        tb->ev[c.next].pad = static_cast<uint32_t>(clock64());
         tb->ev[c.next].t_ns = t;
         ++c.next;
     }
@@ -75,12 +79,14 @@ __device__ __forceinline__ void trace_put(const DecState *state, TraceCursor &c,
 #define AED_TRACE_BEGIN(state, id) trace_begin(state, id)
 #define AED_TRACE_MARK(state, id) trace_mark(state, id)
 #define AED_TRACE_RESERVE(cur, state, n) TraceCursor cur = trace_reserve(state, n)
-#define AED_TRACE_PUT(state, cur, id) trace_put(state, cur, id)
+#define AED_TRACE_PUT(state, cur, id) trace_put<false>(state, cur, id)
+#define AED_TRACE_PUT_NS(state, cur, id) trace_put<true>(state, cur, id)
 #else
 #define AED_TRACE_BEGIN(state, id) ((void)0)
 #define AED_TRACE_MARK(state, id) ((void)0)
 #define AED_TRACE_RESERVE(cur, state, n) ((void)0)
 #define AED_TRACE_PUT(state, cur, id) ((void)0)
+#define AED_TRACE_PUT_NS(state, cur, id) ((void)0)
 #endif
 
 __device__ __forceinline__ float to_f32(float v) { return v; }

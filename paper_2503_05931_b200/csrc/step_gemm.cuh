@@ -19,6 +19,10 @@
 // run, the producer warps of this kernel compute mean and rstd of the rows assigned to their CTA and store
 // them for the consumer.  A second side job clears the fp32 rows a later split-K projection accumulates into.
 //
+// Two matrices in one launch (not in B_PLANES mode): feature tiles blockIdx.x >= tiles_first belong to a second weight
+// matrix over the same activation rows, with its own tensor map (passed in the place of the low plane's), gamma,
+// bias and output buffer.  This is how one launch serves two projections that depend on the same earlier kernel.
+//
 // A CTA walks its k-blocks through a ring of up to 4 stages (weight tile, two planes, fp32 source tile each); with
 // few k-blocks per CTA (small batches, many k-splits) everything is resident at once.  Waits are bounded.
 #pragma once
@@ -50,6 +54,13 @@ struct StepGemmParams {
     float *out;
     int ldo;
     const __nv_bfloat16 *bias;     // added by k-split 0, may be null
+    // second matrix (feature tiles tiles_first .. gridDim.x - 1); tiles_first == 0: none
+    int tiles_first;
+    int a_rows2;
+    const __nv_bfloat16 *gamma2;   // B_GAMMA
+    float *out2;
+    int ldo2;
+    const float *bias2;            // fp32, added by k-split 0, may be null
     // side job 1: (mean, rstd) of the rows of stats_src [rows, stats_d]
     const float *stats_src;
     float2 *stats_out;
@@ -114,10 +125,13 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     __shared__ float red_s[2], red_q[2];
 
     // timeline of the first producer thread of block 0 (debug builds)
-    AED_TRACE_RESERVE(tcur, p.state, (threadIdx.x == 64 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? 8u : 0u);
-    AED_TRACE_PUT(p.state, tcur, 19);
+    AED_TRACE_RESERVE(tcur, p.state, (threadIdx.x == 64 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? 10u : 0u);
+    AED_TRACE_PUT_NS(p.state, tcur, 19);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int a0 = blockIdx.x * kTileM;
+    const bool second_w = MODE != B_PLANES && p.tiles_first > 0 && static_cast<int>(blockIdx.x) >= p.tiles_first;
+    const CUtensorMap *mw = second_w ? &map_lo : &map_w;
+    const int a0 = (second_w ? static_cast<int>(blockIdx.x) - p.tiles_first : static_cast<int>(blockIdx.x)) * kTileM;
+    const int a_rows = second_w ? p.a_rows2 : p.a_rows;
     const int row0 = blockIdx.z * p.n_tile;
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
@@ -150,12 +164,12 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 
     if (warp == 0) {
         if (lane == 0) {
-            prefetch_tensormap(&map_w);
+            prefetch_tensormap(mw);
             prefetch_tensormap(&map_src);
             const int pre = n_kb < S ? n_kb : S;
             for (int i = 0; i < pre; ++i) {       // weights: independent of every earlier kernel
                 mbar_expect_tx(&bar_a[i], kATileBytes);
-                tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[i]);
+                tma_load_2d(tiles + static_cast<size_t>(i) * stage_bytes, mw, (kb_begin + i) * kBlockK, a0, &bar_a[i]);
             }
         }
         pdl_wait();
@@ -166,7 +180,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 if (i >= S) {                     // the stage is free once the MMAs of k-block i - S have read it
                     if (!mbar_wait(&bar_e[s], ((i / S) - 1) & 1, &abort_flag)) break;
                     mbar_expect_tx(&bar_a[s], kATileBytes);
-                    tma_load_2d(stage, &map_w, (kb_begin + i) * kBlockK, a0, &bar_a[s]);
+                    tma_load_2d(stage, mw, (kb_begin + i) * kBlockK, a0, &bar_a[s]);
                 }
                 // fp32 activation source, written by the previous kernels
                 if (MODE != B_PLANES && !direct) {
@@ -279,8 +293,15 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const int c = pt & 7, rbase = pt >> 3;
         const int quarter = warp & 3;
         const int a_idx = a0 + quarter * 32 + lane;
-        const bool a_ok = a_idx < p.a_rows;
-        const float bias = (p.bias && blockIdx.y == 0 && a_ok) ? to_f32(p.bias[a_idx]) : 0.f;
+        const bool a_ok = a_idx < a_rows;
+        float bias = 0.f;
+        if (blockIdx.y == 0 && a_ok) {
+            if (second_w) bias = p.bias2 ? p.bias2[a_idx] : 0.f;
+            else bias = p.bias ? to_f32(p.bias[a_idx]) : 0.f;
+        }
+        float *const out = second_w ? p.out2 : p.out;
+        const int ldo = second_w ? p.ldo2 : p.ldo;
+        const __nv_bfloat16 *const gamma = second_w ? p.gamma2 : p.gamma;
         float dv[2][8];
         if (direct && rbase < p.n_tile) {          // one row per thread (n_tile <= 32), both k-blocks requested at once
             const int rs = min(row0 + rbase, p.src_rows - 1);
@@ -296,7 +317,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
             const float *src_tile = reinterpret_cast<const float *>(lo_tile + plane_bytes);
             const int k = (kb_begin + i) * kBlockK + c * 8;
             float g[8], c1[8], c2[8];
-            if (MODE == B_GAMMA) load8(p.gamma + k, g);
+            if (MODE == B_GAMMA) load8(gamma + k, g);
             if (MODE == B_LN_RELU) { load8(p.c1 + k, c1); load8(p.c2 + k, c2); }
             if (!direct) ok = mbar_wait(&bar_s[s], (i / S) & 1, &abort_flag);
             if (!ok) break;
@@ -353,17 +374,19 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 for (int j = 0; j < 16; ++j) trans[(c0 + j) * kPitch + quarter * 32 + lane] = v[j] + bias;
             }
         }
+        AED_TRACE_PUT(p.state, tcur, 46);  // accumulator in shared memory
         asm volatile("bar.sync 2, 256;" ::: "memory");
+        AED_TRACE_PUT(p.state, tcur, 47);  // all epilogue warps there
         if (ok && fits) {
             const int o4 = (pt & 31) * 4;
             for (int rl = pt >> 5; rl < rows_here; rl += 8) {
                 const float4 v = *reinterpret_cast<const float4 *>(trans + rl * kPitch + o4);
-                float *dst = p.out + static_cast<size_t>(row0 + rl) * p.ldo + a0 + o4;
-                if (a0 + o4 + 3 < p.a_rows) red_add_v4(dst, v);
+                float *dst = out + static_cast<size_t>(row0 + rl) * ldo + a0 + o4;
+                if (a0 + o4 + 3 < a_rows) red_add_v4(dst, v);
                 else {
-                    if (a0 + o4 + 0 < p.a_rows) atomicAdd(dst + 0, v.x);
-                    if (a0 + o4 + 1 < p.a_rows) atomicAdd(dst + 1, v.y);
-                    if (a0 + o4 + 2 < p.a_rows) atomicAdd(dst + 2, v.z);
+                    if (a0 + o4 + 0 < a_rows) atomicAdd(dst + 0, v.x);
+                    if (a0 + o4 + 1 < a_rows) atomicAdd(dst + 1, v.y);
+                    if (a0 + o4 + 2 < a_rows) atomicAdd(dst + 2, v.z);
                 }
             }
         } else if (ok) {
@@ -374,12 +397,12 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 tmem_ld16(taddr + c0, v);
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    if (a_ok && c0 + j < rows_here) atomicAdd(p.out + static_cast<size_t>(row0 + c0 + j) * p.ldo + a_idx, v[j] + bias);
+                    if (a_ok && c0 + j < rows_here) atomicAdd(out + static_cast<size_t>(row0 + c0 + j) * ldo + a_idx, v[j] + bias);
             }
         }
         }
     }
-    AED_TRACE_PUT(p.state, tcur, 45);      // epilogue issued
+    AED_TRACE_PUT_NS(p.state, tcur, 45);   // epilogue issued
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -405,6 +428,41 @@ __global__ void ln_fold_constants_kernel(const __nv_bfloat16 *__restrict__ w, co
     s1 = warp_sum(s1);
     s2 = warp_sum(s2);
     if (lane == 0) { c1[o] = s1; c2[o] = s2 + (bias ? to_f32(bias[o]) : 0.f); }
+}
+
+// Two projections that meet without a nonlinearity between them, composed once at set-up:
+//   C[o][i] = sum_k A[o][k] g[k] B[k][i]   (bf16, row-major [n, n]);   cb[o] = sum_k A[o][k] g[k] b[k]
+// so that (g * (x + y B^T + b)) A^T = (g * x) A^T + y C^T + cb: the second projection no longer has to wait for the
+// sum over all features of the first.  16 x 16 outputs per block, fp32 accumulation.
+__global__ void compose_weights_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ g,
+                                       const __nv_bfloat16 *__restrict__ b, int n, __nv_bfloat16 *__restrict__ c)
+{
+    __shared__ float sa[16][17], sb[16][17];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int o = blockIdx.y * 16 + ty, i = blockIdx.x * 16 + tx;
+    float acc = 0.f;
+    for (int k0 = 0; k0 < n; k0 += 16) {
+        const int ka = k0 + tx, kb = k0 + ty;
+        sa[ty][tx] = (o < n && ka < n) ? to_f32(a[static_cast<size_t>(o) * n + ka]) * to_f32(g[ka]) : 0.f;
+        sb[ty][tx] = (kb < n && i < n) ? to_f32(b[static_cast<size_t>(kb) * n + i]) : 0.f;
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) acc = fmaf(sa[ty][k], sb[k][tx], acc);
+        __syncthreads();
+    }
+    if (o < n && i < n) c[static_cast<size_t>(o) * n + i] = __float2bfloat16_rn(acc);
+}
+
+__global__ void compose_bias_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ g,
+                                    const __nv_bfloat16 *__restrict__ b, int n, float *__restrict__ cb)
+{
+    const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (o >= n) return;
+    float s = 0.f;
+    if (b)
+        for (int k = lane; k < n; k += 32) s = fmaf(to_f32(a[static_cast<size_t>(o) * n + k]) * to_f32(g[k]), to_f32(b[k]), s);
+    s = warp_sum(s);
+    if (lane == 0) cb[o] = s;
 }
 
 }  // namespace sg

@@ -75,7 +75,8 @@ template <typename T>
 __global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ active_list,
                              const int32_t *__restrict__ tokens, const int32_t *__restrict__ t_u,
                              const T *__restrict__ embed, const float *__restrict__ pe, int d, int vocab, float scale,
-                             float *__restrict__ x, float *__restrict__ zero_buf = nullptr, int zero_cols = 0)
+                             float *__restrict__ x, float *__restrict__ zero_buf = nullptr, int zero_cols = 0,
+                             float *__restrict__ zero_buf2 = nullptr, int zero_cols2 = 0)
 {
     AED_TRACE_BEGIN(state, 2);
     int r = blockIdx.x;
@@ -87,6 +88,7 @@ __global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ 
     for (int i = threadIdx.x; i < d; i += blockDim.x)
         x[(size_t)r * d + i] = to_f32(embed[(size_t)tok * d + i]) * scale + pe[(size_t)t * d + i];
     for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
+    for (int i = threadIdx.x; i < zero_cols2; i += blockDim.x) zero_buf2[(size_t)r * zero_cols2 + i] = 0.f;
 }
 
 // out[r] = g * (x[r] - mean) / sqrt(var + eps) + b, biased variance, two passes over a row held in registers.
@@ -409,18 +411,23 @@ constexpr int kFusedMaxWarps = 8;
 
 // kPipe: the loads of a warp's next chunk are issued before the current chunk is reduced (twice the K/V registers,
 // so only two blocks per SM: for grids that fit anyway).
-template <typename CT, bool kCross, bool kAppend, bool kPipe = false>
+// kRowStats: the block computes (mean, rstd) of its row of stats_x itself instead of reading ln_stats.
+template <typename CT, bool kCross, bool kAppend, bool kPipe = false, bool kRowStats = false>
 __global__ void __launch_bounds__(kFusedMaxWarps * 32, ((kAppend || kPipe) ? 2 : 4))      // self-attention holds the new key/value as well
 attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ q, int ldq,
                   CT *__restrict__ cache, int n_heads, int seq_capacity, float scale,
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo,
-                  const float2 *__restrict__ ln_stats, const float *__restrict__ ln_c1, const float *__restrict__ ln_c2)
+                  const float2 *__restrict__ ln_stats, const float *__restrict__ ln_c1, const float *__restrict__ ln_c2,
+                  const float *__restrict__ stats_x = nullptr, float ln_eps = 0.f)
 {
+    // stats_x: rows [*, heads * 64] whose (mean, rstd) this block computes itself instead of reading ln_stats (the
+    // kernel before this one completed those rows, so nobody could have computed the statistics earlier).
     // Launched with programmatic stream serialization.  Before the dependency wait only data that no kernel of
     // this step writes is touched: the row table (written by the step's first kernel, which ran to completion
     // before any programmatic launch of the step) and, for cross-attention, the encoder K/V store.
     __shared__ float sm_m[kFusedMaxWarps], sm_l[kFusedMaxWarps];
     __shared__ float sm_acc[kFusedMaxWarps][kHeadDim];
+    __shared__ float2 sm_red[kFusedMaxWarps];
     const int rh = blockIdx.x;
     const int r = rh / n_heads, h = rh % n_heads;
     const int4 ri = row_info[r];                       // (utterance, t_u, encoder length, encoder offset)
@@ -479,7 +486,8 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     const int d_model = n_heads * kHeadDim;
     const int qcol = h * kHeadDim + dg * 8;
     float qc1[8], qc2[8], kc1[8], kc2[8], vc1[8], vc2[8];
-    if (ln_stats) {
+    const bool fold = ln_stats != nullptr || kRowStats;
+    if (fold) {
         load8(ln_c1 + qcol, qc1); load8(ln_c2 + qcol, qc2);
         if (owns_new) {
             load8(ln_c1 + d_model + qcol, kc1); load8(ln_c2 + d_model + qcol, kc2);
@@ -487,7 +495,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         }
     }
     AED_TRACE_RESERVE(tcur, state, (threadIdx.x == 0 && blockIdx.x == 0) ? 4u : 0u);
-    AED_TRACE_PUT(state, tcur, 8 + (kCross ? 1 : 0));      // resident, first chunk requested
+    AED_TRACE_PUT_NS(state, tcur, 8 + (kCross ? 1 : 0));      // resident, first chunk requested
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     AED_TRACE_PUT(state, tcur, 3);                          // dependency resolved
@@ -502,7 +510,29 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         load8(q + (size_t)r * ldq + d_model + qcol, kn);
         load8(q + (size_t)r * ldq + 2 * d_model + qcol, vn);
     }
-    if (ln_stats) {
+    if (kRowStats) {
+        // mean and rstd of row r in one pass over deviations from the row's first element (a row whose mean is far
+        // from zero loses nothing to cancellation that way): var = (S2 - S1^2 / n) / n, mean = x0 + S1 / n
+        const float *xr = stats_x + (size_t)r * d_model;
+        const float x0 = xr[0];
+        float s1 = 0.f, s2 = 0.f;
+        for (int idx = threadIdx.x * 4; idx < d_model; idx += blockDim.x * 4) {
+            const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+            const float d0 = v.x - x0, d1 = v.y - x0, d2 = v.z - x0, d3 = v.w - x0;
+            s1 += (d0 + d1) + (d2 + d3);
+            s2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+        }
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        if (lane == 0) sm_red[warp] = make_float2(s1, s2);
+        __syncthreads();
+        float t1 = 0.f, t2 = 0.f;
+        for (int w = 0; w < n_warps; ++w) { t1 += sm_red[w].x; t2 += sm_red[w].y; }
+        const float inv_n = 1.f / d_model;
+        const float var = fmaxf((t2 - t1 * t1 * inv_n) * inv_n, 0.f);
+        st = make_float2(x0 + t1 * inv_n, rsqrtf(var + ln_eps));
+    }
+    if (fold) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * qc1[i], qc2[i]);
     }
@@ -510,7 +540,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     for (int i = 0; i < 8; ++i) qv[i] *= scale;
     Raw8<CT> new_k, new_v;
     if (owns_new) {
-        if (ln_stats) {
+        if (fold) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 kn[i] = fmaf(st.y, kn[i] - st.x * kc1[i], kc2[i]);
@@ -626,7 +656,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             out_lo[off] = __float2bfloat16_rn(o - __bfloat162float(hi));
         }
     }
-    AED_TRACE_PUT(state, tcur, 7);                          // output written
+    AED_TRACE_PUT_NS(state, tcur, 7);                       // output written
 }
 
 // Merge the chunk partials of each (row, head): one warp per pair, 2 head dimensions per lane.
@@ -843,7 +873,8 @@ __global__ void build_prefill_rows_kernel(DecState *state, int chunk, int j0, in
 template <typename T>
 __global__ void embed_rows_kernel(const DecState *state, const int4 *__restrict__ row_info, const int32_t *__restrict__ row_tok,
                                   const T *__restrict__ embed, const float *__restrict__ pe, int d, int vocab, float scale,
-                                  float *__restrict__ x, float *__restrict__ zero_buf, int zero_cols)
+                                  float *__restrict__ x, float *__restrict__ zero_buf, int zero_cols,
+                                  float *__restrict__ zero_buf2 = nullptr, int zero_cols2 = 0)
 {
     const int r = blockIdx.x;
     if (r >= state->n_active) return;
@@ -851,6 +882,7 @@ __global__ void embed_rows_kernel(const DecState *state, const int4 *__restrict_
     for (int i = threadIdx.x; i < d; i += blockDim.x)
         x[(size_t)r * d + i] = to_f32(embed[(size_t)tok * d + i]) * scale + pe[(size_t)t * d + i];
     for (int i = threadIdx.x; i < zero_cols; i += blockDim.x) zero_buf[(size_t)r * zero_cols + i] = 0.f;
+    for (int i = threadIdx.x; i < zero_cols2; i += blockDim.x) zero_buf2[(size_t)r * zero_cols2 + i] = 0.f;
 }
 
 // Keys and values of every row into the self-attention cache (raw projection output with the LayerNorm fold applied,

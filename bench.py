@@ -241,9 +241,10 @@ def cpu_baseline(w, budget_tokens: int = 0):
 
 
 def run_stream(args):
-    """cfg5: the same 4096 utterances decoded as random batches of 128 and as 2D buckets on (encoder length,
-    output length), 8 x 4 quantile bins with a 64k frame+token budget per batch.  Reports padding fractions,
-    tokens/s and RTFx of both arms in one JSON line (value = the bucketed arm)."""
+    """cfg5: the same 4096 utterances decoded as random batches of 128, as 2D buckets on (encoder length, output
+    length) (8 x 4 quantile bins with a 64k frame+token budget per batch; the paper's 30 x 2 bins), and through 128
+    continuously refilled slots in random arrival order.  Reports padding fractions, tokens/s and RTFx of every arm in
+    one JSON line (value = the 8 x 4 bucketed arm)."""
     import torch
     from paper_2503_05931_b200 import binding, bucketing
 
@@ -265,8 +266,9 @@ def run_stream(args):
             "bucketed8x4": bucketing.bucket_batches_2d(w.enc_lens, w.dec_lens),
             "bucketed30x2": paper_batches}
     all_batches = [b for bs in arms.values() for b in bs]
-    dec = binding.Decoder(w.model, w.weights, w.dtype, max_batch=max(len(b) for b in all_batches),
-                          max_total_enc_frames=max(int(w.enc_lens[b].sum()) for b in all_batches),
+    slot_counts = (128, 256)
+    dec = binding.Decoder(w.model, w.weights, w.dtype, max_batch=max(max(slot_counts), max(len(b) for b in all_batches)),
+                          max_total_enc_frames=max(max(slot_counts) * int(w.enc_lens.max()), max(int(w.enc_lens[b].sum()) for b in all_batches)),
                           max_enc_len=int(w.enc_lens.max()), max_dec_len=int(w.dec_lens.max()), bos_id=w.bos_id,
                           eos_id=w.eos_id, ln_eps=w.ln_eps, device=device)
     enc_all = torch.from_numpy(w.enc).to(device).to(dec.tdtype)
@@ -301,6 +303,38 @@ def run_stream(args):
                         "roofline_ms": 1e3 * roof, "roofline_frac": 1e3 * roof / ms,
                         "gpu_launches": int((dec.launch_count() - launches0) / args.steps)}
         del packed
+    # continuous batching: no sorting by lengths that a server does not know; a slot is refilled when its utterance ends
+    arrival = np.random.default_rng(6).permutation(w.batch)
+    host_toks = torch.empty((w.batch, dec.max_dec_len), dtype=torch.int32).pin_memory()
+    host_lens = torch.zeros(w.batch, dtype=torch.int32).pin_memory()
+    per_step, pre_bytes, pre_flops, step_params = step_bytes_and_flops(w)
+    e = 2 if w.dtype == "bf16" else 4
+    bw, fl = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    kv_bytes = sum(b - e * step_params for b, _, _ in per_step)
+    for slots in slot_counts:
+        stats = {}
+        def run_slots():
+            _, _, steps, row_steps = dec.decode_stream(enc_all, w.enc_lens, w.dec_lens, slots, order=arrival, tokens_out=host_toks,
+                                                       out_lens=host_lens)
+            stats.update({"steps": steps, "row_steps": row_steps})
+        run_slots()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = dec.launch_count()
+        e0.record()
+        for _ in range(args.steps):
+            run_slots()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        assert np.array_equal(host_lens.numpy(), w.dec_lens)
+        # roofline of this schedule: the step weights once per issued step, every (utterance, position)'s K/V once, and
+        # the precompute of every utterance
+        roof = (stats["steps"] * e * step_params + kv_bytes) / bw + max(pre_bytes / bw, pre_flops / fl)
+        result[f"slots{slots}"] = {"slots": slots, "steps": stats["steps"], "occupancy": stats["row_steps"] / (stats["steps"] * slots),
+                                   "ms": ms, "tokens_per_s": float(w.dec_lens.sum()) / (ms * 1e-3), "rtfx": w.audio_seconds / (ms * 1e-3),
+                                   "roofline_ms": 1e3 * roof, "roofline_frac": 1e3 * roof / ms,
+                                   "gpu_launches": int((dec.launch_count() - launches0) / args.steps)}
     dec.sync_status()
     dec.close()
     best = result["bucketed8x4"]

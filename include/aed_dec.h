@@ -198,6 +198,56 @@ size_t aed_dec_static_scratch_bytes(void);
  */
 aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max_len, int32_t *tokens_out, int32_t *out_lens);
 
+/*
+ * Continuous batching: instead of one batch that thins out until its longest utterance ends, the handle keeps a fixed
+ * number of slots, and a new utterance enters a slot as soon as the previous one has left it, so every step runs with
+ * (nearly) all rows occupied.  The paper counts padded positions as wasted computation (Introduction; "Methods",
+ * bucketing) and shows the spread of output lengths per second of audio (Fig. "tpsdist"); the tail of a static batch
+ * is the decoder-side form of that waste.  An utterance's tokens do not depend on what else is in the batch.
+ *
+ * aed_dec_open_slots: replaces the current batch by `slots` empty slots (1..max_batch).  Slot s owns rows
+ *   s * max_enc_len .. (s + 1) * max_enc_len - 1 of the cross-K/V store, so slots * max_enc_len <= max_total_enc_frames
+ *   is required (AED_ERR_CAPACITY otherwise).
+ * aed_dec_admit: a new utterance takes slot `slot` (empty, or left by an utterance that is finished): the cross-K/V of
+ *   its frames is computed into the slot's rows (step A0 for one utterance), its position returns to 0 with the start
+ *   token, and out_lens[slot] is set to 0 if out_lens is not NULL.
+ *     enc      DEVICE [enc_len, d_enc] row-major, config dtype, 16-byte aligned; read during the call's kernels only
+ *     enc_len  1..max_enc_len;  max_len 1..max_dec_len (forced length, an upper bound when eos_id >= 0)
+ *   Without an end-of-sequence id a slot whose utterance still decodes is refused (AED_ERR_STATE); with one the
+ *   caller must have seen out_lens[slot] > 0 first.
+ * aed_dec_greedy_steps: up to n_steps greedy steps over the occupied slots (fewer when the host already knows that no
+ *   slot decodes any more; *steps_done, if not NULL, receives the number issued).  Tokens and lengths are written as by
+ *   aed_dec_greedy_decode, indexed by slot: tokens_out DEVICE int32 [slots, max_dec_len], out_lens DEVICE int32
+ *   [slots]; out_lens[slot] becomes the utterance's length in the step that retires it, which is how the caller
+ *   learns that the slot is free (copy its tokens out before admitting the next utterance).  Entries of tokens_out
+ *   beyond an utterance's length keep whatever an earlier occupant left there.  Does not synchronise.
+ * aed_dec_step, aed_dec_prefill and aed_dec_greedy_decode do not run on slots (AED_ERR_STATE); a later
+ * aed_dec_precompute_cross_kv returns the handle to batch operation.
+ */
+aed_status_t aed_dec_open_slots(aed_dec_t *dec, int32_t slots);
+aed_status_t aed_dec_admit(aed_dec_t *dec, int32_t slot, const void *enc, int32_t enc_len, int32_t max_len,
+                           int32_t *out_lens);
+aed_status_t aed_dec_greedy_steps(aed_dec_t *dec, int32_t n_steps, int32_t *tokens_out, int32_t *out_lens,
+                                  int32_t *steps_done /* HOST out, may be NULL */);
+
+/*
+ * The whole stream through the slots: utterances enter in arrival order (order[i], or 0, 1, 2, ... if order is NULL) as
+ * slots become free, and leave with their tokens.  Without an end-of-sequence id the host knows the step in which every
+ * utterance ends, issues exactly the steps up to the next departure and never waits for the device; with one it issues
+ * poll_steps steps at a time and reads the slots' lengths back.
+ *   enc_packed  DEVICE [sum(enc_lens), d_enc], utterance i at rows off[i] .. off[i+1] (index order, not arrival order)
+ *   enc_lens, max_lens, order   HOST [n]
+ *   tokens_out  HOST int32 [n, max_dec_len] (pinned memory keeps the host from waiting on every departure); row i holds
+ *               out_lens[i] tokens, entries beyond are unspecified
+ *   out_lens    HOST int32 [n]
+ *   steps_out, row_steps_out   HOST, may be NULL: steps issued, and (slot, step) pairs that held a decoding utterance
+ *               by the host's bounds (their ratio over `slots` is the occupancy)
+ * The slots' token rows live in the workspace.  Synchronises the stream before returning.
+ */
+aed_status_t aed_dec_decode_stream(aed_dec_t *dec, const void *enc_packed, const int32_t *enc_lens, const int32_t *max_lens,
+                                   const int32_t *order, int32_t n, int32_t slots, int32_t poll_steps, int32_t *tokens_out,
+                                   int32_t *out_lens, int64_t *steps_out, int64_t *row_steps_out);
+
 /* Synchronise the stream and report any sticky device-side error (AED_OK if none). */
 aed_status_t aed_dec_sync_status(aed_dec_t *dec);
 

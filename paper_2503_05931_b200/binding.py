@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = [
     "aed_dec_greedy_decode", "aed_dec_sync_status", "aed_dec_launch_count", "aed_dec_destroy",
     "aed_dec_last_error", "aed_dec_create_error", "aed_dec_profile_enable", "aed_dec_profile_read",
     "aed_dec_step_static_scratch", "aed_dec_static_scratch_bytes", "aed_dec_status_of_error_word", "aed_dec_prefill",
+    "aed_dec_open_slots", "aed_dec_admit", "aed_dec_greedy_steps", "aed_dec_decode_stream",
 ]
 
 _GLOBAL_FIELDS = ["embed", "final_ln_g", "final_ln_b", "w_out", "b_out"]
@@ -70,6 +71,16 @@ def load_library() -> C.CDLL:
     lib.aed_dec_precompute_cross_kv.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32), C.c_int32]
     lib.aed_dec_step.restype = C.c_int
     lib.aed_dec_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.aed_dec_open_slots.restype = C.c_int
+    lib.aed_dec_open_slots.argtypes = [C.c_void_p, C.c_int32]
+    lib.aed_dec_admit.restype = C.c_int
+    lib.aed_dec_admit.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+    lib.aed_dec_greedy_steps.restype = C.c_int
+    lib.aed_dec_greedy_steps.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.aed_dec_decode_stream.restype = C.c_int
+    lib.aed_dec_decode_stream.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                          C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64),
+                                          C.POINTER(C.c_int64)]
     lib.aed_dec_prefill.restype = C.c_int
     lib.aed_dec_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     lib.aed_dec_step_static_scratch.restype = C.c_int
@@ -213,6 +224,47 @@ class Decoder:
         self._check(self.lib.aed_dec_greedy_decode(self.handle, ml.ctypes.data_as(C.POINTER(C.c_int32)),
                                                    tokens_out.data_ptr(), out_lens.data_ptr()))
         return tokens_out, out_lens
+
+    def open_slots(self, slots: int) -> None:
+        self._check(self.lib.aed_dec_open_slots(self.handle, int(slots)))
+        self.batch = int(slots)
+
+    def admit(self, slot: int, enc, max_len: int, out_lens=None) -> None:
+        """enc: device tensor [enc_len, d_enc] in the handle's dtype (a contiguous slice of a packed buffer will do)."""
+        assert enc.is_cuda and enc.dtype == self.tdtype and enc.is_contiguous() and enc.dim() == 2
+        self._check(self.lib.aed_dec_admit(self.handle, int(slot), enc.data_ptr(), int(enc.shape[0]), int(max_len),
+                                           out_lens.data_ptr() if out_lens is not None else None))
+
+    def greedy_steps(self, n_steps: int, tokens_out, out_lens) -> int:
+        done = C.c_int32(0)
+        self._check(self.lib.aed_dec_greedy_steps(self.handle, int(n_steps), tokens_out.data_ptr(), out_lens.data_ptr(),
+                                                  C.byref(done)))
+        return int(done.value)
+
+    def decode_stream(self, enc_packed, enc_lens, max_lens, slots: int, *, order=None, poll_steps: int = 8,
+                      tokens_out=None, out_lens=None):
+        """tokens_out / out_lens: pinned host tensors int32 [n, max_dec_len] / [n] (allocated if None).
+        Returns (tokens_out, out_lens, steps, row_steps)."""
+        torch = self._torch
+        assert enc_packed.is_cuda and enc_packed.dtype == self.tdtype and enc_packed.is_contiguous()
+        el = np.ascontiguousarray(enc_lens, dtype=np.int32)
+        ml = np.ascontiguousarray(max_lens, dtype=np.int32)
+        n = len(el)
+        assert len(ml) == n and int(el.sum()) == enc_packed.shape[0]
+        od = None if order is None else np.ascontiguousarray(order, dtype=np.int32)
+        if tokens_out is None:
+            tokens_out = torch.empty((n, self.max_dec_len), dtype=torch.int32).pin_memory()
+        if out_lens is None:
+            out_lens = torch.zeros(n, dtype=torch.int32).pin_memory()
+        assert not tokens_out.is_cuda and not out_lens.is_cuda and tokens_out.is_contiguous() and out_lens.is_contiguous()
+        steps, row_steps = C.c_int64(0), C.c_int64(0)
+        i32p = C.POINTER(C.c_int32)
+        self._check(self.lib.aed_dec_decode_stream(self.handle, enc_packed.data_ptr(), el.ctypes.data_as(i32p), ml.ctypes.data_as(i32p),
+                                                   od.ctypes.data_as(i32p) if od is not None else None, n, int(slots),
+                                                   int(poll_steps), tokens_out.data_ptr(), out_lens.data_ptr(),
+                                                   C.byref(steps), C.byref(row_steps)))
+        self.batch = int(slots)
+        return tokens_out, out_lens, int(steps.value), int(row_steps.value)
 
     def sync_status(self) -> None:
         self._check(self.lib.aed_dec_sync_status(self.handle))

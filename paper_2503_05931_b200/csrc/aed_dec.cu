@@ -51,6 +51,7 @@ struct Layout {
     // bf16 mode: activation planes (high, low) that feed the tensor-core projections
     size_t actd_hi, actd_lo, actf_hi, actf_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
+    size_t slot_tokens, slot_lens;        // aed_dec_decode_stream: token rows and lengths of the slots
     size_t comp_w, comp_b;                // per layer: Wqc diag(gamma2) Wo as bf16 [d, d], and Wqc (gamma2 * bo) as fp32 [d]
     size_t ckv_maps, ckv_bias;            // per-layer tensor maps and bias pointers of the cross-K/V weights
     size_t fold_layer_floats;
@@ -114,6 +115,8 @@ Layout make_layout(const aed_dec_config_t &c)
     L.row_tok = take((size_t)rows_bucket(c.max_batch) * 4);        // prefill: the token of every (utterance, position) row
     L.len_order = take(B * 4);                                     // utterances by decreasing encoder length
     L.rows_cap = (int)align_up(B, 16);
+    L.slot_tokens = take(B * (size_t)c.max_dec_len * 4);
+    L.slot_lens = take(B * 4);
     if (c.dtype == AED_DTYPE_BF16) {
         L.actd_hi = take((size_t)L.rows_cap * d * 2);
         L.actd_lo = take((size_t)L.rows_cap * d * 2);
@@ -150,6 +153,9 @@ struct aed_dec {
     int full_steps = 0;             // steps without a mask: lower bound on t_u of every utterance not retired
     int total_frames = 0;
     std::vector<int32_t> enc_len, enc_off;
+    // continuous batching: the batch is a set of slots that utterances enter and leave one by one
+    bool slot_mode = false;
+    std::vector<int32_t> slot_t, slot_max;      // steps issued since the slot's utterance entered (-1: empty), its forced length
     std::string err;
     int64_t launches = 0;
     // optional per-kernel-family timing (CUDA events around every launch)
@@ -883,17 +889,21 @@ aed_status_t forward_step_planes(aed_dec *dec, int rows_ub, int self_len_ub, con
 }
 
 // Cross K/V of every layer on tensor cores, one persistent launch: D[frame, feature] = enc[frame, :] . w_kv_c[feature, :]
-aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
+// Cross-K/V of runs of encoder frames: run i is rows src0[i] .. src0[i] + frames[i] - 1 of the tensor at enc_base
+// (enc_rows rows in all) and goes to store rows dst0[i] .. (see ckv::CkvSegs; tile0 is filled here).
+aed_status_t precompute_tc(aed_dec *dec, const void *enc_base, long long enc_rows, ckv::CkvSegs segs)
 {
     typedef __nv_bfloat16 T;
     const auto &c = dec->cfg;
     const Layout &L = dec->lay;
-    if (reinterpret_cast<uintptr_t>(enc_packed) % 16) return fail(dec, AED_ERR_INVALID_ARG, "enc_packed must be 16-byte aligned");
+    if (reinterpret_cast<uintptr_t>(enc_base) % 16) return fail(dec, AED_ERR_INVALID_ARG, "the encoder states must be 16-byte aligned");
     CUtensorMap map_enc;
-    if (!encode_map(&map_enc, enc_packed, dec->total_frames, c.d_enc, tc::kTileM))
+    if (!encode_map(&map_enc, enc_base, (size_t)enc_rows, c.d_enc, tc::kTileM))
         return fail(dec, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed for the encoder states");
+    segs.tile0[0] = 0;
+    for (int i = 0; i < segs.n; ++i) segs.tile0[i + 1] = segs.tile0[i] + (segs.frames[i] + tc::kTileM - 1) / tc::kTileM;
     ckv::CkvParams p{};
-    p.total_frames = dec->total_frames;
+    p.segs = segs;
     p.frame_capacity = c.max_total_enc_frames;
     p.d_model = c.d_model; p.n_heads = c.n_heads; p.d_enc = c.d_enc;
     p.n_layers = c.n_layers;
@@ -901,8 +911,7 @@ aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
     p.layer_elems = L.cross_layer_elems;
     p.bias = dec->at<const T *>(L.ckv_bias);
     p.state = dec->state();
-    const long long tiles = (long long)((dec->total_frames + tc::kTileM - 1) / tc::kTileM) * c.n_layers *
-                            ((2 * c.d_model + ckv::kTileN - 1) / ckv::kTileN);
+    const long long tiles = (long long)segs.tile0[segs.n] * c.n_layers * ((2 * c.d_model + ckv::kTileN - 1) / ckv::kTileN);
     ProfScope ps(dec, KF_PRECOMPUTE);
     ckv::crosskv_gemm_kernel<<<(unsigned)std::min<long long>(tiles, dec->sm_count), ckv::kCkvThreads, ckv::kStages * ckv::kStageBytes + 1024, dec->stream>>>(
         map_enc, dec->at<CUtensorMap>(L.ckv_maps), p);
@@ -910,8 +919,16 @@ aed_status_t precompute_tc(aed_dec *dec, const void *enc_packed)
     return AED_OK;
 }
 
+ckv::CkvSegs one_run(int frames, int dst0)
+{
+    ckv::CkvSegs g{};
+    g.n = 1;
+    g.src0[0] = 0; g.frames[0] = frames; g.dst0[0] = dst0;
+    return g;
+}
+
 template <typename T>
-aed_status_t precompute_impl(aed_dec *dec, const void *enc_packed)
+aed_status_t precompute_impl(aed_dec *dec, const void *enc_packed, int frames, int frame0)
 {
     const auto &c = dec->cfg;
     const Layout &L = dec->lay;
@@ -919,9 +936,10 @@ aed_status_t precompute_impl(aed_dec *dec, const void *enc_packed)
     ep.d_model = c.d_model;
     ep.n_heads = c.n_heads;
     ep.frame_capacity = c.max_total_enc_frames;
+    ep.frame0 = frame0;
     for (int l = 0; l < c.n_layers; ++l) {
         ep.cross_store = dec->at<T>(L.cross_store) + (size_t)l * L.cross_layer_elems;
-        AED_TRY((launch_gemm<T, T, EPI_CROSSKV>(dec, KF_PRECOMPUTE, dec->total_frames, dec->total_frames, (const T *)enc_packed, c.d_enc,
+        AED_TRY((launch_gemm<T, T, EPI_CROSSKV>(dec, KF_PRECOMPUTE, frames, frames, (const T *)enc_packed, c.d_enc,
                                                 dec->layers[l].w_kv_c, dec->layers[l].b_kv_c, 2 * c.d_model, c.d_enc, ep)));
     }
     return AED_OK;
@@ -1078,7 +1096,9 @@ extern "C" aed_status_t aed_dec_precompute_cross_kv(aed_dec_t *dec, const void *
     }
     AED_CUDA(dec, cudaMemsetAsync(dec->ws + L.keys, 0, L.enc_off - L.keys, dec->stream));   // keys, state, t_u, retired, lists
     AED_CUDA(dec, cudaMemcpyAsync(&dec->state()->batch, &dec->batch, sizeof(int32_t), cudaMemcpyHostToDevice, dec->stream));
-    aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed) : precompute_impl<float>(dec, enc_packed);
+    dec->slot_mode = false;
+    aed_status_t s = dec->use_tc ? precompute_tc(dec, enc_packed, dec->total_frames, one_run(dec->total_frames, 0))
+                                 : precompute_impl<float>(dec, enc_packed, dec->total_frames, 0);
     if (s != AED_OK) return s;
     dec->have_batch = true;
     dec->fresh_batch = true;
@@ -1093,6 +1113,7 @@ extern "C" aed_status_t aed_dec_step(aed_dec_t *dec, const int32_t *tokens_in, c
     if (!dec) return AED_ERR_INVALID_ARG;
     if (!tokens_in) return fail(dec, AED_ERR_INVALID_ARG, "tokens_in must not be NULL");
     if (!dec->have_batch) return fail(dec, AED_ERR_STATE, "aed_dec_step needs a batch: call aed_dec_precompute_cross_kv first");
+    if (dec->slot_mode) return fail(dec, AED_ERR_STATE, "aed_dec_step does not run on slots: use aed_dec_greedy_steps");
     if (dec->full_steps >= dec->cfg.max_dec_len)
         return fail(dec, AED_ERR_CAPACITY, "every utterance already holds max_dec_len = %d tokens", dec->cfg.max_dec_len);
     AED_TRY(launch_build_active(dec, active));
@@ -1257,7 +1278,7 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
     if (!dec) return AED_ERR_INVALID_ARG;
     if (!max_len || !tokens_out || !out_lens) return fail(dec, AED_ERR_INVALID_ARG, "max_len, tokens_out and out_lens must not be NULL");
     if (!dec->have_batch) return fail(dec, AED_ERR_STATE, "aed_dec_greedy_decode needs a batch: call aed_dec_precompute_cross_kv first");
-    if (!dec->fresh_batch) return fail(dec, AED_ERR_STATE, "aed_dec_greedy_decode must directly follow aed_dec_precompute_cross_kv");
+    if (!dec->fresh_batch || dec->slot_mode) return fail(dec, AED_ERR_STATE, "aed_dec_greedy_decode must directly follow aed_dec_precompute_cross_kv");
     const int B = dec->batch;
     int longest = 0;
     for (int u = 0; u < B; ++u) {
@@ -1315,6 +1336,238 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
         }
     }
     dec->full_steps = dec->cfg.max_dec_len;   // every utterance is retired: further steps are refused
+    return aed_dec_sync_status(dec);
+}
+
+// ---- continuous batching: utterances enter and leave slots one by one -----------------------------------------------
+
+extern "C" aed_status_t aed_dec_open_slots(aed_dec_t *dec, int32_t slots)
+{
+    if (!dec) return AED_ERR_INVALID_ARG;
+    const auto &c = dec->cfg;
+    if (slots < 1) return fail(dec, AED_ERR_INVALID_ARG, "slots must be at least 1");
+    if (slots > c.max_batch) return fail(dec, AED_ERR_CAPACITY, "%d slots exceed max_batch %d", slots, c.max_batch);
+    if ((long long)slots * c.max_enc_len > c.max_total_enc_frames)
+        return fail(dec, AED_ERR_CAPACITY, "%d slots of max_enc_len %d frames exceed max_total_enc_frames %d", slots, c.max_enc_len,
+                    c.max_total_enc_frames);
+    const Layout &L = dec->lay;
+    dec->have_batch = false;
+    dec->batch = slots;
+    dec->total_frames = 0;
+    dec->enc_len.assign(slots, 0);
+    dec->enc_off.assign(slots + 1, 0);
+    for (int u = 0; u <= slots; ++u) dec->enc_off[u] = u * c.max_enc_len;       // every slot owns max_enc_len store rows
+    dec->slot_t.assign(slots, -1);
+    dec->slot_max.assign(slots, 0);
+    AED_CUDA(dec, cudaMemsetAsync(dec->ws + L.keys, 0, L.enc_off - L.keys, dec->stream));   // keys, state, t_u, retired, lists
+    AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.enc_off, dec->enc_off.data(), (slots + 1) * 4, cudaMemcpyHostToDevice, dec->stream));
+    AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.enc_len, dec->enc_len.data(), slots * 4, cudaMemcpyHostToDevice, dec->stream));
+    {
+        std::vector<int32_t> order(slots);
+        for (int u = 0; u < slots; ++u) order[u] = u;
+        AED_CUDA(dec, cudaMemcpyAsync(dec->ws + L.len_order, order.data(), slots * 4, cudaMemcpyHostToDevice, dec->stream));
+    }
+    AED_CUDA(dec, cudaMemcpyAsync(&dec->state()->batch, &dec->batch, sizeof(int32_t), cudaMemcpyHostToDevice, dec->stream));
+    AED_TRY(fill_i32(dec, dec->at<int32_t>(L.retired), 1, slots));      // empty slots take no part in a step
+    dec->slot_mode = true;
+    dec->have_batch = true;
+    dec->fresh_batch = false;
+    dec->steps_issued = 0;
+    dec->full_steps = 0;
+    return AED_OK;
+}
+
+namespace {
+
+struct Admission { int slot; long long src_row; int frames, max_len; };
+
+aed_status_t check_admission(aed_dec *dec, const Admission &a)
+{
+    const auto &c = dec->cfg;
+    if (a.slot < 0 || a.slot >= dec->batch) return fail(dec, AED_ERR_INVALID_ARG, "slot %d is outside 0..%d", a.slot, dec->batch - 1);
+    if (a.frames < 1) return fail(dec, AED_ERR_INVALID_ARG, "enc_len = %d: an utterance needs at least one frame", a.frames);
+    if (a.frames > c.max_enc_len) return fail(dec, AED_ERR_CAPACITY, "enc_len = %d exceeds max_enc_len %d", a.frames, c.max_enc_len);
+    if (a.max_len < 1) return fail(dec, AED_ERR_INVALID_ARG, "max_len = %d: must be at least 1", a.max_len);
+    if (a.max_len > c.max_dec_len) return fail(dec, AED_ERR_CAPACITY, "max_len = %d exceeds max_dec_len %d", a.max_len, c.max_dec_len);
+    // Without an end-of-sequence id the host knows when a slot's utterance ends; with one the caller has seen
+    // out_lens[slot] > 0 before it reuses the slot.
+    if (c.eos_id < 0 && dec->slot_t[a.slot] >= 0 && dec->slot_t[a.slot] < dec->slot_max[a.slot])
+        return fail(dec, AED_ERR_STATE, "slot %d still decodes (%d of %d tokens)", a.slot, dec->slot_t[a.slot], dec->slot_max[a.slot]);
+    return AED_OK;
+}
+
+// Up to ckv::kMaxSegs utterances enter their slots with one cross-K/V launch and one bookkeeping launch.  The encoder
+// states of admission i are rows src_row .. src_row + frames - 1 of the tensor at enc_base (enc_rows rows).
+aed_status_t admit_many(aed_dec *dec, const void *enc_base, long long enc_rows, const Admission *adm, int n, int32_t *out_lens)
+{
+    static_assert(kMaxAdmit == ckv::kMaxSegs, "one bookkeeping entry per run of frames");
+    const auto &c = dec->cfg;
+    const Layout &L = dec->lay;
+    const size_t row_bytes = (size_t)c.d_enc * (c.dtype == AED_DTYPE_BF16 ? 2 : 4);
+    ckv::CkvSegs segs{};
+    AdmitBatch ab{};
+    segs.n = ab.n = n;
+    for (int i = 0; i < n; ++i) {
+        AED_TRY(check_admission(dec, adm[i]));
+        for (int k = 0; k < i; ++k)
+            if (adm[k].slot == adm[i].slot) return fail(dec, AED_ERR_INVALID_ARG, "slot %d is admitted into twice", adm[i].slot);
+        segs.src0[i] = (int)adm[i].src_row; segs.frames[i] = adm[i].frames; segs.dst0[i] = adm[i].slot * c.max_enc_len;
+        ab.slot[i] = adm[i].slot; ab.n_frames[i] = adm[i].frames; ab.frame0[i] = segs.dst0[i]; ab.forced_len[i] = adm[i].max_len;
+    }
+    if (dec->use_tc) {
+        AED_TRY(precompute_tc(dec, enc_base, enc_rows, segs));
+    } else {
+        for (int i = 0; i < n; ++i)
+            AED_TRY(precompute_impl<float>(dec, static_cast<const char *>(enc_base) + (size_t)adm[i].src_row * row_bytes, adm[i].frames, segs.dst0[i]));
+    }
+    {
+        ProfScope ps(dec, KF_BOOKKEEPING);
+        admit_slots_kernel<<<1, 32, 0, dec->stream>>>(ab, c.bos_id, dec->at<int32_t>(L.enc_len), dec->at<int32_t>(L.enc_off),
+                                                      dec->at<int32_t>(L.t_u), dec->at<int32_t>(L.retired), dec->at<int32_t>(L.cur_tok),
+                                                      dec->at<int32_t>(L.max_len), out_lens);
+        AED_LAUNCHED(dec);
+    }
+    for (int i = 0; i < n; ++i) {
+        dec->enc_len[adm[i].slot] = adm[i].frames;
+        dec->slot_t[adm[i].slot] = 0;
+        dec->slot_max[adm[i].slot] = adm[i].max_len;
+    }
+    return AED_OK;
+}
+
+}  // namespace
+
+extern "C" aed_status_t aed_dec_admit(aed_dec_t *dec, int32_t slot, const void *enc, int32_t enc_len, int32_t max_len,
+                                      int32_t *out_lens)
+{
+    if (!dec) return AED_ERR_INVALID_ARG;
+    if (!dec->have_batch || !dec->slot_mode) return fail(dec, AED_ERR_STATE, "aed_dec_admit needs slots: call aed_dec_open_slots first");
+    if (!enc) return fail(dec, AED_ERR_INVALID_ARG, "enc must not be NULL");
+    const Admission a{slot, 0, enc_len, max_len};
+    AED_TRY(check_admission(dec, a));           // before enc_len is used as the extent of the tensor
+    return admit_many(dec, enc, enc_len, &a, 1, out_lens);
+}
+
+extern "C" aed_status_t aed_dec_greedy_steps(aed_dec_t *dec, int32_t n_steps, int32_t *tokens_out, int32_t *out_lens,
+                                             int32_t *steps_done)
+{
+    if (steps_done) *steps_done = 0;
+    if (!dec) return AED_ERR_INVALID_ARG;
+    if (!dec->have_batch || !dec->slot_mode) return fail(dec, AED_ERR_STATE, "aed_dec_greedy_steps needs slots: call aed_dec_open_slots first");
+    if (!tokens_out || !out_lens) return fail(dec, AED_ERR_INVALID_ARG, "tokens_out and out_lens must not be NULL");
+    if (n_steps < 0) return fail(dec, AED_ERR_INVALID_ARG, "n_steps must not be negative");
+    for (int s = 0; s < n_steps; ++s) {
+        // what the host knows: a slot decodes until its forced length (with an end-of-sequence id it may stop earlier
+        // on the device; its row then simply is not there any more)
+        int rows_ub = 0, longest = 0;
+        for (int u = 0; u < dec->batch; ++u)
+            if (dec->slot_t[u] >= 0 && dec->slot_t[u] < dec->slot_max[u]) { ++rows_ub; longest = std::max(longest, dec->slot_t[u] + 1); }
+        if (rows_ub == 0) break;
+        if (dec->use_graphs && !dec->profiling) {
+            const int rows_b = rows_bucket(rows_ub), chunks = (longest + kAttnChunk - 1) / kAttnChunk;
+            const aed_dec::GraphKey key(rows_b, chunks, tokens_out, out_lens);
+            auto it = dec->graphs.find(key);
+            if (it == dec->graphs.end()) {
+                aed_dec::GraphEntry entry{};
+                AED_TRY(capture_greedy_step(dec, rows_b, chunks * kAttnChunk, tokens_out, out_lens, &entry));
+                it = dec->graphs.emplace(key, entry).first;
+            }
+            AED_CUDA(dec, cudaGraphLaunch(it->second.exec, dec->stream));
+            dec->launches += it->second.nodes;
+        } else {
+            AED_TRY(enqueue_greedy_step(dec, rows_ub, longest, tokens_out, out_lens));
+        }
+        for (int u = 0; u < dec->batch; ++u)
+            if (dec->slot_t[u] >= 0 && dec->slot_t[u] < dec->slot_max[u]) ++dec->slot_t[u];
+        if (steps_done) ++*steps_done;
+    }
+    return AED_OK;
+}
+
+extern "C" aed_status_t aed_dec_decode_stream(aed_dec_t *dec, const void *enc_packed, const int32_t *enc_lens,
+                                              const int32_t *max_lens, const int32_t *order, int32_t n, int32_t slots,
+                                              int32_t poll_steps, int32_t *tokens_out, int32_t *out_lens,
+                                              int64_t *steps_out, int64_t *row_steps_out)
+{
+    if (steps_out) *steps_out = 0;
+    if (row_steps_out) *row_steps_out = 0;
+    if (!dec) return AED_ERR_INVALID_ARG;
+    if (!enc_packed || !enc_lens || !max_lens || !tokens_out || !out_lens)
+        return fail(dec, AED_ERR_INVALID_ARG, "enc_packed, enc_lens, max_lens, tokens_out and out_lens must not be NULL");
+    if (n < 1) return fail(dec, AED_ERR_INVALID_ARG, "n must be at least 1");
+    const auto &c = dec->cfg;
+    const bool eos = c.eos_id >= 0;
+    if (eos && poll_steps < 1) return fail(dec, AED_ERR_INVALID_ARG, "poll_steps must be at least 1 when eos_id >= 0");
+    std::vector<long long> off(n + 1, 0);
+    std::vector<char> seen(n, 0);
+    for (int i = 0; i < n; ++i) {
+        if (enc_lens[i] < 1 || enc_lens[i] > c.max_enc_len)
+            return fail(dec, enc_lens[i] < 1 ? AED_ERR_INVALID_ARG : AED_ERR_CAPACITY, "enc_lens[%d] = %d is outside 1..max_enc_len = %d", i, enc_lens[i], c.max_enc_len);
+        if (max_lens[i] < 1 || max_lens[i] > c.max_dec_len)
+            return fail(dec, max_lens[i] < 1 ? AED_ERR_INVALID_ARG : AED_ERR_CAPACITY, "max_lens[%d] = %d is outside 1..max_dec_len = %d", i, max_lens[i], c.max_dec_len);
+        off[i + 1] = off[i] + enc_lens[i];
+        if (order) {
+            if (order[i] < 0 || order[i] >= n || seen[order[i]]) return fail(dec, AED_ERR_INVALID_ARG, "order is not a permutation of 0..n-1");
+            seen[order[i]] = 1;
+        }
+    }
+    AED_TRY(aed_dec_open_slots(dec, slots));
+    const Layout &L = dec->lay;
+    int32_t *toks = dec->at<int32_t>(L.slot_tokens), *lens = dec->at<int32_t>(L.slot_lens);
+    const int ld = c.max_dec_len;
+    if (off[n] > 0x7fffffffLL) return fail(dec, AED_ERR_CAPACITY, "the stream has %lld encoder frames; at most 2^31 - 1 per call", off[n]);
+    std::vector<int> occupant(slots, -1), remaining(slots, 0);
+    std::vector<int32_t> lens_host(slots, 0);
+    int next = 0;
+    long long steps = 0, row_steps = 0;
+    auto fill = [&]() -> aed_status_t {
+        Admission adm[ckv::kMaxSegs];
+        int k = 0;
+        for (int s = 0; s < slots && next < n; ++s) {
+            if (occupant[s] >= 0) continue;
+            const int u = order ? order[next] : next;
+            ++next;
+            adm[k++] = Admission{s, off[u], enc_lens[u], max_lens[u]};
+            occupant[s] = u;
+            remaining[s] = max_lens[u];
+            if (k == ckv::kMaxSegs) { AED_TRY(admit_many(dec, enc_packed, off[n], adm, k, lens)); k = 0; }
+        }
+        if (k) AED_TRY(admit_many(dec, enc_packed, off[n], adm, k, lens));
+        return AED_OK;
+    };
+    // The finished utterance's tokens and length go to the host behind the steps that produced them and before the
+    // slot's next occupant (stream order); with pinned host buffers the host does not wait for them.
+    auto harvest = [&](int s) -> aed_status_t {
+        const int u = occupant[s];
+        AED_CUDA(dec, cudaMemcpyAsync(tokens_out + (size_t)u * ld, toks + (size_t)s * ld, (size_t)max_lens[u] * 4, cudaMemcpyDeviceToHost, dec->stream));
+        AED_CUDA(dec, cudaMemcpyAsync(out_lens + u, lens + s, 4, cudaMemcpyDeviceToHost, dec->stream));
+        occupant[s] = -1;
+        return AED_OK;
+    };
+    AED_TRY(fill());
+    for (;;) {
+        int busy = 0, lo = 1 << 30, hi = 0;
+        for (int s = 0; s < slots; ++s)
+            if (occupant[s] >= 0) { ++busy; lo = std::min(lo, remaining[s]); hi = std::max(hi, remaining[s]); }
+        if (!busy) break;
+        // without an end-of-sequence id the host knows the step in which the next utterance leaves
+        const int want = eos ? std::min(poll_steps, hi) : lo;
+        int32_t done = 0;
+        AED_TRY(aed_dec_greedy_steps(dec, want, toks, lens, &done));
+        steps += done;
+        for (int s = 0; s < slots; ++s)
+            if (occupant[s] >= 0) { row_steps += std::min<int>(done, remaining[s]); remaining[s] = std::max(remaining[s] - done, 0); }
+        if (eos) {
+            AED_CUDA(dec, cudaMemcpyAsync(lens_host.data(), lens, (size_t)slots * 4, cudaMemcpyDeviceToHost, dec->stream));
+            AED_CUDA(dec, cudaStreamSynchronize(dec->stream));
+        }
+        for (int s = 0; s < slots; ++s)
+            if (occupant[s] >= 0 && (remaining[s] == 0 || (eos && lens_host[s] > 0))) AED_TRY(harvest(s));
+        AED_TRY(fill());
+        if (done == 0 && next >= n) break;
+    }
+    if (steps_out) *steps_out = steps;
+    if (row_steps_out) *row_steps_out = row_steps;
     return aed_dec_sync_status(dec);
 }
 

@@ -34,8 +34,20 @@ constexpr int kProducers = 4;
 constexpr int kCkvThreads = 384;
 constexpr int kMaxLayers = 64;
 
+// The frames of a launch: up to kMaxSegs runs of consecutive rows of the encoder tensor, each with a store row of its
+// own (a packed batch is one run; utterances admitted into slots are one run each).  Frame tiles never straddle runs.
+constexpr int kMaxSegs = 16;
+struct CkvSegs {
+    int n;
+    int tile0[kMaxSegs + 1];          // first frame tile of every run, and the total
+    int src0[kMaxSegs];               // row of the run's first frame in the encoder tensor
+    int frames[kMaxSegs];
+    int dst0[kMaxSegs];               // store row of the run's first frame
+};
+
 struct CkvParams {
-    int total_frames, frame_capacity;
+    CkvSegs segs;
+    int frame_capacity;
     int d_model, n_heads, d_enc;
     int n_layers;
     __nv_bfloat16 *store;             // layer 0; layers are layer_elems apart
@@ -88,7 +100,13 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
     const int k_blocks = p.d_enc / kBlockK;
-    const int m_tiles = (p.total_frames + kTileM - 1) / kTileM;
+    const int m_tiles = p.segs.tile0[p.segs.n];
+    // run and tile inside the run of a frame tile
+    auto locate = [&](int m_tile, int &seg, int &j) {
+        seg = 0;
+        while (seg + 1 < p.segs.n && m_tile >= p.segs.tile0[seg + 1]) ++seg;
+        j = m_tile - p.segs.tile0[seg];
+    };
     const int n_tiles = (2 * p.d_model + kTileN - 1) / kTileN;
     const int per_group = p.n_layers * n_tiles;
 
@@ -112,7 +130,9 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
             long long issued_last = -1;
             for (TileWalk w(m_tiles, per_group, gridDim.x, blockIdx.x); w.valid() && ok; w.next()) {
                 const int layer = w.lnt() / n_tiles, nt = w.lnt() % n_tiles;
-                const int m0 = w.m_tile() * kTileM;
+                int seg, j;
+                locate(w.m_tile(), seg, j);
+                const int m0 = p.segs.src0[seg] + j * kTileM;          // rows past the run's end are loaded and never stored
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     if (static_cast<int>(it % kProducers) != warp) continue;
                     const int s = static_cast<int>(it % kStages);
@@ -165,7 +185,11 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
         long long t = 0;
         for (TileWalk w(m_tiles, per_group, gridDim.x, blockIdx.x); w.valid() && ok; w.next(), ++t) {
             const int layer = w.lnt() / n_tiles, nt = w.lnt() % n_tiles;
-            const int frame = w.m_tile() * kTileM + quarter * 32 + lane;
+            int seg, j;
+            locate(w.m_tile(), seg, j);
+            const int frame_in_run = j * kTileM + quarter * 32 + lane;
+            const bool frame_ok = frame_in_run < p.segs.frames[seg];
+            const int frame = p.segs.dst0[seg] + frame_in_run;
             const int buf = static_cast<int>(t & 1);
             ok = mbar_wait(&bar_acc_full[buf], static_cast<uint32_t>(t >> 1) & 1, &abort_flag);
             if (!ok) break;
@@ -177,7 +201,7 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
                 float v[16];
                 tmem_ld16(taddr + c0, v);
                 const int o = nt * kTileN + c0;                  // 16 consecutive features inside one head
-                if (frame >= p.total_frames || o >= 2 * p.d_model) continue;
+                if (!frame_ok || o >= 2 * p.d_model) continue;
                 const int kv = o / p.d_model, cc = o % p.d_model, h = cc / kHeadDim, e = cc % kHeadDim;
                 uint32_t packed[8];
 #pragma unroll

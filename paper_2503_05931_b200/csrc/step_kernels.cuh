@@ -158,6 +158,7 @@ struct GemmEpilogueArgs {
     // CROSSKV: store of this layer [2][H][frame_capacity][64]
     CT *cross_store;
     int frame_capacity;
+    int frame0;                 // CROSSKV: store row of the first frame (an utterance admitted into a slot of its own)
 };
 
 template <typename AT, typename WT, typename CT, int EPI>
@@ -244,7 +245,7 @@ gemm_rows_kernel(const DecState *state, int rows_fixed, const AT *__restrict__ A
             } else if (EPI == EPI_CROSSKV) {
                 const int d = ep.d_model;
                 const int kv = o / d, c = o % d, h = c / kHeadDim, e = c % kHeadDim;
-                size_t off = (((size_t)kv * ep.n_heads + h) * ep.frame_capacity + r) * kHeadDim + e;
+                size_t off = (((size_t)kv * ep.n_heads + h) * ep.frame_capacity + ep.frame0 + r) * kHeadDim + e;
                 ep.cross_store[off] = from_f32<CT>(v);
             }
         }
@@ -958,6 +959,28 @@ __global__ void finish_step_kernel(DecState *state, const int32_t *__restrict__ 
             atomicAdd(&state->n_retired, 1);          // the host polls this to stop issuing steps once every utterance is done
         }
     }
+}
+
+// New utterances take over slots: position 0, start token, their encoder range and forced length.  One thread each.
+constexpr int kMaxAdmit = 16;
+struct AdmitBatch {
+    int n;
+    int slot[kMaxAdmit], n_frames[kMaxAdmit], frame0[kMaxAdmit], forced_len[kMaxAdmit];
+};
+__global__ void admit_slots_kernel(AdmitBatch b, int bos, int32_t *__restrict__ enc_len, int32_t *__restrict__ enc_off,
+                                   int32_t *__restrict__ t_u, int32_t *__restrict__ retired, int32_t *__restrict__ cur_tok,
+                                   int32_t *__restrict__ max_len, int32_t *__restrict__ out_lens)
+{
+    const int i = threadIdx.x;
+    if (blockIdx.x != 0 || i >= b.n) return;
+    const int slot = b.slot[i];
+    enc_len[slot] = b.n_frames[i];
+    enc_off[slot] = b.frame0[i];
+    t_u[slot] = 0;
+    cur_tok[slot] = bos;
+    max_len[slot] = b.forced_len[i];
+    if (out_lens) out_lens[slot] = 0;
+    retired[slot] = 0;
 }
 
 __global__ void fill_i32_kernel(int32_t *p, int32_t v, size_t n)

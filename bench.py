@@ -97,14 +97,15 @@ KERNEL_OF_FAMILY = {
 # dram__bytes_write.sum of the captured launches over their algorithmic bytes).  An entry is removed when its kernel
 # changes, which turns the reported traffic back into null.
 NCU_TRAFFIC_RATIO = {
-    # six launches of one layer at 64 rows: 64.27 MB read for 29.36 MB of weights; each launch also prefetches the next
-    # layer's matrix of its kind into L2, which under the profiler's serialised replay is a second DRAM read
-    "step_gemm_kernel": 2.19,
-    # self + cross attention of one layer at 64 rows: 0.84 + 30.79 MB for 0.52 + 30.49 MB of K/V
-    "attn_fused_kernel": 1.02,
+    # five launches of one layer at 64 rows: 68.44 MB read for 29.36 MB of layer weights; the launches also read the
+    # composite cross-query matrix (2.1 MB) and each prefetches the next layer's matrices of its kind into L2, which
+    # under the profiler's serialised replay is a second DRAM read
+    "step_gemm_kernel": 2.33,
+    # self + cross attention of one layer at 64 rows: 0.84 + 31.05 MB for 0.52 + 30.49 MB of K/V
+    "attn_fused_kernel": 1.03,
     # vocabulary projection: 33.85 MB for the 33.55 MB output matrix
     "tc_gemm_kernel": 1.01,
-    # cross-K/V of 7444 frames: 116.3 MB read + 680.4 MB written for 847.7 MB (part of the output is still in L2 at exit)
+    # cross-K/V of 7444 frames: 117.2 MB read + 677.2 MB written for 847.7 MB (part of the output is still in L2 at exit)
     "crosskv_gemm_kernel": 0.94,
 }
 

@@ -61,6 +61,7 @@ typedef ORC_REAL real;
 typedef struct {
     int32_t n_layers, d_model, n_heads, d_ffn, vocab, d_enc;
     double ln_eps;
+    int32_t cross_kv_e4m3;   /* nonzero: the cross-attention keys and values are stored as 8-bit floats (see below) */
 } orc_config_t;
 
 /* Row-major [out, in] matrices; per-layer members are arrays of n_layers pointers; NULL bias = no bias. */
@@ -168,6 +169,25 @@ static void embed_token(const orc_config_t *cfg, const orc_weights_t *w, int32_t
     }
 }
 
+/* Nearest value of the 8-bit floating-point format E4M3 (OCP 8-bit Floating Point Specification: 1 sign bit, 4
+ * exponent bits with bias 7, 3 mantissa bits, subnormals at exponent field 0, no infinities, largest finite value
+ * 448), ties to the even mantissa, magnitudes beyond the largest finite value saturate to it.  A storage format the
+ * paper does not discuss: the cross-attention K/V store is the largest stream of a decode step, and storing it in
+ * 8 bits is this repository's extension; both sides of a parity test round the same way. */
+double orc_round_e4m3(double x)
+{
+    if (x != x || x == 0.0) return x;
+    double a = fabs(x);
+    int e;
+    (void)frexp(a, &e);                 /* a = m * 2^e with m in [0.5, 1): the leading bit has weight 2^(e-1) */
+    int lead = e - 1;
+    if (lead < -6) lead = -6;           /* subnormals share the quantum of the smallest normal binade: 2^-9 */
+    double quantum = ldexp(1.0, lead - 3);
+    double r = nearbyint(a / quantum) * quantum;     /* default rounding mode: to nearest, ties to even */
+    if (r > 448.0) r = 448.0;
+    return x < 0 ? -r : r;
+}
+
 /* Kc, Vc of one layer: [T][d] each */
 static void cross_kv(const orc_config_t *cfg, const orc_weights_t *w, int layer, const float *enc, int T,
                      real *Kc, real *Vc, real *tmp /* [2d] */)
@@ -175,6 +195,8 @@ static void cross_kv(const orc_config_t *cfg, const orc_weights_t *w, int layer,
     int d = cfg->d_model;
     for (int j = 0; j < T; ++j) {
         linear_f(w->w_kv_c[layer], w->b_kv_c ? w->b_kv_c[layer] : NULL, enc + (size_t)j * cfg->d_enc, 2 * d, cfg->d_enc, tmp);
+        if (cfg->cross_kv_e4m3)
+            for (int o = 0; o < 2 * d; ++o) tmp[o] = (real)orc_round_e4m3((double)tmp[o]);
         memcpy(Kc + (size_t)j * d, tmp, sizeof(real) * d);
         memcpy(Vc + (size_t)j * d, tmp + d, sizeof(real) * d);
     }

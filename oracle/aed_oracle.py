@@ -28,7 +28,7 @@ _FPP = C.POINTER(_FP)
 
 class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "d_ffn", "vocab", "d_enc")] + \
-               [("ln_eps", C.c_double)]
+               [("ln_eps", C.c_double), ("cross_kv_e4m3", C.c_int32)]
 
 
 class _Weights(C.Structure):
@@ -91,10 +91,12 @@ class Model:
     """Decoder parameters marshalled for the C checker.  ``weights`` maps tensor names to float32
     arrays (per-layer tensors: a list with one array per layer); a missing/None bias means no bias."""
 
-    def __init__(self, model: Dict[str, int], weights: Dict[str, object], ln_eps: float = 1e-5):
+    def __init__(self, model: Dict[str, int], weights: Dict[str, object], ln_eps: float = 1e-5,
+                 cross_kv_e4m3: bool = False):
+        """cross_kv_e4m3: the cross-attention keys and values are rounded to the 8-bit format E4M3 when stored."""
         self.model = dict(model)
         self.cfg = _Config(model["n_layers"], model["d_model"], model["n_heads"], model["d_ffn"],
-                           model["vocab"], model["d_enc"], float(ln_eps))
+                           model["vocab"], model["d_enc"], float(ln_eps), 1 if cross_kv_e4m3 else 0)
         self._keep: List[object] = []
         w = _Weights()
         nl = model["n_layers"]
@@ -211,6 +213,15 @@ def layernorm(x, g, b, eps: float = 1e-5, precision: str = "f64") -> np.ndarray:
     lib.orc_layernorm_f64(x.ctypes.data_as(C.POINTER(C.c_double)), g.ctypes.data_as(_FP), b.ctypes.data_as(_FP),
                           C.c_int(x.shape[0]), C.c_double(eps), y.ctypes.data_as(C.POINTER(C.c_double)))
     return y
+
+
+def round_e4m3(x, precision: str = "f64") -> np.ndarray:
+    """Element-wise rounding to the 8-bit format E4M3 as the checker stores cross-attention keys and values."""
+    lib = _lib(precision)
+    lib.orc_round_e4m3.restype = C.c_double
+    lib.orc_round_e4m3.argtypes = [C.c_double]
+    x = np.asarray(x, dtype=np.float64)
+    return np.array([lib.orc_round_e4m3(float(v)) for v in x.ravel()], dtype=np.float64).reshape(x.shape)
 
 
 def argmax(z, precision: str = "f64"):

@@ -16,6 +16,10 @@ from paper_2503_05931_b200 import workloads as wl
 SRC = os.path.join(os.path.dirname(orc.__file__), "aed_oracle.c")
 
 MUTATIONS = [
+    ("8-bit format with one mantissa bit too many", "double quantum = ldexp(1.0, lead - 3);", "double quantum = ldexp(1.0, lead - 4);"),
+    ("8-bit format with the wrong smallest normal exponent", "if (lead < -6) lead = -6;", "if (lead < -7) lead = -7;"),
+    ("8-bit format saturating at the wrong value", "if (r > 448.0) r = 448.0;", "if (r > 480.0) r = 480.0;"),
+    ("8-bit format rounding halves away from zero", "double r = nearbyint(a / quantum) * quantum;", "double r = floor(a / quantum + 0.5) * quantum;"),
     ("attention scale dropped", "real scale = (real)1 / (real)sqrt((double)dh);", "real scale = (real)1;"),
     ("softmax without max subtraction sign", "score[j] = (real)exp((double)(score[j] - mx));", "score[j] = (real)exp((double)(mx - score[j]));"),
     ("layernorm unbiased variance", "var /= (real)d;", "var /= (real)(d - 1);"),
@@ -93,6 +97,22 @@ def _pins(precision):
     assert not np.any(out["next"] == 17)                    # ties go to the lowest index
     idx, _ = orc.argmax(np.array([1.0, 3.0, 3.0, 2.0]), precision=precision)
     assert idx == 1
+    # 8-bit storage format of the cross-attention keys and values: nearest value of the format decoded from its bit
+    # fields, ties to the even mantissa, saturation at the largest finite value
+    vals = sorted({(m / 8.0 * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7))
+                   for e in range(16) for m in range(8) if not (e == 15 and m == 7)})
+    vals = np.array(vals)
+    xs = np.concatenate([rng.normal(0, 1, 300), rng.normal(0, 0.01, 200), rng.uniform(200, 470, 50), [1e5, 0.1875 * 2.0 ** -6]])
+    got = orc.round_e4m3(xs, precision=precision)
+    for x, g in zip(xs, got):
+        a = min(abs(x), 448.0)
+        dist = np.abs(vals - a)
+        near = vals[dist == dist.min()]
+        assert abs(g) in near and (g < 0) == (x < 0 and g != 0), (x, g)
+    mids = (vals[1:-1] + vals[2:]) / 2
+    for lo, hi, g in zip(vals[1:-1], vals[2:], orc.round_e4m3(mids, precision=precision)):
+        even = lo if int(round(lo / (2.0 ** -9 if lo < 2.0 ** -6 else 2.0 ** (math.floor(math.log2(lo)) - 3)))) % 2 == 0 else hi
+        assert g == even, (lo, hi, g)
 
 
 def test_pins_pass_on_the_real_checker():

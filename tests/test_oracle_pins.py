@@ -400,3 +400,83 @@ def test_eos_in_a_batch_stops_each_utterance_on_its_own():
         assert np.array_equal(cut["next"][u, :expect], free["next"][u, :expect])
         assert np.all(cut["next"][u, expect:] == -1)
     assert cut["lens"][0] <= 5
+
+
+# ---- 8-bit storage of the cross-attention keys and values (an extension; the format is the OCP E4M3 one) ------------
+
+def _e4m3_values():
+    """Every finite value of the format, decoded from its bit fields: sign, 4 exponent bits (bias 7), 3 mantissa bits;
+    exponent field 0 holds the subnormals; the code with all exponent and mantissa bits set is not a number."""
+    vals = []
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e, m = (code >> 3) & 0xF, code & 0x7
+        if e == 0xF and m == 0x7:
+            continue
+        vals.append(sign * (m / 8.0 * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)))
+    return np.array(sorted(set(vals)))
+
+
+def test_e4m3_rounding_against_the_enumerated_format():
+    vals = _e4m3_values()
+    assert vals.max() == 448.0 and vals[vals > 0].min() == 2.0 ** -9 and len(vals) == 253
+    # every value of the format is a fixed point
+    assert np.array_equal(orc.round_e4m3(vals), vals)
+    rng = np.random.default_rng(8)
+    x = np.concatenate([rng.normal(0, 1, 4000), rng.normal(0, 100, 2000), rng.normal(0, 0.01, 2000),
+                        rng.uniform(-2.0 ** -6, 2.0 ** -6, 1000), [449.0, 463.9, 464.0, 1e6, -1e6, 2.0 ** -10, 0.0]])
+    got = orc.round_e4m3(x)
+    clipped = np.clip(x, -448.0, 448.0)
+    nearest = vals[np.argmin(np.abs(vals[None, :] - clipped[:, None]), axis=1)]
+    dist = np.abs(vals[None, :] - clipped[:, None])
+    best = dist.min(axis=1)
+    ties = (np.isclose(dist, best[:, None], rtol=0, atol=0)).sum(axis=1) > 1
+    assert np.array_equal(got[~ties], nearest[~ties])
+    assert np.all(np.abs(got - clipped) <= best + 0.0)
+    # ties go to the even mantissa: midpoints between neighbours
+    pos = vals[vals > 0]
+    mids = (pos[:-1] + pos[1:]) / 2
+    r = orc.round_e4m3(mids)
+    for lo, hi, v in zip(pos[:-1], pos[1:], r):
+        assert v in (lo, hi)
+        mant = v / 2.0 ** -9 if v < 2.0 ** -6 else (v / 2.0 ** np.floor(np.log2(v)) - 1.0) * 8
+        assert int(round(mant)) % 2 == 0, (lo, hi, v)
+
+
+def test_e4m3_rounding_against_torch():
+    import torch
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    rng = np.random.default_rng(9)
+    x = np.concatenate([rng.normal(0, 1, 5000), rng.normal(0, 60, 3000), rng.uniform(-0.02, 0.02, 2000)])
+    x = x[np.abs(x) < 440].astype(np.float32)                    # inside the finite range
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    assert np.array_equal(orc.round_e4m3(x.astype(np.float64)), want)
+
+
+def test_cross_kv_in_e4m3_changes_what_it_should():
+    """With the 8-bit store only the cross-attention keys and values change: a model whose cross-attention output
+    projection is zero decodes identically, a normal one does not, and when the encoder states and weights make
+    every key and value a value of the format already, nothing changes either."""
+    model = dict(n_layers=2, d_model=128, n_heads=2, d_ffn=256, vocab=50, d_enc=64)
+    w = wl.make_custom(model, [9, 4], [5, 5], dtype="fp32", seed=12, out_std=0.2)
+    a = orc.decode_batch(orc.Model(w.model, w.weights), w.enc, w.enc_lens, w.dec_lens, want_logits=True)
+    b = orc.decode_batch(orc.Model(w.model, w.weights, cross_kv_e4m3=True), w.enc, w.enc_lens, w.dec_lens, want_logits=True)
+    diff = max(float(np.max(np.abs(x - y))) for x, y in zip(a["logits"], b["logits"]))
+    assert 1e-6 < diff < 0.5
+    w0 = dict(w.weights)
+    w0["w_o_c"] = [np.zeros_like(m) for m in w.weights["w_o_c"]]
+    w0["b_o_c"] = [np.zeros_like(m) for m in w.weights["b_o_c"]]
+    a = orc.decode_batch(orc.Model(w.model, w0), w.enc, w.enc_lens, w.dec_lens, want_logits=True)
+    b = orc.decode_batch(orc.Model(w.model, w0, cross_kv_e4m3=True), w.enc, w.enc_lens, w.dec_lens, want_logits=True)
+    assert all(np.array_equal(x, y) for x, y in zip(a["logits"], b["logits"]))
+    # keys and values that are small integers: one-hot encoder frames, integer weights, no bias
+    w1 = dict(w.weights)
+    rng = np.random.default_rng(4)
+    w1["w_kv_c"] = [rng.integers(-8, 9, size=m.shape).astype(np.float32) for m in w.weights["w_kv_c"]]
+    w1["b_kv_c"] = [np.zeros_like(m) for m in w.weights["b_kv_c"]]
+    enc = np.zeros_like(w.enc)
+    enc[np.arange(len(enc)), rng.integers(0, model["d_enc"], size=len(enc))] = 1.0
+    a = orc.decode_batch(orc.Model(w.model, w1), enc, w.enc_lens, w.dec_lens, want_logits=True)
+    b = orc.decode_batch(orc.Model(w.model, w1, cross_kv_e4m3=True), enc, w.enc_lens, w.dec_lens, want_logits=True)
+    assert all(np.array_equal(x, y) for x, y in zip(a["logits"], b["logits"]))

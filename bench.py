@@ -40,6 +40,10 @@ def load_peaks():
     return p
 
 
+# Bytes per element of the cross-attention K/V store when it is not the workload's dtype (--cross-kv e4m3: 1).
+CROSS_KV_BYTES = None
+
+
 def step_bytes_and_flops(w):
     """Algorithmic bytes and flops of greedy decoding, step by step (weights once per step, each active row's
     own self and cross K/V once per layer), and of the cross-K/V precompute."""
@@ -48,15 +52,17 @@ def step_bytes_and_flops(w):
     NL, d, F, V, de = m["n_layers"], m["d_model"], m["d_ffn"], m["vocab"], m["d_enc"]
     step_params = NL * (4 * d * d + 2 * d * d + 2 * d * F) + V * d
     T, L = w.enc_lens.astype(np.int64), w.dec_lens.astype(np.int64)
+    ec = CROSS_KV_BYTES or e
     per_step = []
     for s in range(int(L.max())):
         act = L > s
         n = int(act.sum())
         kv_pos = int((T[act] + s + 1).sum())
-        per_step.append((e * step_params + e * NL * 2 * d * kv_pos, 2 * n * step_params + 4 * d * NL * kv_pos, n))
+        kv_bytes = NL * 2 * d * (ec * int(T[act].sum()) + e * int((act.sum()) * (s + 1)))
+        per_step.append((e * step_params + kv_bytes, 2 * n * step_params + 4 * d * NL * kv_pos, n))
     total_T = int(T.sum())
     pre_flops = 2 * total_T * de * NL * 2 * d
-    pre_bytes = e * (total_T * de + NL * 2 * d * de + total_T * NL * 2 * d)
+    pre_bytes = e * (total_T * de + NL * 2 * d * de) + ec * total_T * NL * 2 * d
     return per_step, pre_bytes, pre_flops, step_params
 
 
@@ -74,12 +80,12 @@ def family_bytes(family, w):
     if family == "gemm_vocab":
         return e * V * d * steps
     if family == "attn_cross":
-        return sum(e * NL * 2 * d * int(T[L > s].sum()) for s in range(steps))
+        return sum((CROSS_KV_BYTES or e) * NL * 2 * d * int(T[L > s].sum()) for s in range(steps))
     if family == "attn_self":
         return sum(e * NL * 2 * d * int((L > s).sum()) * (s + 1) for s in range(steps))
     if family == "precompute_cross_kv":
         total_T = int(T.sum())
-        return e * (total_T * de + NL * 2 * d * de + total_T * NL * 2 * d)
+        return e * (total_T * de + NL * 2 * d * de) + (CROSS_KV_BYTES or e) * total_T * NL * 2 * d
     return None
 
 
@@ -357,10 +363,15 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=list(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--cross-kv", default="dtype", choices=["dtype", "e4m3"],
+                    help="storage of the cross-attention K/V: the workload's dtype (the measured configuration) or 8-bit E4M3")
     ap.add_argument("--clip-len", type=int, default=0,
                     help="shorten every forced output length to at most this many tokens (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    if args.cross_kv == "e4m3":
+        global CROSS_KV_BYTES
+        CROSS_KV_BYTES = 1
 
     if args.impl == "reference":
         run_reference(args)
@@ -389,7 +400,7 @@ def main():
     if args.clip_len > 0:
         w.dec_lens = np.minimum(w.dec_lens, args.clip_len).astype(np.int32)
     peaks = load_peaks()
-    dec = binding.decoder_for_workload(w, device=device)
+    dec = binding.decoder_for_workload(w, device=device, cross_kv_e4m3=args.cross_kv == "e4m3")
     enc_host = torch.from_numpy(w.enc).to(dec.tdtype).pin_memory()
     enc_dev = enc_host.to(device)
     B, Lmax = w.batch, int(w.dec_lens.max())
@@ -456,6 +467,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, **w.model, "batch_per_gpu": w.batch, "total_enc_frames": int(w.enc_lens.sum()),
                        "total_out_tokens": n_tok, "decode_steps": Lmax, "clip_len": args.clip_len,
+                       "cross_kv_store": "e4m3" if args.cross_kv == "e4m3" else w.dtype,
                        "l2": "inputs larger than L2 (weights + K/V stores stream every decode step)",
                        "step": "cross-K/V precompute + greedy decode of one batch"},
             "rtfx": rtfx,

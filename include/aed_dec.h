@@ -60,6 +60,11 @@ typedef enum {
 } aed_status_t;
 
 enum { AED_DTYPE_F32 = 0, AED_DTYPE_BF16 = 1 };
+/* Storage of the cross-attention keys and values: in the configured dtype, or (bf16 configuration only) rounded to
+ * the 8-bit floating-point format E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; nearest, ties to even,
+ * saturating at 448).  The paper does not discuss storage formats; the store is the largest stream of a decode step
+ * and the 8-bit form halves it.  Projections, softmax and accumulation are unchanged. */
+enum { AED_CROSS_KV_DTYPE = 0, AED_CROSS_KV_E4M3 = 1 };
 
 typedef struct {
     int32_t n_layers, d_model, n_heads, d_ffn, vocab, d_enc;
@@ -71,6 +76,7 @@ typedef struct {
     int32_t bos_id;               /* start token of aed_dec_greedy_decode */
     int32_t eos_id;               /* < 0: no end-of-sequence stopping */
     float ln_eps;                 /* LayerNorm epsilon (biased variance) */
+    int32_t cross_kv_format;      /* AED_CROSS_KV_DTYPE or AED_CROSS_KV_E4M3 */
     void *workspace;              /* DEVICE, 256-byte aligned, at least aed_dec_workspace_bytes() */
     size_t workspace_bytes;
     void *stream;                 /* cudaStream_t of the caller (NULL = default stream) */

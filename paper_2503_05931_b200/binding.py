@@ -18,6 +18,7 @@ LIB_PATH = os.environ.get("AED_DEC_LIB") or os.path.join(_HERE, "libaed_dec.so")
 AED_OK, AED_ERR_INVALID_ARG, AED_ERR_CAPACITY, AED_ERR_STATE = 0, -1, -2, -3
 AED_ERR_CUDA, AED_ERR_TIMEOUT, AED_ERR_UNSUPPORTED = -4, -5, -6
 AED_DTYPE_F32, AED_DTYPE_BF16 = 0, 1
+AED_CROSS_KV_DTYPE, AED_CROSS_KV_E4M3 = 0, 1
 
 EXPORTED_SYMBOLS = [
     "aed_dec_workspace_bytes", "aed_dec_create", "aed_dec_precompute_cross_kv", "aed_dec_step",
@@ -37,7 +38,7 @@ class AedConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "d_ffn", "vocab", "d_enc", "dtype",
                                          "max_batch", "max_total_enc_frames", "max_enc_len", "max_dec_len",
                                          "bos_id", "eos_id")] + \
-               [("ln_eps", C.c_float), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+               [("ln_eps", C.c_float), ("cross_kv_format", C.c_int32), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("stream", C.c_void_p)]
 
 
@@ -111,10 +112,12 @@ def load_library() -> C.CDLL:
 
 
 def make_config(model: Dict[str, int], dtype: str, *, max_batch: int, max_total_enc_frames: int, max_enc_len: int,
-                max_dec_len: int, bos_id: int = 1, eos_id: int = -1, ln_eps: float = 1e-5) -> AedConfig:
+                max_dec_len: int, bos_id: int = 1, eos_id: int = -1, ln_eps: float = 1e-5,
+                cross_kv_e4m3: bool = False) -> AedConfig:
     return AedConfig(model["n_layers"], model["d_model"], model["n_heads"], model["d_ffn"], model["vocab"],
                      model["d_enc"], AED_DTYPE_BF16 if dtype == "bf16" else AED_DTYPE_F32, max_batch,
-                     max_total_enc_frames, max_enc_len, max_dec_len, bos_id, eos_id, ln_eps, None, 0, None)
+                     max_total_enc_frames, max_enc_len, max_dec_len, bos_id, eos_id, ln_eps,
+                     AED_CROSS_KV_E4M3 if cross_kv_e4m3 else AED_CROSS_KV_DTYPE, None, 0, None)
 
 
 def workspace_bytes(cfg: AedConfig) -> int:
@@ -130,7 +133,7 @@ class Decoder:
 
     def __init__(self, model: Dict[str, int], weights: Dict[str, object], dtype: str = "fp32", *, max_batch: int,
                  max_total_enc_frames: int, max_enc_len: int, max_dec_len: int, bos_id: int = 1, eos_id: int = -1,
-                 ln_eps: float = 1e-5, device: str = "cuda:0", stream=None):
+                 ln_eps: float = 1e-5, device: str = "cuda:0", stream=None, cross_kv_e4m3: bool = False):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -142,7 +145,7 @@ class Decoder:
         self.handle = C.c_void_p()
         self.cfg = make_config(model, dtype, max_batch=max_batch, max_total_enc_frames=max_total_enc_frames,
                                max_enc_len=max_enc_len, max_dec_len=max_dec_len, bos_id=bos_id, eos_id=eos_id,
-                               ln_eps=ln_eps)
+                               ln_eps=ln_eps, cross_kv_e4m3=cross_kv_e4m3)
         need = int(self.lib.aed_dec_workspace_bytes(C.byref(self.cfg)))
         if need == 0:
             # let create produce the precise error
@@ -305,9 +308,9 @@ class Decoder:
 
 
 def decoder_for_workload(w, *, max_batch: Optional[int] = None, max_dec_len: Optional[int] = None,
-                         device: str = "cuda:0", eos_id: Optional[int] = None) -> Decoder:
+                         device: str = "cuda:0", eos_id: Optional[int] = None, cross_kv_e4m3: bool = False) -> Decoder:
     """A Decoder sized for one seeded workload (see ``workloads.make_workload``)."""
     return Decoder(w.model, w.weights, w.dtype, max_batch=max_batch or w.batch,
                    max_total_enc_frames=int(w.enc_lens.sum()), max_enc_len=int(w.enc_lens.max()),
                    max_dec_len=max_dec_len or int(w.dec_lens.max()), bos_id=w.bos_id,
-                   eos_id=w.eos_id if eos_id is None else eos_id, ln_eps=w.ln_eps, device=device)
+                   eos_id=w.eos_id if eos_id is None else eos_id, ln_eps=w.ln_eps, device=device, cross_kv_e4m3=cross_kv_e4m3)

@@ -68,6 +68,8 @@ bool config_supported(const aed_dec_config_t &c, std::string *why)
         return fail("capacities must be positive");
     if (c.max_enc_len > c.max_total_enc_frames) return fail("max_enc_len exceeds max_total_enc_frames");
     if (!(c.ln_eps > 0.f)) return fail("ln_eps must be positive");
+    if (c.cross_kv_format != AED_CROSS_KV_DTYPE && c.cross_kv_format != AED_CROSS_KV_E4M3)
+        return fail("cross_kv_format must be AED_CROSS_KV_DTYPE or AED_CROSS_KV_E4M3");
     return true;
 }
 
@@ -77,6 +79,8 @@ bool shape_supported(const aed_dec_config_t &c, std::string *why)
     if (c.d_model % c.n_heads != 0 || c.d_model / c.n_heads != kHeadDim) return fail("head_dim must be 64");
     if (c.d_model % 64 || c.d_ffn % 64 || c.d_enc % 64) return fail("d_model, d_ffn and d_enc must be multiples of 64");
     if (c.d_model > 8192) return fail("d_model above 8192 is not supported");
+    if (c.cross_kv_format == AED_CROSS_KV_E4M3 && c.dtype != AED_DTYPE_BF16)
+        return fail("the 8-bit cross-attention K/V store needs the bf16 configuration");
     return true;
 }
 
@@ -90,7 +94,7 @@ Layout make_layout(const aed_dec_config_t &c)
     L.self_layer_elems = B * 2 * d * (size_t)c.max_dec_len;
     L.cross_layer_elems = 2 * d * (size_t)c.max_total_enc_frames;
     L.self_cache = take(L.self_layer_elems * c.n_layers * e);
-    L.cross_store = take(L.cross_layer_elems * c.n_layers * e);
+    L.cross_store = take(L.cross_layer_elems * c.n_layers * (c.cross_kv_format == AED_CROSS_KV_E4M3 ? 1 : e));
     L.x = take(B * d * 4);
     L.act = take(B * (d > F ? d : F) * 4);
     L.qkv = take(B * 3 * d * 4);
@@ -316,7 +320,7 @@ aed_status_t launch_attention_fused(aed_dec *dec, int rows_ub, int len_ub, const
                                     const float *ln_c2 = nullptr, bool pdl = false, const float *stats_x = nullptr)
 {
     ProfScope ps(dec, kCross ? KF_ATTN_CROSS : KF_ATTN_SELF);
-    int warps = (len_ub + kFusedChunk - 1) / kFusedChunk;
+    int warps = (len_ub + fused_chunk<T>() - 1) / fused_chunk<T>();
     if (warps < 2) warps = 2;                    // at least 64 threads: the merge uses one thread per head dimension
     if (warps > kFusedMaxWarps) warps = kFusedMaxWarps;
     // Attention starts early (programmatic launch) and holds each warp's first chunk in registers; rows longer than
@@ -752,8 +756,14 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.prefetch2_ptr = dec->at<T>(L.comp_w) + (size_t)((l + 1) % c.n_layers) * d * d; p.prefetch2_bytes = (size_t)d * d * e2;
         AED_TRY(launch_step_gemm<sg::B_PLAIN>(dec, KF_GEMM_O, m.o, dec->tc_src_att, d, d, rows_ub, p, nullptr, &m.o_qc, d));
         // 4. cross-attention; every block computes the LN2 statistics of its row of x_new itself
-        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
-                                                        nullptr, nullptr, nullptr, c1_qc, c2_qc, pdl, x)));
+        if (c.cross_kv_format == AED_CROSS_KV_E4M3) {
+            const fp8e4m3 *cross8 = dec->at<fp8e4m3>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+            AED_TRY((launch_attention_fused<fp8e4m3, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross8, c.max_total_enc_frames, att,
+                                                                  nullptr, nullptr, nullptr, c1_qc, c2_qc, pdl, x)));
+        } else {
+            AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, att,
+                                                            nullptr, nullptr, nullptr, c1_qc, c2_qc, pdl, x)));
+        }
         // 5. x += att Woc^T + boc ; side: clear the [q | k | v] rows for the next layer
         p = sg::StepGemmParams{};
         p.src = att; p.ld_src = d;
@@ -859,8 +869,14 @@ aed_status_t forward_step_planes(aed_dec *dec, int rows_ub, int self_len_ub, con
         p = sg::StepGemmParams{};
         p.out = qc; p.ldo = d;
         AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_QC, m.qc, nullptr, d, d, rows_ub, p, dec->tc_actd));
-        AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, nullptr,
-                                                        ad_hi, ad_lo, stats + stats_stride, c1_qc, c2_qc, pdl)));
+        if (c.cross_kv_format == AED_CROSS_KV_E4M3) {
+            const fp8e4m3 *cross8 = dec->at<fp8e4m3>(L.cross_store) + (size_t)l * L.cross_layer_elems;
+            AED_TRY((launch_attention_fused<fp8e4m3, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross8, c.max_total_enc_frames, nullptr,
+                                                                  ad_hi, ad_lo, stats + stats_stride, c1_qc, c2_qc, pdl)));
+        } else {
+            AED_TRY((launch_attention_fused<T, true, false>(dec, rows_ub, c.max_enc_len, qc, d, cross, c.max_total_enc_frames, nullptr,
+                                                            ad_hi, ad_lo, stats + stats_stride, c1_qc, c2_qc, pdl)));
+        }
         p = sg::StepGemmParams{};
         p.out = x; p.ldo = d; p.bias = (const T *)w.b_o_c;
         AED_TRY(launch_step_gemm<sg::B_PLANES>(dec, KF_GEMM_OC, m.oc, nullptr, d, d, rows_ub, p, dec->tc_actd));
@@ -907,7 +923,8 @@ aed_status_t precompute_tc(aed_dec *dec, const void *enc_base, long long enc_row
     p.frame_capacity = c.max_total_enc_frames;
     p.d_model = c.d_model; p.n_heads = c.n_heads; p.d_enc = c.d_enc;
     p.n_layers = c.n_layers;
-    p.store = dec->at<T>(L.cross_store);
+    p.store = dec->ws + L.cross_store;
+    p.store_e4m3 = c.cross_kv_format == AED_CROSS_KV_E4M3 ? 1 : 0;
     p.layer_elems = L.cross_layer_elems;
     p.bias = dec->at<const T *>(L.ckv_bias);
     p.state = dec->state();

@@ -1,6 +1,7 @@
 // Shared device helpers for the AED decoder kernels (sm_100a).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -125,6 +126,25 @@ __device__ __forceinline__ void load4(const __nv_bfloat16 *p, float (&v)[4])
     uint2 raw = *reinterpret_cast<const uint2 *>(p);
     v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
     v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+}
+
+// One byte of the 8-bit floating-point format E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no
+// infinities, largest finite value 448): the optional storage type of the cross-attention K/V store.
+struct fp8e4m3 { uint8_t bits; };
+
+// two floats -> two E4M3 bytes (lo in the low byte), round to nearest even, saturating at the largest finite value
+__device__ __forceinline__ uint16_t pack_e4m3x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// two E4M3 bytes -> two floats (exact)
+__device__ __forceinline__ float2 unpack_e4m3x2(uint16_t v)
+{
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(v));
+    return __half22float2(*reinterpret_cast<__half2 *>(&h2));
 }
 
 __device__ __forceinline__ float warp_sum(float v)

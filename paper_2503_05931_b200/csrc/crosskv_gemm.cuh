@@ -1,6 +1,7 @@
 // Cross-attention K/V of every layer in one persistent tensor-core GEMM (sm_100a).
 //
 //   store[l][k|v][head][frame][64] = bf16( enc[frame, :] . w_kv_c[l][feature, :] + b_kv_c[l][feature] )
+// (or rounded to the 8-bit format E4M3 instead of bf16 when the handle stores the cross-attention K/V in 8 bits)
 //
 // over the packed encoder frames (no padding rows).  One block per SM walks a list of output tiles
 // (128 frames x 256 features, K = d_enc in 64-wide k-blocks).  Tile order: groups of gridDim.x frame tiles outermost;
@@ -50,7 +51,8 @@ struct CkvParams {
     int frame_capacity;
     int d_model, n_heads, d_enc;
     int n_layers;
-    __nv_bfloat16 *store;             // layer 0; layers are layer_elems apart
+    void *store;                      // layer 0; layers are layer_elems elements apart; bf16, or E4M3 bytes if store_e4m3
+    int store_e4m3;
     size_t layer_elems;
     const __nv_bfloat16 *const *bias; // [n_layers] device pointers (entries may be null), or null
     DecState *state;
@@ -195,7 +197,7 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + static_cast<uint32_t>(buf * kTileN) + (static_cast<uint32_t>(quarter * 32) << 16);
-            __nv_bfloat16 *store = p.store + static_cast<size_t>(layer) * p.layer_elems;
+            const size_t layer_off = static_cast<size_t>(layer) * p.layer_elems;
             const __nv_bfloat16 *bias = p.bias ? p.bias[layer] : nullptr;
             for (int c0 = 0; c0 < kTileN; c0 += 16) {
                 float v[16];
@@ -203,17 +205,28 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
                 const int o = nt * kTileN + c0;                  // 16 consecutive features inside one head
                 if (!frame_ok || o >= 2 * p.d_model) continue;
                 const int kv = o / p.d_model, cc = o % p.d_model, h = cc / kHeadDim, e = cc % kHeadDim;
-                uint32_t packed[8];
+                if (bias) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float lo = v[2 * j] + (bias ? to_f32(bias[o + 2 * j]) : 0.f);
-                    const float hi = v[2 * j + 1] + (bias ? to_f32(bias[o + 2 * j + 1]) : 0.f);
-                    __nv_bfloat162 pair = __floats2bfloat162_rn(lo, hi);
-                    packed[j] = *reinterpret_cast<uint32_t *>(&pair);
+                    for (int j = 0; j < 16; ++j) v[j] += to_f32(bias[o + j]);
                 }
-                __nv_bfloat16 *dst = store + ((static_cast<size_t>(kv) * p.n_heads + h) * p.frame_capacity + frame) * kHeadDim + e;
-                reinterpret_cast<uint4 *>(dst)[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                reinterpret_cast<uint4 *>(dst)[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                const size_t elem = layer_off + ((static_cast<size_t>(kv) * p.n_heads + h) * p.frame_capacity + frame) * kHeadDim + e;
+                uint32_t packed[8];
+                if (p.store_e4m3) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        packed[j] = static_cast<uint32_t>(pack_e4m3x2(v[4 * j], v[4 * j + 1])) |
+                                    (static_cast<uint32_t>(pack_e4m3x2(v[4 * j + 2], v[4 * j + 3])) << 16);
+                    *reinterpret_cast<uint4 *>(static_cast<uint8_t *>(p.store) + elem) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        __nv_bfloat162 pair = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+                        packed[j] = *reinterpret_cast<uint32_t *>(&pair);
+                    }
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.store) + elem;
+                    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    reinterpret_cast<uint4 *>(dst)[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                }
             }
             // this warp is done with the buffer
             tc_fence_before_sync();

@@ -374,8 +374,8 @@ attn_partial_kernel(const DecState *state, const int32_t *__restrict__ active_li
 //   kAppend (self-attention): q row is [q | k | v]; k and v of the new position are stored first.
 //   Output: fp32 [row, d] (out) and/or bf16 high/low planes (out_hi/out_lo), whichever pointers are non-null.
 // ------------------------------------------------------------------------------------------------------------
-template <typename CT> struct Raw8;
-template <> struct Raw8<__nv_bfloat16> {
+template <typename CT> struct RawLane;
+template <> struct RawLane<__nv_bfloat16> {
     uint4 v;
     __device__ __forceinline__ void load(const __nv_bfloat16 *p) { v = *reinterpret_cast<const uint4 *>(p); }
     __device__ __forceinline__ void zero() { v = make_uint4(0u, 0u, 0u, 0u); }
@@ -397,7 +397,24 @@ template <> struct Raw8<__nv_bfloat16> {
         for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
     }
 };
-template <> struct Raw8<float> {
+template <> struct RawLane<fp8e4m3> {
+    uint2 v;                                                                   // 8 bytes = 8 values
+    __device__ __forceinline__ void load(const fp8e4m3 *p) { v = *reinterpret_cast<const uint2 *>(p); }
+    __device__ __forceinline__ void zero() { v = make_uint2(0u, 0u); }
+    __device__ __forceinline__ void set(const float (&f)[8])
+    {
+        v.x = static_cast<uint32_t>(pack_e4m3x2(f[0], f[1])) | (static_cast<uint32_t>(pack_e4m3x2(f[2], f[3])) << 16);
+        v.y = static_cast<uint32_t>(pack_e4m3x2(f[4], f[5])) | (static_cast<uint32_t>(pack_e4m3x2(f[6], f[7])) << 16);
+    }
+    __device__ __forceinline__ void store(fp8e4m3 *p) const { *reinterpret_cast<uint2 *>(p) = v; }
+    __device__ __forceinline__ void get(float (&f)[8]) const
+    {
+        const float2 a = unpack_e4m3x2(static_cast<uint16_t>(v.x & 0xFFFFu)), b = unpack_e4m3x2(static_cast<uint16_t>(v.x >> 16));
+        const float2 c = unpack_e4m3x2(static_cast<uint16_t>(v.y & 0xFFFFu)), d = unpack_e4m3x2(static_cast<uint16_t>(v.y >> 16));
+        f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y; f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
+    }
+};
+template <> struct RawLane<float> {
     float4 a, b;
     __device__ __forceinline__ void load(const float *p) { a = *reinterpret_cast<const float4 *>(p); b = *reinterpret_cast<const float4 *>(p + 4); }
     __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
@@ -407,14 +424,29 @@ template <> struct Raw8<float> {
     { f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w; }
 };
 
-constexpr int kFusedChunk = 16;       // positions per warp and iteration
+// Head dimensions per lane.  8 for every storage type: with single-byte keys and values, 16 per lane (one 16-byte load
+// per row and lane, 32 positions per warp and pass) was measured slower at 512 rows (693 against 654 ms per pass of
+// the 24-layer batch-512 workload): the kernel is bound by how many loads its resident warps keep in flight, not by
+// bytes per load, and the wider lanes cost a resident block per SM.
+template <typename CT> struct LaneWidth { static constexpr int kE = 8; };
+// positions per warp and iteration: 4 passes over the 32 / (64 / kE) position groups of a warp
+template <typename CT> constexpr int fused_chunk() { return 4 * (32 / (kHeadDim / LaneWidth<CT>::kE)); }
 constexpr int kFusedMaxWarps = 8;
+
+template <int N> __device__ __forceinline__ void load_n(const float *p, float (&v)[N])
+{
+#pragma unroll
+    for (int i = 0; i < N; i += 4) {
+        const float4 a = *reinterpret_cast<const float4 *>(p + i);
+        v[i] = a.x; v[i + 1] = a.y; v[i + 2] = a.z; v[i + 3] = a.w;
+    }
+}
 
 // kPipe: the loads of a warp's next chunk are issued before the current chunk is reduced (twice the K/V registers,
 // so only two blocks per SM: for grids that fit anyway).
 // kRowStats: the block computes (mean, rstd) of its row of stats_x itself instead of reading ln_stats.
 template <typename CT, bool kCross, bool kAppend, bool kPipe = false, bool kRowStats = false>
-__global__ void __launch_bounds__(kFusedMaxWarps * 32, ((kAppend || kPipe) ? 2 : 4))      // self-attention holds the new key/value as well
+__global__ void __launch_bounds__(kFusedMaxWarps * 32, ((kAppend || kPipe) ? 2 : (LaneWidth<CT>::kE > 8 ? 3 : 4)))      // self-attention holds the new key/value as well; wider lanes need more registers
 attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, const float *__restrict__ q, int ldq,
                   CT *__restrict__ cache, int n_heads, int seq_capacity, float scale,
                   float *__restrict__ out, __nv_bfloat16 *__restrict__ out_hi, __nv_bfloat16 *__restrict__ out_lo, int ldo,
@@ -450,28 +482,29 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     // Positions that earlier steps (or the precompute) wrote are static for this kernel; the position appended
     // by this step (self-attention only) is taken from the projection output after the dependency wait.
     const int len_static = (kAppend && !kCross) ? len - 1 : len;
-    const int dg = lane & 7, pg = lane >> 3;
-    Raw8<CT> rk[4], rv[4];
+    constexpr int kE = LaneWidth<CT>::kE, kDG = kHeadDim / kE, kPG = 32 / kDG, kChunk = 4 * kPG;
+    const int dg = lane % kDG, pg = lane / kDG;      // lanes: kDG groups of kE head dimensions x kPG positions
+    RawLane<CT> rk[4], rv[4];
     // Self-attention without an append of its own (prefill pass): the cache positions it reads are written by the
     // kernel before it, so nothing is loaded ahead of the dependency wait.
     if (!kCross && !kAppend) asm volatile("griddepcontrol.wait;" ::: "memory");
     {
         // This warp's first chunk starts streaming while the kernel that produces the query is still running.
-        const int p0 = warp * kFusedChunk;
+        const int p0 = warp * kChunk;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int p = p0 + i * 4 + pg;
+            const int p = p0 + i * kPG + pg;
             if (p < len_static) {
-                rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
-                rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
+                rk[i].load(kbase + (size_t)p * kHeadDim + dg * kE);
+                rv[i].load(vbase + (size_t)p * kHeadDim + dg * kE);
             } else { rk[i].zero(); rv[i].zero(); }
         }
         // later chunks of this warp: pull them into L2 now (one 128-byte row per lane group)
         if (dg == 0) {
-            for (int q0 = p0 + n_warps * kFusedChunk; q0 < len_static; q0 += n_warps * kFusedChunk) {
+            for (int q0 = p0 + n_warps * kChunk; q0 < len_static; q0 += n_warps * kChunk) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int p = q0 + i * 4 + pg;
+                    const int p = q0 + i * kPG + pg;
                     if (p < len_static) {
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(kbase + (size_t)p * kHeadDim));
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(vbase + (size_t)p * kHeadDim));
@@ -482,17 +515,17 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     }
     // The LayerNorm-fold constants of this block's columns are static as well (read once per step and layer, so
     // they come from DRAM): requested here, before the dependency wait.
-    const int new_chunk = (len - 1) / kFusedChunk;
+    const int new_chunk = (len - 1) / kChunk;
     const bool owns_new = kAppend && !kCross && warp == new_chunk % n_warps;
     const int d_model = n_heads * kHeadDim;
-    const int qcol = h * kHeadDim + dg * 8;
-    float qc1[8], qc2[8], kc1[8], kc2[8], vc1[8], vc2[8];
+    const int qcol = h * kHeadDim + dg * kE;
+    float qc1[kE], qc2[kE], kc1[kE], kc2[kE], vc1[kE], vc2[kE];
     const bool fold = ln_stats != nullptr || kRowStats;
     if (fold) {
-        load8(ln_c1 + qcol, qc1); load8(ln_c2 + qcol, qc2);
+        load_n<kE>(ln_c1 + qcol, qc1); load_n<kE>(ln_c2 + qcol, qc2);
         if (owns_new) {
-            load8(ln_c1 + d_model + qcol, kc1); load8(ln_c2 + d_model + qcol, kc2);
-            load8(ln_c1 + 2 * d_model + qcol, vc1); load8(ln_c2 + 2 * d_model + qcol, vc2);
+            load_n<kE>(ln_c1 + d_model + qcol, kc1); load_n<kE>(ln_c2 + d_model + qcol, kc2);
+            load_n<kE>(ln_c1 + 2 * d_model + qcol, vc1); load_n<kE>(ln_c2 + 2 * d_model + qcol, vc2);
         }
     }
     AED_TRACE_RESERVE(tcur, state, (threadIdx.x == 0 && blockIdx.x == 0) ? 4u : 0u);
@@ -504,12 +537,12 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     // warp that owns the new position) the new key and value.  When the projection ran on gamma*x, its raw output
     // y becomes rstd*(y - mean*c1) + c2 here.
     float2 st = make_float2(0.f, 1.f);
-    float qv[8], kn[8], vn[8];
+    float qv[kE], kn[kE], vn[kE];
     if (ln_stats) st = ln_stats[r];
-    load8(q + (size_t)r * ldq + qcol, qv);
+    load_n<kE>(q + (size_t)r * ldq + qcol, qv);
     if (owns_new) {
-        load8(q + (size_t)r * ldq + d_model + qcol, kn);
-        load8(q + (size_t)r * ldq + 2 * d_model + qcol, vn);
+        load_n<kE>(q + (size_t)r * ldq + d_model + qcol, kn);
+        load_n<kE>(q + (size_t)r * ldq + 2 * d_model + qcol, vn);
     }
     if (kRowStats) {
         // mean and rstd of row r in one pass over deviations from the row's first element (a row whose mean is far
@@ -535,15 +568,15 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
     }
     if (fold) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * qc1[i], qc2[i]);
+        for (int i = 0; i < kE; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * qc1[i], qc2[i]);
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) qv[i] *= scale;
-    Raw8<CT> new_k, new_v;
+    for (int i = 0; i < kE; ++i) qv[i] *= scale;
+    RawLane<CT> new_k, new_v;
     if (owns_new) {
         if (fold) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < kE; ++i) {
                 kn[i] = fmaf(st.y, kn[i] - st.x * kc1[i], kc2[i]);
                 vn[i] = fmaf(st.y, vn[i] - st.x * vc1[i], vc2[i]);
             }
@@ -551,73 +584,72 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         new_k.set(kn);
         new_v.set(vn);
         if (pg == 0) {      // append to the cache; no other block reads this position during the kernel
-            new_k.store(const_cast<CT *>(kbase) + (size_t)(len - 1) * kHeadDim + dg * 8);
-            new_v.store(const_cast<CT *>(vbase) + (size_t)(len - 1) * kHeadDim + dg * 8);
+            new_k.store(const_cast<CT *>(kbase) + (size_t)(len - 1) * kHeadDim + dg * kE);
+            new_v.store(const_cast<CT *>(vbase) + (size_t)(len - 1) * kHeadDim + dg * kE);
         }
     }
 
-    float m = -INFINITY, l = 0.f, acc[8];
+    float m = -INFINITY, l = 0.f, acc[kE];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int i = 0; i < kE; ++i) acc[i] = 0.f;
     bool loaded = true;
-    Raw8<CT> nk[4], nv[4];
-    for (int p0 = warp * kFusedChunk; p0 < len; p0 += n_warps * kFusedChunk) {
+    RawLane<CT> nk[4], nv[4];
+    for (int p0 = warp * kChunk; p0 < len; p0 += n_warps * kChunk) {
         if (kPipe) {
-            const int pn = p0 + n_warps * kFusedChunk;
+            const int pn = p0 + n_warps * kChunk;
             if (pn < len) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int p = pn + i * 4 + pg;
+                    const int p = pn + i * kPG + pg;
                     if (p < len_static) {
-                        nk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
-                        nv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
+                        nk[i].load(kbase + (size_t)p * kHeadDim + dg * kE);
+                        nv[i].load(vbase + (size_t)p * kHeadDim + dg * kE);
                     } else { nk[i].zero(); nv[i].zero(); }
                 }
             }
         } else if (!loaded) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {          // keys and values of the chunk are requested together
-                const int p = p0 + i * 4 + pg;
+                const int p = p0 + i * kPG + pg;
                 if (p < len_static) {
-                    rk[i].load(kbase + (size_t)p * kHeadDim + dg * 8);
-                    rv[i].load(vbase + (size_t)p * kHeadDim + dg * 8);
+                    rk[i].load(kbase + (size_t)p * kHeadDim + dg * kE);
+                    rv[i].load(vbase + (size_t)p * kHeadDim + dg * kE);
                 } else { rk[i].zero(); rv[i].zero(); }
             }
         }
         loaded = false;
-        if (owns_new && p0 == new_chunk * kFusedChunk) {
+        if (owns_new && p0 == new_chunk * kChunk) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                if (p0 + i * 4 + pg == len - 1) { rk[i] = new_k; rv[i] = new_v; }
+                if (p0 + i * kPG + pg == len - 1) { rk[i] = new_k; rv[i] = new_v; }
         }
         float s[4], cmax = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            float kf[8], d = 0.f;
+            float kf[kE], d = 0.f;
             rk[i].get(kf);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) d = fmaf(qv[j], kf[j], d);
-            d += __shfl_xor_sync(0xffffffffu, d, 1);
-            d += __shfl_xor_sync(0xffffffffu, d, 2);
-            d += __shfl_xor_sync(0xffffffffu, d, 4);
-            s[i] = (p0 + i * 4 + pg < len) ? d : -INFINITY;
+            for (int j = 0; j < kE; ++j) d = fmaf(qv[j], kf[j], d);
+#pragma unroll
+            for (int o = 1; o < kDG; o <<= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            s[i] = (p0 + i * kPG + pg < len) ? d : -INFINITY;
             cmax = fmaxf(cmax, s[i]);
         }
-        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 8));
-        cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, 16));     // chunk max, uniform over the warp, finite
+#pragma unroll
+        for (int o = kDG; o < 32; o <<= 1) cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));     // chunk max, uniform over the warp, finite
         const float m_new = fmaxf(m, cmax);
         const float corr = expf(m - m_new);
         l *= corr;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] *= corr;
+        for (int j = 0; j < kE; ++j) acc[j] *= corr;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const float pr = expf(s[i] - m_new);      // exp(-inf) = 0 for positions past the end
-            float vf[8];
+            float vf[kE];
             rv[i].get(vf);
             l += pr;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) acc[j] = fmaf(pr, vf[j], acc[j]);
+            for (int j = 0; j < kE; ++j) acc[j] = fmaf(pr, vf[j], acc[j]);
         }
         m = m_new;
         if (kPipe) {
@@ -625,18 +657,17 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             for (int i = 0; i < 4; ++i) { rk[i] = nk[i]; rv[i] = nv[i]; }
         }
     }
-    // sum the 4 position groups (they share m)
-    l += __shfl_xor_sync(0xffffffffu, l, 8);
-    l += __shfl_xor_sync(0xffffffffu, l, 16);
+    // sum the position groups (they share m)
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 8);
-        acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 16);
+    for (int o = kDG; o < 32; o <<= 1) {
+        l += __shfl_xor_sync(0xffffffffu, l, o);
+#pragma unroll
+        for (int j = 0; j < kE; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
     }
     if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
     if (pg == 0) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) sm_acc[warp][dg * 8 + j] = acc[j];
+        for (int j = 0; j < kE; ++j) sm_acc[warp][dg * kE + j] = acc[j];
     }
     __syncthreads();
     if (threadIdx.x < kHeadDim) {

@@ -7,10 +7,10 @@ TOL = {"fp32": 1e-4, "bf16": 3e-2}       # max-abs tolerance on teacher-forced l
 MARGIN = 0.1                             # greedy ids must match where the checker's top-2 margin exceeds this
 
 
-def oracle_reference(w, rows=None, want_logits=True, n_threads=0, eos=-1):
+def oracle_reference(w, rows=None, want_logits=True, n_threads=0, eos=-1, cross_kv_e4m3=False):
     """Free-running greedy decode of the given utterances (default: all) by the CPU checker."""
     sub = w if rows is None else w.subset(rows)
-    model = orc.Model(w.model, w.weights, ln_eps=w.ln_eps)
+    model = orc.Model(w.model, w.weights, ln_eps=w.ln_eps, cross_kv_e4m3=cross_kv_e4m3)
     return orc.decode_batch(model, sub.enc, sub.enc_lens, sub.dec_lens, bos=w.bos_id, want_logits=want_logits,
                             n_threads=n_threads, eos=eos)
 

@@ -18,6 +18,7 @@
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
 #include "crosskv_gemm.cuh"
+#include "stream_schedule.h"
 
 using namespace aed;
 
@@ -1530,59 +1531,50 @@ extern "C" aed_status_t aed_dec_decode_stream(aed_dec_t *dec, const void *enc_pa
     }
     AED_TRY(aed_dec_open_slots(dec, slots));
     const Layout &L = dec->lay;
-    int32_t *toks = dec->at<int32_t>(L.slot_tokens), *lens = dec->at<int32_t>(L.slot_lens);
-    const int ld = c.max_dec_len;
     if (off[n] > 0x7fffffffLL) return fail(dec, AED_ERR_CAPACITY, "the stream has %lld encoder frames; at most 2^31 - 1 per call", off[n]);
-    std::vector<int> occupant(slots, -1), remaining(slots, 0);
-    std::vector<int32_t> lens_host(slots, 0);
-    int next = 0;
-    long long steps = 0, row_steps = 0;
-    auto fill = [&]() -> aed_status_t {
-        Admission adm[ckv::kMaxSegs];
-        int k = 0;
-        for (int s = 0; s < slots && next < n; ++s) {
-            if (occupant[s] >= 0) continue;
-            const int u = order ? order[next] : next;
-            ++next;
-            adm[k++] = Admission{s, off[u], enc_lens[u], max_lens[u]};
-            occupant[s] = u;
-            remaining[s] = max_lens[u];
-            if (k == ckv::kMaxSegs) { AED_TRY(admit_many(dec, enc_packed, off[n], adm, k, lens)); k = 0; }
+    // The scheduling decisions are in stream_schedule.h; here are its operations on the device.
+    struct Ops {
+        aed_dec *dec;
+        const void *enc_packed;
+        const std::vector<long long> &off;
+        const int32_t *enc_lens, *max_lens;
+        int32_t *toks, *lens, *tokens_out, *out_lens;
+        int ld, slots;
+        int admit(const StreamAdmission *a, int k)
+        {
+            Admission adm[ckv::kMaxSegs];
+            for (int i = 0; i < k; ++i) adm[i] = Admission{a[i].slot, off[a[i].utterance], enc_lens[a[i].utterance], max_lens[a[i].utterance]};
+            return admit_many(dec, enc_packed, off.back(), adm, k, lens);
         }
-        if (k) AED_TRY(admit_many(dec, enc_packed, off[n], adm, k, lens));
-        return AED_OK;
-    };
-    // The finished utterance's tokens and length go to the host behind the steps that produced them and before the
-    // slot's next occupant (stream order); with pinned host buffers the host does not wait for them.
-    auto harvest = [&](int s) -> aed_status_t {
-        const int u = occupant[s];
-        AED_CUDA(dec, cudaMemcpyAsync(tokens_out + (size_t)u * ld, toks + (size_t)s * ld, (size_t)max_lens[u] * 4, cudaMemcpyDeviceToHost, dec->stream));
-        AED_CUDA(dec, cudaMemcpyAsync(out_lens + u, lens + s, 4, cudaMemcpyDeviceToHost, dec->stream));
-        occupant[s] = -1;
-        return AED_OK;
-    };
-    AED_TRY(fill());
-    for (;;) {
-        int busy = 0, lo = 1 << 30, hi = 0;
-        for (int s = 0; s < slots; ++s)
-            if (occupant[s] >= 0) { ++busy; lo = std::min(lo, remaining[s]); hi = std::max(hi, remaining[s]); }
-        if (!busy) break;
-        // without an end-of-sequence id the host knows the step in which the next utterance leaves
-        const int want = eos ? std::min(poll_steps, hi) : lo;
-        int32_t done = 0;
-        AED_TRY(aed_dec_greedy_steps(dec, want, toks, lens, &done));
-        steps += done;
-        for (int s = 0; s < slots; ++s)
-            if (occupant[s] >= 0) { row_steps += std::min<int>(done, remaining[s]); remaining[s] = std::max(remaining[s] - done, 0); }
-        if (eos) {
-            AED_CUDA(dec, cudaMemcpyAsync(lens_host.data(), lens, (size_t)slots * 4, cudaMemcpyDeviceToHost, dec->stream));
-            AED_CUDA(dec, cudaStreamSynchronize(dec->stream));
+        int steps(int want, int *done)
+        {
+            int32_t d = 0;
+            const aed_status_t st = aed_dec_greedy_steps(dec, want, toks, lens, &d);
+            *done = d;
+            return st;
         }
-        for (int s = 0; s < slots; ++s)
-            if (occupant[s] >= 0 && (remaining[s] == 0 || (eos && lens_host[s] > 0))) AED_TRY(harvest(s));
-        AED_TRY(fill());
-        if (done == 0 && next >= n) break;
-    }
+        int read_lens(int32_t *host)
+        {
+            if (cudaMemcpyAsync(host, lens, (size_t)slots * 4, cudaMemcpyDeviceToHost, dec->stream) != cudaSuccess ||
+                cudaStreamSynchronize(dec->stream) != cudaSuccess)
+                return fail(dec, AED_ERR_CUDA, "reading the slot lengths: %s", cudaGetErrorString(cudaGetLastError()));
+            return AED_OK;
+        }
+        // The finished utterance's tokens and length go to the host behind the steps that produced them and before
+        // the slot's next occupant (stream order); with pinned host buffers the host does not wait for them.
+        int harvest(int s, int u)
+        {
+            if (cudaMemcpyAsync(tokens_out + (size_t)u * ld, toks + (size_t)s * ld, (size_t)max_lens[u] * 4, cudaMemcpyDeviceToHost, dec->stream) != cudaSuccess ||
+                cudaMemcpyAsync(out_lens + u, lens + s, 4, cudaMemcpyDeviceToHost, dec->stream) != cudaSuccess)
+                return fail(dec, AED_ERR_CUDA, "copying a finished utterance out: %s", cudaGetErrorString(cudaGetLastError()));
+            return AED_OK;
+        }
+    } ops{dec, enc_packed, off, enc_lens, max_lens, dec->at<int32_t>(L.slot_tokens), dec->at<int32_t>(L.slot_lens), tokens_out,
+          out_lens, c.max_dec_len, slots};
+    StreamTotals tot;
+    const int rc = run_stream_schedule(n, slots, order, max_lens, eos, poll_steps, ckv::kMaxSegs, ops, &tot);
+    if (rc < 0) return static_cast<aed_status_t>(rc);
+    const long long steps = tot.steps, row_steps = tot.row_steps;
     if (steps_out) *steps_out = steps;
     if (row_steps_out) *row_steps_out = row_steps;
     return aed_dec_sync_status(dec);

@@ -87,3 +87,45 @@ def greedy_compare(dec, w, ref, rows=None):
             compared += 1
     assert compared == comparable_tokens(w, ref, rows)
     return compared, toks
+
+
+def sinusoid(t, d):
+    """PE(t) of the decoder's definition, written out with math.sin / math.cos."""
+    import math
+    pe = np.zeros(d)
+    for i in range(0, d, 2):
+        ang = t / (10000.0 ** (i / d))
+        pe[i], pe[i + 1] = math.sin(ang), math.cos(ang)
+    return pe
+
+
+def torch_layer_logits(model, weights, enc, forced, ln_eps=1e-5):
+    """Teacher-forced logits of one utterance from torch.nn.TransformerDecoderLayer(norm_first=True) in fp64, a final
+    LayerNorm and a Linear: the library routine that pins the checker's layer."""
+    import math
+    import torch
+    d, NL, L = model["d_model"], model["n_layers"], len(forced)
+    t64 = lambda a: torch.tensor(np.asarray(a), dtype=torch.float64)
+    x = torch.stack([t64(weights["embed"][y]) * math.sqrt(d) + t64(sinusoid(t, d)) for t, y in enumerate(forced)])[None]
+    mem = t64(enc)[None]
+    mask = torch.nn.Transformer.generate_square_subsequent_mask(L, dtype=torch.float64)
+    with torch.no_grad():
+        for l in range(NL):
+            lay = torch.nn.TransformerDecoderLayer(d, model["n_heads"], model["d_ffn"], dropout=0.0, activation="relu",
+                                                   batch_first=True, norm_first=True, dtype=torch.float64)
+            lay.self_attn.in_proj_weight.copy_(t64(weights["w_qkv"][l])); lay.self_attn.in_proj_bias.copy_(t64(weights["b_qkv"][l]))
+            lay.self_attn.out_proj.weight.copy_(t64(weights["w_o"][l])); lay.self_attn.out_proj.bias.copy_(t64(weights["b_o"][l]))
+            lay.multihead_attn.in_proj_weight.copy_(t64(np.concatenate([weights["w_q_c"][l], weights["w_kv_c"][l]])))
+            lay.multihead_attn.in_proj_bias.copy_(t64(np.concatenate([weights["b_q_c"][l], weights["b_kv_c"][l]])))
+            lay.multihead_attn.out_proj.weight.copy_(t64(weights["w_o_c"][l])); lay.multihead_attn.out_proj.bias.copy_(t64(weights["b_o_c"][l]))
+            lay.linear1.weight.copy_(t64(weights["w_ff1"][l])); lay.linear1.bias.copy_(t64(weights["b_ff1"][l]))
+            lay.linear2.weight.copy_(t64(weights["w_ff2"][l])); lay.linear2.bias.copy_(t64(weights["b_ff2"][l]))
+            for i, nm in ((1, "ln1"), (2, "ln2"), (3, "ln3")):
+                getattr(lay, f"norm{i}").weight.copy_(t64(weights[nm + "_g"][l]))
+                getattr(lay, f"norm{i}").bias.copy_(t64(weights[nm + "_b"][l]))
+            x = lay.eval()(x, mem, tgt_mask=mask)
+        x = torch.nn.functional.layer_norm(x, (d,), t64(weights["final_ln_g"]), t64(weights["final_ln_b"]), ln_eps)
+        z = x @ t64(weights["w_out"]).T
+        if weights.get("b_out") is not None:
+            z = z + t64(weights["b_out"])
+    return z[0].numpy()

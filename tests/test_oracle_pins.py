@@ -9,6 +9,7 @@ import torch
 
 from oracle import aed_oracle as orc
 from paper_2503_05931_b200 import workloads as wl
+from tests.helpers import torch_layer_logits
 
 SMALL = dict(n_layers=2, d_model=32, n_heads=4, d_ffn=64, vocab=50, d_enc=32)
 
@@ -252,34 +253,7 @@ def test_matches_torch_transformer_decoder_layer(seed):
     forced = rng.integers(0, model["vocab"], size=L)
     out = orc.decode(m, w.enc, L, forced=forced)
 
-    t64 = lambda a: torch.tensor(np.asarray(a), dtype=torch.float64)
-    layers = []
-    for l in range(NL):
-        lay = torch.nn.TransformerDecoderLayer(d, model["n_heads"], model["d_ffn"], dropout=0.0, activation="relu",
-                                               batch_first=True, norm_first=True, dtype=torch.float64)
-        with torch.no_grad():
-            lay.self_attn.in_proj_weight.copy_(t64(w.weights["w_qkv"][l]))
-            lay.self_attn.in_proj_bias.copy_(t64(w.weights["b_qkv"][l]))
-            lay.self_attn.out_proj.weight.copy_(t64(w.weights["w_o"][l]))
-            lay.self_attn.out_proj.bias.copy_(t64(w.weights["b_o"][l]))
-            lay.multihead_attn.in_proj_weight.copy_(t64(np.concatenate([w.weights["w_q_c"][l], w.weights["w_kv_c"][l]])))
-            lay.multihead_attn.in_proj_bias.copy_(t64(np.concatenate([w.weights["b_q_c"][l], w.weights["b_kv_c"][l]])))
-            lay.multihead_attn.out_proj.weight.copy_(t64(w.weights["w_o_c"][l]))
-            lay.multihead_attn.out_proj.bias.copy_(t64(w.weights["b_o_c"][l]))
-            lay.linear1.weight.copy_(t64(w.weights["w_ff1"][l])); lay.linear1.bias.copy_(t64(w.weights["b_ff1"][l]))
-            lay.linear2.weight.copy_(t64(w.weights["w_ff2"][l])); lay.linear2.bias.copy_(t64(w.weights["b_ff2"][l]))
-            for i, nm in ((1, "ln1"), (2, "ln2"), (3, "ln3")):
-                getattr(lay, f"norm{i}").weight.copy_(t64(w.weights[nm + "_g"][l]))
-                getattr(lay, f"norm{i}").bias.copy_(t64(w.weights[nm + "_b"][l]))
-        layers.append(lay.eval())
-    x = torch.stack([t64(w.weights["embed"][y]) * math.sqrt(d) + t64(pos_enc(t, d)) for t, y in enumerate(forced)])[None]
-    mem = t64(w.enc)[None]
-    mask = torch.nn.Transformer.generate_square_subsequent_mask(L, dtype=torch.float64)
-    with torch.no_grad():
-        for lay in layers:
-            x = lay(x, mem, tgt_mask=mask)
-        x = torch.nn.functional.layer_norm(x, (d,), t64(w.weights["final_ln_g"]), t64(w.weights["final_ln_b"]), 1e-5)
-        z = (x @ t64(w.weights["w_out"]).T + t64(w.weights["b_out"]))[0].numpy()
+    z = torch_layer_logits(model, w.weights, w.enc, forced)
     assert np.max(np.abs(z)) > 0.5          # the comparison is not vacuous
     np.testing.assert_allclose(out["logits"], z, atol=1e-10)
     assert np.array_equal(out["next"], z.argmax(-1))

@@ -37,6 +37,16 @@ int rows_bucket(int rows)
     return b;
 }
 
+// Row count a step graph is captured for.  Kernels whose grids follow the row count (attention: one block per row and
+// head) pay for every row of the grid, also for those beyond the device-side count, whose blocks only find out that
+// they have nothing to do; so the graphs are keyed finer than the power-of-two tiles of the projections: multiples of 8
+// up to 64 rows, of 16 up to 256, of 32 beyond.  Never above rows_bucket(rows).
+int rows_key(int rows)
+{
+    const int g = rows <= 64 ? 8 : rows <= 256 ? 16 : 32;
+    return (rows + g - 1) / g * g;
+}
+
 struct LayerWeights {
     const void *ln1_g, *ln1_b, *w_qkv, *b_qkv, *w_o, *b_o;
     const void *ln2_g, *ln2_b, *w_q_c, *b_q_c, *w_kv_c, *b_kv_c, *w_o_c, *b_o_c;
@@ -1332,8 +1342,8 @@ extern "C" aed_status_t aed_dec_greedy_decode(aed_dec_t *dec, const int32_t *max
         }
         const int rows_ub = alive[s];
         if (dec->use_graphs && !dec->profiling) {
-            // grids are sized for the bucket; kernels leave rows beyond the device-side row count alone
-            const int rows_b = rows_bucket(rows_ub), chunks = (s + 1 + kAttnChunk - 1) / kAttnChunk;
+            // grids are sized for the keyed row count; kernels leave rows beyond the device-side row count alone
+            const int rows_b = rows_key(rows_ub), chunks = (s + 1 + kAttnChunk - 1) / kAttnChunk;
             const aed_dec::GraphKey key(rows_b, chunks, tokens_out, out_lens);
             auto it = dec->graphs.find(key);
             if (it == dec->graphs.end()) {
@@ -1482,7 +1492,7 @@ extern "C" aed_status_t aed_dec_greedy_steps(aed_dec_t *dec, int32_t n_steps, in
             if (dec->slot_t[u] >= 0 && dec->slot_t[u] < dec->slot_max[u]) { ++rows_ub; longest = std::max(longest, dec->slot_t[u] + 1); }
         if (rows_ub == 0) break;
         if (dec->use_graphs && !dec->profiling) {
-            const int rows_b = rows_bucket(rows_ub), chunks = (longest + kAttnChunk - 1) / kAttnChunk;
+            const int rows_b = rows_key(rows_ub), chunks = (longest + kAttnChunk - 1) / kAttnChunk;
             const aed_dec::GraphKey key(rows_b, chunks, tokens_out, out_lens);
             auto it = dec->graphs.find(key);
             if (it == dec->graphs.end()) {

@@ -107,6 +107,9 @@ NCU_TRAFFIC_RATIO = {
     # composite cross-query matrix (2.1 MB) and each prefetches the next layer's matrices of its kind into L2, which
     # under the profiler's serialised replay is a second DRAM read
     "step_gemm_kernel": 2.33,
+    # the same five launches at 16 and at 4 rows: 63.82 MB and 62.82 MB read
+    "step_gemv_staged_kernel": 2.17,
+    "step_gemv_kernel": 2.14,
     # self + cross attention of one layer at 64 rows: 0.84 + 31.05 MB for 0.52 + 30.49 MB of K/V
     "attn_fused_kernel": 1.03,
     # vocabulary projection: 33.85 MB for the 33.55 MB output matrix
@@ -363,6 +366,8 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=list(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--clip-batch", type=int, default=0,
+                    help="keep only this many utterances, those with the longest outputs (profiling captures of the few-row kernels)")
     ap.add_argument("--cross-kv", default="dtype", choices=["dtype", "e4m3"],
                     help="storage of the cross-attention K/V: the workload's dtype (the measured configuration) or 8-bit E4M3")
     ap.add_argument("--clip-len", type=int, default=0,
@@ -397,6 +402,9 @@ def main():
     # Every rank decodes its own batch of the same distribution (utterances are independent: no collective
     # on the data path, weak scaling).
     w = wl.make_workload(args.workload, seed=rank_seed(args.workload, rank))
+    if args.clip_batch > 0:
+        keep = np.sort(np.argsort(-w.dec_lens, kind="stable")[:args.clip_batch])
+        w = w.subset(keep)
     if args.clip_len > 0:
         w.dec_lens = np.minimum(w.dec_lens, args.clip_len).astype(np.int32)
     peaks = load_peaks()
@@ -466,7 +474,7 @@ def main():
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, **w.model, "batch_per_gpu": w.batch, "total_enc_frames": int(w.enc_lens.sum()),
-                       "total_out_tokens": n_tok, "decode_steps": Lmax, "clip_len": args.clip_len,
+                       "total_out_tokens": n_tok, "decode_steps": Lmax, "clip_len": args.clip_len, "clip_batch": args.clip_batch,
                        "cross_kv_store": "e4m3" if args.cross_kv == "e4m3" else w.dtype,
                        "l2": "inputs larger than L2 (weights + K/V stores stream every decode step)",
                        "step": "cross-K/V precompute + greedy decode of one batch"},
@@ -502,13 +510,24 @@ def profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step):
         return None
     total = sum(v["ms"] for v in prof.values())
     kernels = {}
+    m = w.model
+    e = 2 if w.dtype == "bf16" else 4
+    d, F = m["d_model"], m["d_ffn"]
+    # bytes of weights one launch of a projection call site reads (what the layer's definition contains)
+    site_weights = {"gemm_qkv": 3 * d * d, "gemm_o": d * d, "gemm_qc": d * d, "gemm_oc": d * d, "gemm_ff1": d * F, "gemm_ff2": d * F}
     for fam, v in prof.items():
-        k = kernels.setdefault(KERNEL_OF_FAMILY.get(fam, fam), {"ms": 0.0, "launches": 0, "bytes": 0.0, "families": []})
+        base, _, variant = fam.partition("@")                  # "gemm_qkv@gemv_staged": call site and the kernel that ran it
+        kernel = {"gemv": "step_gemv_kernel", "gemv_staged": "step_gemv_staged_kernel"}.get(variant, KERNEL_OF_FAMILY.get(base, base))
+        k = kernels.setdefault(kernel, {"ms": 0.0, "launches": 0, "bytes": 0.0, "families": []})
         k["ms"] += v["ms"]; k["launches"] += v["launches"]; k["families"].append(fam)
-        k["bytes"] += family_bytes(fam, w) or 0.0
-    if "gemm_qkv" in prof and "gemm_qc" not in prof:
-        # steps of at most 128 rows: the cross-attention query matrix is read by the launch that reads Wqkv
-        kernels["step_gemm_kernel"]["bytes"] += family_bytes("gemm_qc", w) or 0.0
+        if base in site_weights:
+            per_launch_w = site_weights[base]
+            # steps of at most 128 rows: the cross-attention query matrix is read by the launch that reads Wqkv
+            if base == "gemm_qkv" and not any(f.partition("@")[0] == "gemm_qc" for f in prof):
+                per_launch_w += d * d
+            k["bytes"] += e * per_launch_w * v["launches"]
+        else:
+            k["bytes"] += family_bytes(base, w) or 0.0
     top = max(kernels, key=lambda k: kernels[k]["ms"])
     info = kernels[top]
     share = info["ms"] / total
@@ -516,6 +535,10 @@ def profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step):
     per_launch = info["bytes"] / max(info["launches"], 1)
     achieved = info["bytes"] / (in_graph_ms * 1e-3) / 1e9 if info["bytes"] else None
     ratio = NCU_TRAFFIC_RATIO.get(top)
+    family_shares = {}
+    for fam, v in prof.items():
+        base = fam.partition("@")[0]
+        family_shares[base] = family_shares.get(base, 0.0) + v["ms"] / total
     return {"bound": "hbm", "kernel": top, "families": sorted(info["families"]), "achieved": achieved,
             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
             "traffic": ratio * per_launch if (ratio and per_launch) else None,
@@ -526,7 +549,7 @@ def profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step):
             "avg_us_ungraphed": 1e3 * info["ms"] / max(info["launches"], 1),
             "peak_source": peaks["source"],
             "shares": {k: round(v["ms"] / total, 4) for k, v in sorted(kernels.items(), key=lambda kv: -kv[1]["ms"])},
-            "family_shares": {k: round(v["ms"] / total, 4) for k, v in prof.items()}}
+            "family_shares": {k: round(v, 4) for k, v in family_shares.items()}}
 
 
 if __name__ == "__main__":

@@ -17,6 +17,7 @@
 #include "step_kernels.cuh"
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
+#include "step_gemv.cuh"
 #include "crosskv_gemm.cuh"
 #include "stream_schedule.h"
 
@@ -39,10 +40,11 @@ int rows_bucket(int rows)
 
 // Row count a step graph is captured for.  Kernels whose grids follow the row count (attention: one block per row and
 // head) pay for every row of the grid, also for those beyond the device-side count, whose blocks only find out that
-// they have nothing to do; so the graphs are keyed finer than the power-of-two tiles of the projections: multiples of 8
-// up to 64 rows, of 16 up to 256, of 32 beyond.  Never above rows_bucket(rows).
+// they have nothing to do; so the graphs are keyed finer than the power-of-two tiles of the projections: 4, then multiples
+// of 8 up to 64 rows, of 16 up to 256, of 32 beyond.  Never above rows_bucket(rows).
 int rows_key(int rows)
 {
+    if (rows <= 4) return 4;         // the projections of steps of at most 4 rows take a form of their own
     const int g = rows <= 64 ? 8 : rows <= 256 ? 16 : 32;
     return (rows + g - 1) / g * g;
 }
@@ -190,6 +192,9 @@ struct aed_dec {
     bool tc_target_fixed = false;         // set from the environment: use tc_target_ctas at every row count
     bool use_pdl = true;
     bool attn_pipe = true;
+    bool use_gemv = true;           // steps of few rows: projections by warp-level MMAs (step_gemv.cuh)
+    int gemv_rows = 32;             // ... up to this many rows
+    int gemv_direct_rows = 4;       // ... with the activation fragments straight from global memory up to this many
     int planes_rows = 128;                // steps with more rows make their activation planes once per projection input
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
     typedef std::tuple<int, int, const void *, const void *> GraphKey;
@@ -241,6 +246,10 @@ enum KernelFamily { KF_BOOKKEEPING = 0, KF_EMBED, KF_LAYERNORM, KF_GEMM_QKV, KF_
 const char *const kFamilyNames[KF_COUNT] = {"bookkeeping", "embed", "layernorm", "gemm_qkv", "attn_self", "attn_combine",
                                             "gemm_o", "gemm_qc", "attn_cross", "gemm_oc", "gemm_ff1", "gemm_ff2",
                                             "gemm_vocab", "precompute_cross_kv"};
+// The projections of steps with few rows run in kernels of their own (step_gemv.cuh); the profile keeps the call site
+// and says which kernel ran it: family + KF_COUNT * variant, reported as "gemm_qkv@gemv", "gemm_qkv@gemv_staged".
+enum { KV_TCGEN05 = 0, KV_GEMV = 1, KV_GEMV_STAGED = 2, KV_COUNT = 3 };
+const char *const kVariantSuffix[KV_COUNT] = {"", "@gemv", "@gemv_staged"};
 
 // Records an event before and after the launches issued while it is alive (profiling mode only).
 struct ProfScope {
@@ -515,7 +524,8 @@ aed_status_t tc_setup(aed_dec *dec)
     if (!ok) return fail(nullptr, AED_ERR_CUDA, "cuTensorMapEncodeTiled failed (are all weight tensors 16-byte aligned?)");
     const int smem = kTcSmemBudget + 1024;
     cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<tc::TC_EPI_LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv::crosskv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ckv::kStages * ckv::kStageBytes + 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv::crosskv_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ckv::kStages * ckv::kStageBytes + 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ckv::crosskv_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ckv::kStages * ckv::kStageBytes + 1024);
     // tensor maps and bias pointers of the cross-K/V weights: read by the precompute kernel from the workspace
     if (e == cudaSuccess) e = cudaMemcpyAsync(dec->ws + L.ckv_maps, kvc_maps.data(), kvc_maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, dec->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dec->ws + L.ckv_bias, kvc_bias.data(), kvc_bias.size() * sizeof(void *), cudaMemcpyHostToDevice, dec->stream);
@@ -529,6 +539,10 @@ aed_status_t tc_setup(aed_dec *dec)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_GAMMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_LN_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sg::step_gemm_kernel<sg::B_PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_PLAIN, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_GAMMA, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_LN_RELU, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4));
+
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
     // LayerNorm-fold constants of every layer
     for (int l = 0; l < c.n_layers; ++l) {
@@ -557,6 +571,12 @@ aed_status_t tc_setup(aed_dec *dec)
         dec->use_pdl = !(v && v[0] == '1');
         v = getenv("AED_DEC_NO_ATTN_PIPE");
         dec->attn_pipe = !(v && v[0] == '1');
+        v = getenv("AED_DEC_NO_GEMV");
+        dec->use_gemv = !(v && v[0] == '1');
+        v = getenv("AED_DEC_GEMV_ROWS");
+        if (v && atoi(v) >= 1 && atoi(v) <= 32) dec->gemv_rows = atoi(v);
+        v = getenv("AED_DEC_GEMV_DIRECT_ROWS");
+        if (v && atoi(v) >= 0 && atoi(v) <= 8) dec->gemv_direct_rows = atoi(v);
         v = getenv("AED_DEC_PLANES_ROWS");
         if (v && atoi(v) > 0) dec->planes_rows = atoi(v);
 
@@ -635,7 +655,6 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
 {
     // map_w2, M2: a second weight matrix [M2, K] over the same rows (its output, gamma and bias are in p)
     // plane_maps (B_PLANES only): [log2(N/16)][high, low] tensor maps of the ready-made activation planes
-    ProfScope ps(dec, family);
     // Rows per CTA tile: up to 128 (two ring stages still fit beside the transposition buffer); more rows are
     // covered by row tiles that re-read the weight tile from L2.
     int ni = tc_n_index(rows_ub);
@@ -667,6 +686,33 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     p.n_tile = n_tile;
     p.state = dec->state();
     p.eps = dec->cfg.ln_eps;
+    const bool gemv = MODE != sg::B_PLANES && dec->use_gemv && rows_ub <= dec->gemv_rows && kb_max <= sv::kSvMaxKb;
+    ProfScope ps(dec, family + KF_COUNT * (!gemv ? KV_TCGEN05 : rows_ub <= dec->gemv_direct_rows ? KV_GEMV : KV_GEMV_STAGED));
+    if constexpr (MODE != sg::B_PLANES) {
+        // Steps of at most 32 rows whose CTAs cover at most two k-blocks: warp-level MMAs (step_gemv.cuh), activation
+        // fragments straight from global memory up to 8 rows, through shared memory beyond
+        if (gemv) {
+            cudaLaunchConfig_t gc = {};
+            gc.gridDim = dim3(m_tiles, splits, 1);
+            gc.blockDim = dim3(sv::kSvThreads);
+            const bool direct = rows_ub <= dec->gemv_direct_rows;
+            const int nt = rows_ub <= 16 ? 2 : 4;
+            gc.dynamicSmemBytes = direct ? (size_t)sv::kSvMaxKb * tc::kATileBytes + 1024 : (size_t)sv::sv_staged_smem(nt);
+            gc.stream = dec->stream;
+            cudaLaunchAttribute ga[1];
+            ga[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            ga[0].val.programmaticStreamSerializationAllowed = dec->use_pdl ? 1 : 0;
+            gc.attrs = ga;
+            gc.numAttrs = 1;
+            const CUtensorMap &second = map_w2 ? *map_w2 : map_w;
+            cudaError_t ge = direct    ? cudaLaunchKernelEx(&gc, sv::step_gemv_kernel<MODE, 1>, map_w, second, p)
+                             : nt == 2 ? cudaLaunchKernelEx(&gc, sv::step_gemv_staged_kernel<MODE, 2>, map_w, second, p)
+                                       : cudaLaunchKernelEx(&gc, sv::step_gemv_staged_kernel<MODE, 4>, map_w, second, p);
+            if (ge != cudaSuccess) return fail(dec, AED_ERR_CUDA, "projection launch: %s", cudaGetErrorString(ge));
+            AED_LAUNCHED(dec);
+            return AED_OK;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(m_tiles, splits, row_tiles);
     cfg.blockDim = dim3(sg::kSgThreads);
@@ -935,14 +981,17 @@ aed_status_t precompute_tc(aed_dec *dec, const void *enc_base, long long enc_row
     p.d_model = c.d_model; p.n_heads = c.n_heads; p.d_enc = c.d_enc;
     p.n_layers = c.n_layers;
     p.store = dec->ws + L.cross_store;
-    p.store_e4m3 = c.cross_kv_format == AED_CROSS_KV_E4M3 ? 1 : 0;
     p.layer_elems = L.cross_layer_elems;
     p.bias = dec->at<const T *>(L.ckv_bias);
     p.state = dec->state();
     const long long tiles = (long long)segs.tile0[segs.n] * c.n_layers * ((2 * c.d_model + ckv::kTileN - 1) / ckv::kTileN);
     ProfScope ps(dec, KF_PRECOMPUTE);
-    ckv::crosskv_gemm_kernel<<<(unsigned)std::min<long long>(tiles, dec->sm_count), ckv::kCkvThreads, ckv::kStages * ckv::kStageBytes + 1024, dec->stream>>>(
-        map_enc, dec->at<CUtensorMap>(L.ckv_maps), p);
+    const unsigned grid = (unsigned)std::min<long long>(tiles, dec->sm_count);
+    const size_t smem = ckv::kStages * ckv::kStageBytes + 1024;
+    if (c.cross_kv_format == AED_CROSS_KV_E4M3)
+        ckv::crosskv_gemm_kernel<true><<<grid, ckv::kCkvThreads, smem, dec->stream>>>(map_enc, dec->at<CUtensorMap>(L.ckv_maps), p);
+    else
+        ckv::crosskv_gemm_kernel<false><<<grid, ckv::kCkvThreads, smem, dec->stream>>>(map_enc, dec->at<CUtensorMap>(L.ckv_maps), p);
     AED_LAUNCHED(dec);
     return AED_OK;
 }
@@ -1626,8 +1675,14 @@ extern "C" int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, co
 {
     if (!dec || !names || !ms || !launches || max_families < 1) return AED_ERR_INVALID_ARG;
     if (cudaStreamSynchronize(dec->stream) != cudaSuccess) return AED_ERR_CUDA;
-    double sum[KF_COUNT] = {0};
-    int64_t cnt[KF_COUNT] = {0};
+    double sum[KF_COUNT * KV_COUNT] = {0};
+    int64_t cnt[KF_COUNT * KV_COUNT] = {0};
+    static std::string variant_names[KF_COUNT * KV_COUNT];
+    static std::once_flag once;
+    std::call_once(once, [] {
+        for (int v = 0; v < KV_COUNT; ++v)
+            for (int f = 0; f < KF_COUNT; ++f) variant_names[f + KF_COUNT * v] = std::string(kFamilyNames[f]) + kVariantSuffix[v];
+    });
     for (size_t i = 0; i < dec->prof_family.size() && 2 * i + 1 < dec->prof_used + 1; ++i) {
         float t = 0.f;
         if (cudaEventElapsedTime(&t, dec->prof_events[2 * i], dec->prof_events[2 * i + 1]) != cudaSuccess) continue;
@@ -1635,9 +1690,9 @@ extern "C" int32_t aed_dec_profile_read(aed_dec_t *dec, int32_t max_families, co
         cnt[dec->prof_family[i]]++;
     }
     int n = 0;
-    for (int f = 0; f < KF_COUNT && n < max_families; ++f) {
+    for (int f = 0; f < KF_COUNT * KV_COUNT && n < max_families; ++f) {
         if (!cnt[f]) continue;
-        names[n] = kFamilyNames[f]; ms[n] = sum[f]; launches[n] = cnt[f];
+        names[n] = variant_names[f].c_str(); ms[n] = sum[f]; launches[n] = cnt[f];
         ++n;
     }
     return n;

@@ -51,8 +51,7 @@ struct CkvParams {
     int frame_capacity;
     int d_model, n_heads, d_enc;
     int n_layers;
-    void *store;                      // layer 0; layers are layer_elems elements apart; bf16, or E4M3 bytes if store_e4m3
-    int store_e4m3;
+    void *store;                      // layer 0; layers are layer_elems elements apart; bf16, or E4M3 bytes (template argument)
     size_t layer_elems;
     const __nv_bfloat16 *const *bias; // [n_layers] device pointers (entries may be null), or null
     DecState *state;
@@ -88,8 +87,9 @@ struct TileWalk {
 };
 
 // grid: persistent blocks.  map_w: one tensor map per layer over w_kv_c [2d, d_enc], boxes of 256 rows x 64.
+template <bool kE4M3>
 __global__ void __launch_bounds__(kCkvThreads, 1)
-crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorMap *__restrict__ map_w, CkvParams p)
+crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorMap *__restrict__ map_w, const __grid_constant__ CkvParams p)
 {
     extern __shared__ uint8_t smem_dyn[];
     __shared__ __align__(8) uint64_t bar_full[kStages];
@@ -211,7 +211,7 @@ crosskv_gemm_kernel(const __grid_constant__ CUtensorMap map_enc, const CUtensorM
                 }
                 const size_t elem = layer_off + ((static_cast<size_t>(kv) * p.n_heads + h) * p.frame_capacity + frame) * kHeadDim + e;
                 uint32_t packed[8];
-                if (p.store_e4m3) {
+                if (kE4M3) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
                         packed[j] = static_cast<uint32_t>(pack_e4m3x2(v[4 * j], v[4 * j + 1])) |

@@ -105,6 +105,58 @@ __device__ __forceinline__ void red_add_v4(float *addr, float4 v)
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
+// ---- side jobs of a projection launch, run by 64 threads (two warps) of every CTA, off the critical path -----------
+// st: 0..63 among those threads; cta / n_cta: this CTA among all CTAs of the launch.
+// Static data (a later kernel's weights) into L2: no need to wait for the previous kernel.  4 KB pieces.
+__device__ __forceinline__ void side_prefetch(const StepGemmParams &p, int cta, int n_cta, int st)
+{
+    for (int range = 0; range < 2; ++range) {
+        const char *base = static_cast<const char *>(range ? p.prefetch2_ptr : p.prefetch_ptr);
+        if (!base) continue;
+        const size_t pieces = (range ? p.prefetch2_bytes : p.prefetch_bytes) / 4096;
+        for (size_t i = static_cast<size_t>(cta) * 64 + st; i < pieces; i += static_cast<size_t>(n_cta) * 64)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + i * 4096), "r"(4096) : "memory");
+    }
+}
+// After the dependency wait: clear the rows a later split-K projection accumulates into, and (mean, rstd) of the rows
+// assigned to this CTA.  w: 0 or 1, which of the two warps; red_s, red_q: two floats of shared memory each.
+__device__ __forceinline__ void side_after_wait(const StepGemmParams &p, int cta, int n_cta, int st, int lane, int w,
+                                                float *red_s, float *red_q)
+{
+    const int n_rows = p.state->n_active;
+    if (p.zero_buf) {
+        const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
+        float4 *z = reinterpret_cast<float4 *>(p.zero_buf);
+        for (size_t idx = static_cast<size_t>(cta) * 64 + st; idx < total4; idx += static_cast<size_t>(n_cta) * 64)
+            z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (p.stats_src) {
+        for (int r = cta; r < n_rows; r += n_cta) {    // uniform over the two warps
+            const float *xr = p.stats_src + static_cast<size_t>(r) * p.stats_d;
+            float s = 0.f;
+            for (int idx = st * 4; idx < p.stats_d; idx += 256) {
+                const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+                s += (v.x + v.y) + (v.z + v.w);
+            }
+            s = warp_sum(s);
+            if (lane == 0) red_s[w] = s;
+            asm volatile("bar.sync 1, 64;" ::: "memory");
+            const float mean = (red_s[0] + red_s[1]) / p.stats_d;
+            float q = 0.f;
+            for (int idx = st * 4; idx < p.stats_d; idx += 256) {
+                const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
+                const float d0 = v.x - mean, d1 = v.y - mean, d2 = v.z - mean, d3 = v.w - mean;
+                q += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+            }
+            q = warp_sum(q);
+            if (lane == 0) red_q[w] = q;
+            asm volatile("bar.sync 1, 64;" ::: "memory");
+            if (st == 0) p.stats_out[r] = make_float2(mean, rsqrtf((red_q[0] + red_q[1]) / p.stats_d + p.eps));
+            asm volatile("bar.sync 1, 64;" ::: "memory");
+        }
+    }
+}
+
 // grid: x = 128-feature tiles, y = k-splits, z = row tiles.
 // Dynamic smem per k-block: weight tile 16 KB | high plane | low plane (n_tile x 128 B each) | fp32 source tile
 // (n_tile x 256 B, filled by TMA, later reused to transpose the accumulator); plus 1024 for alignment.
@@ -223,14 +275,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
         const int st = threadIdx.x - 320;                 // 0..63
         const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
         const int n_cta = gridDim.x * gridDim.y * gridDim.z;
-        for (int range = 0; range < 2; ++range) {
-            // static data: no need to wait for the previous kernel.  4 KB pieces, spread over all CTAs and threads.
-            const char *base = static_cast<const char *>(range ? p.prefetch2_ptr : p.prefetch_ptr);
-            if (!base) continue;
-            const size_t pieces = (range ? p.prefetch2_bytes : p.prefetch_bytes) / 4096;
-            for (size_t i = static_cast<size_t>(cta) * 64 + st; i < pieces; i += static_cast<size_t>(n_cta) * 64)
-                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + i * 4096), "r"(4096) : "memory");
-        }
+        side_prefetch(p, cta, n_cta, st);
         pdl_wait();
         if (MODE == B_PLANES) {
             // the activation planes of every k-block, by the first lane of these two warps (a thread's copies complete
@@ -249,38 +294,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
                 }
             }
         }
-        const int n_rows = p.state->n_active;
-        if (p.zero_buf) {
-            const size_t total4 = static_cast<size_t>(n_rows) * p.zero_cols / 4;
-            float4 *z = reinterpret_cast<float4 *>(p.zero_buf);
-            for (size_t idx = static_cast<size_t>(cta) * 64 + st; idx < total4; idx += static_cast<size_t>(n_cta) * 64)
-                z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (p.stats_src) {
-            for (int r = cta; r < n_rows; r += n_cta) {    // uniform over the two warps
-                const float *xr = p.stats_src + static_cast<size_t>(r) * p.stats_d;
-                float s = 0.f;
-                for (int idx = st * 4; idx < p.stats_d; idx += 256) {
-                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
-                    s += (v.x + v.y) + (v.z + v.w);
-                }
-                s = warp_sum(s);
-                if (lane == 0) red_s[warp - 10] = s;
-                asm volatile("bar.sync 1, 64;" ::: "memory");
-                const float mean = (red_s[0] + red_s[1]) / p.stats_d;
-                float q = 0.f;
-                for (int idx = st * 4; idx < p.stats_d; idx += 256) {
-                    const float4 v = *reinterpret_cast<const float4 *>(xr + idx);
-                    const float d0 = v.x - mean, d1 = v.y - mean, d2 = v.z - mean, d3 = v.w - mean;
-                    q += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
-                }
-                q = warp_sum(q);
-                if (lane == 0) red_q[warp - 10] = q;
-                asm volatile("bar.sync 1, 64;" ::: "memory");
-                if (st == 0) p.stats_out[r] = make_float2(mean, rsqrtf((red_q[0] + red_q[1]) / p.stats_d + p.eps));
-                asm volatile("bar.sync 1, 64;" ::: "memory");
-            }
-        }
+        side_after_wait(p, cta, n_cta, st, lane, warp - 10, red_s, red_q);
     } else {
         pdl_wait();
         AED_TRACE_PUT(p.state, tcur, 41);  // dependency resolved

@@ -193,7 +193,7 @@ struct aed_dec {
     bool use_pdl = true;
     bool attn_pipe = true;
     bool use_gemv = true;           // steps of few rows: projections by warp-level MMAs (step_gemv.cuh)
-    int gemv_rows = 32;             // ... up to this many rows
+    int gemv_rows = 64;             // ... up to this many rows
     int gemv_direct_rows = 4;       // ... with the activation fragments straight from global memory up to this many
     int planes_rows = 128;                // steps with more rows make their activation planes once per projection input
     // greedy decoding replays one captured CUDA graph per (row bucket, self-attention chunk count, output buffers)
@@ -542,6 +542,9 @@ aed_status_t tc_setup(aed_dec *dec)
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_PLAIN, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_GAMMA, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_LN_RELU, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_PLAIN, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4, 4));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_GAMMA, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4, 4));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sv::step_gemv_staged_kernel<sg::B_LN_RELU, 4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, sv::sv_staged_smem(4, 4));
 
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "tensor-core path set-up: %s", cudaGetErrorString(e));
     // LayerNorm-fold constants of every layer
@@ -574,7 +577,7 @@ aed_status_t tc_setup(aed_dec *dec)
         v = getenv("AED_DEC_NO_GEMV");
         dec->use_gemv = !(v && v[0] == '1');
         v = getenv("AED_DEC_GEMV_ROWS");
-        if (v && atoi(v) >= 1 && atoi(v) <= 32) dec->gemv_rows = atoi(v);
+        if (v && atoi(v) >= 1 && atoi(v) <= 64) dec->gemv_rows = atoi(v);
         v = getenv("AED_DEC_GEMV_DIRECT_ROWS");
         if (v && atoi(v) >= 0 && atoi(v) <= 8) dec->gemv_direct_rows = atoi(v);
         v = getenv("AED_DEC_PLANES_ROWS");
@@ -686,7 +689,12 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
     p.n_tile = n_tile;
     p.state = dec->state();
     p.eps = dec->cfg.ln_eps;
-    const bool gemv = MODE != sg::B_PLANES && dec->use_gemv && rows_ub <= dec->gemv_rows && kb_max <= sv::kSvMaxKb;
+    // (41 to 64 rows: two row halves on grid.z and half the k-splits, up to four k-blocks per CTA.  Measured per decode
+    // step of the 24-layer model against the tcgen05 kernel: 1036 / 1094 / 1129 / 1160 us against 1002 / 1103 / 1160 /
+    // 1200 at 33 / 48 / 56 / 64 rows, hence not between 33 and 40.)
+    const int splits_wide = std::max((k_blocks + 3) / 4, splits / 2);
+    const bool gemv = MODE != sg::B_PLANES && dec->use_gemv && rows_ub <= dec->gemv_rows && !(rows_ub > 32 && rows_ub <= 40) &&
+                      (rows_ub <= 32 ? kb_max <= sv::kSvMaxKb : (k_blocks + splits_wide - 1) / splits_wide <= 4);
     ProfScope ps(dec, family + KF_COUNT * (!gemv ? KV_TCGEN05 : rows_ub <= dec->gemv_direct_rows ? KV_GEMV : KV_GEMV_STAGED));
     if constexpr (MODE != sg::B_PLANES) {
         // Steps of at most 32 rows whose CTAs cover at most two k-blocks: warp-level MMAs (step_gemv.cuh), activation
@@ -695,9 +703,10 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
             cudaLaunchConfig_t gc = {};
             gc.gridDim = dim3(m_tiles, splits, 1);
             gc.blockDim = dim3(sv::kSvThreads);
-            const bool direct = rows_ub <= dec->gemv_direct_rows;
+            const bool direct = rows_ub <= dec->gemv_direct_rows, wide = rows_ub > 32;
             const int nt = rows_ub <= 16 ? 2 : 4;
-            gc.dynamicSmemBytes = direct ? (size_t)sv::kSvMaxKb * tc::kATileBytes + 1024 : (size_t)sv::sv_staged_smem(nt);
+            if (wide) gc.gridDim = dim3(m_tiles, splits_wide, 2);
+            gc.dynamicSmemBytes = direct ? (size_t)sv::kSvMaxKb * tc::kATileBytes + 1024 : (size_t)sv::sv_staged_smem(nt, wide ? 4 : sv::kSvMaxKb);
             gc.stream = dec->stream;
             cudaLaunchAttribute ga[1];
             ga[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -706,6 +715,7 @@ aed_status_t launch_step_gemm(aed_dec *dec, int family, const CUtensorMap &map_w
             gc.numAttrs = 1;
             const CUtensorMap &second = map_w2 ? *map_w2 : map_w;
             cudaError_t ge = direct    ? cudaLaunchKernelEx(&gc, sv::step_gemv_kernel<MODE, 1>, map_w, second, p)
+                             : wide    ? cudaLaunchKernelEx(&gc, sv::step_gemv_staged_kernel<MODE, 4, 4>, map_w, second, p)
                              : nt == 2 ? cudaLaunchKernelEx(&gc, sv::step_gemv_staged_kernel<MODE, 2>, map_w, second, p)
                                        : cudaLaunchKernelEx(&gc, sv::step_gemv_staged_kernel<MODE, 4>, map_w, second, p);
             if (ge != cudaSuccess) return fail(dec, AED_ERR_CUDA, "projection launch: %s", cudaGetErrorString(ge));

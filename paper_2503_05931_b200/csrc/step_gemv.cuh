@@ -1,4 +1,4 @@
-// Decode-step projections for steps of at most 32 rows.
+// Decode-step projections for steps of at most 64 rows.
 //
 //   out[r, o] += sum_k B(r, k) * W[o, k]      (+ bias[o] from the CTA of the first k-split)
 //
@@ -229,26 +229,29 @@ step_gemv_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 // the 8 warps fetch and split the same activation values; beyond a handful of rows that traffic costs more than one
 // hand-over through shared memory.  Here the 256 compute threads load the rows' k range once (coalesced 16-byte loads),
 // apply the transform, write bf16 high and low planes [row][k] into shared memory (row pitch padded against bank
-// conflicts), meet at one named barrier, and every warp reads its B fragments with ldmatrix.  (With 64 rows per CTA the
-// accumulators alone take 64 registers, one CTA fits per SM and the tcgen05 kernel is faster: 1350 against 1195 us per
-// step of the 24-layer model.)
-constexpr int kSvPitch = kSvMaxKb * kBlockK * 2 + 16;          // bytes per row of a plane: 128 k of bf16 + pad
+// conflicts), meet at one named barrier, and every warp reads its B fragments with ldmatrix.  A CTA covers at most 32
+// rows: with 64 the accumulators alone take 64 registers, one CTA fits per SM and the tcgen05 kernel is faster (1350
+// against 1195 us per step of the 24-layer model); launches of up to 64 rows put two row halves on grid.z.
+// kKB: most k-blocks per CTA (2, or 4 for the launches of 33 to 64 rows, which halve the k-splits and put two row
+// halves on grid.z instead: the same number of CTAs, half the reduction traffic).
+__host__ __device__ constexpr int sv_pitch(int kb) { return kb * kBlockK * 2 + 16; }          // bytes per row of a plane: the CTA's k range in bf16 + pad
+__host__ __device__ constexpr int sv_staged_smem(int nt, int kb = kSvMaxKb) { return kb * kATileBytes + 2 * nt * 8 * sv_pitch(kb) + 1024; }
 
-constexpr int sv_staged_smem(int nt) { return kSvMaxKb * kATileBytes + 2 * nt * 8 * kSvPitch + 1024; }
-
-template <int MODE, int kNT>
+// grid: x = 128-feature tiles, y = k-splits, z = row tiles of kNT * 8 rows.
+template <int MODE, int kNT, int kKB = kSvMaxKb>
 __global__ void __launch_bounds__(kSvThreads, 2)
 step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2, StepGemmParams p)
 {
     extern __shared__ uint8_t smem_dyn[];
-    __shared__ __align__(8) uint64_t bar_a[kSvMaxKb];
+    __shared__ __align__(8) uint64_t bar_a[kKB];
     __shared__ int abort_flag;
     __shared__ float red_s[2], red_q[2];
-    __shared__ __align__(16) float s_g[kSvMaxKb * kBlockK], s_c1[kSvMaxKb * kBlockK], s_c2[kSvMaxKb * kBlockK];
+    __shared__ __align__(16) float s_g[kKB * kBlockK], s_c1[kKB * kBlockK], s_c2[kKB * kBlockK];
     __shared__ __align__(16) float s_t[8][8][16 + 4];
 
     static_assert(kNT == 2 || kNT == 4, "row tiles are read in pairs");
-    constexpr int kRows = kNT * 8;
+    constexpr int kRows = kNT * 8, kSvPitch = sv_pitch(kKB), kF4 = kKB * kBlockK / 4;      // kF4: 16-byte loads per row
+    const int row0 = blockIdx.z * kRows;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool second_w = p.tiles_first > 0 && static_cast<int>(blockIdx.x) >= p.tiles_first;
     const CUtensorMap *mw = second_w ? &map_w2 : &map_w;
@@ -256,12 +259,12 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
     const int a_rows = second_w ? p.a_rows2 : p.a_rows;
     const int kb_begin = static_cast<int>((static_cast<long long>(p.k_blocks) * blockIdx.y) / gridDim.y);
     const int kb_end = static_cast<int>((static_cast<long long>(p.k_blocks) * (blockIdx.y + 1)) / gridDim.y);
-    const int n_kb = min(kb_end - kb_begin, kSvMaxKb);
+    const int n_kb = min(kb_end - kb_begin, kKB);
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint8_t *plane_hi = tiles + kSvMaxKb * kATileBytes, *plane_lo = plane_hi + kRows * kSvPitch;
+    uint8_t *plane_hi = tiles + kKB * kATileBytes, *plane_lo = plane_hi + kRows * kSvPitch;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSvMaxKb; ++s) mbar_init(&bar_a[s], 1);
+        for (int s = 0; s < kKB; ++s) mbar_init(&bar_a[s], 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -277,8 +280,8 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
             }
         }
         const int st = threadIdx.x - 256;
-        const int cta = blockIdx.x + gridDim.x * blockIdx.y;
-        const int n_cta = gridDim.x * gridDim.y;
+        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        const int n_cta = gridDim.x * gridDim.y * gridDim.z;
         sg::side_prefetch(p, cta, n_cta, st);
         sg::pdl_wait();
         sg::side_after_wait(p, cta, n_cta, st, lane, warp - 8, red_s, red_q);
@@ -307,13 +310,13 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
 
     sg::pdl_wait();
     const int n_rows = p.state->n_active;
-    // ---- the rows' k range -> planes: element e of the tile is row e / 32, floats 4 (e % 32) .. + 3 --------------------
-    constexpr int kPer = kRows * 32 / 256;                     // 16-byte loads per thread (1 for 8 rows, 2 for 16, 4 for 32)
+    // ---- the rows' k range -> planes: element e of the tile is row e / kF4, floats 4 (e % kF4) .. + 3 ------------------
+    constexpr int kPer = kRows * kF4 / 256;                    // 16-byte loads per thread
     float4 xv[kPer];
     float2 st[kPer];
 #pragma unroll
     for (int j = 0; j < kPer; ++j) {
-        const int e = threadIdx.x + 256 * j, r = e >> 5, c4 = e & 31;
+        const int e = threadIdx.x + 256 * j, rl = e / kF4, r = row0 + rl, c4 = e % kF4;
         const bool live = r < n_rows && c4 * 4 < n_kb * kBlockK;
         xv[j] = live ? *reinterpret_cast<const float4 *>(p.src + static_cast<size_t>(r) * p.ld_src + kb_begin * kBlockK + c4 * 4)
                      : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -321,7 +324,7 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
     }
 #pragma unroll
     for (int j = 0; j < kPer; ++j) {
-        const int e = threadIdx.x + 256 * j, r = e >> 5, c4 = e & 31;
+        const int e = threadIdx.x + 256 * j, rl = e / kF4, r = row0 + rl, c4 = e % kF4;
         float y[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
         if (MODE == B_GAMMA) {
             const float4 g = *reinterpret_cast<const float4 *>(&s_g[c4 * 4]);
@@ -335,8 +338,8 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
         uint32_t h0, l0, h1, l1;
         split2(y[0], y[1], h0, l0);
         split2(y[2], y[3], h1, l1);
-        *reinterpret_cast<uint2 *>(plane_hi + r * kSvPitch + c4 * 8) = make_uint2(h0, h1);
-        *reinterpret_cast<uint2 *>(plane_lo + r * kSvPitch + c4 * 8) = make_uint2(l0, l1);
+        *reinterpret_cast<uint2 *>(plane_hi + rl * kSvPitch + c4 * 8) = make_uint2(h0, h1);
+        *reinterpret_cast<uint2 *>(plane_lo + rl * kSvPitch + c4 * 8) = make_uint2(l0, l1);
     }
     asm volatile("bar.sync 2, 256;" ::: "memory");           // planes complete
 
@@ -350,7 +353,7 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
     const uint32_t b_off = static_cast<uint32_t>(((lane & 7) + ((lane >> 4) << 3)) * kSvPitch + ((lane >> 3) & 1) * 16);
     const uint32_t hi_base = smem_u32(plane_hi), lo_base = smem_u32(plane_lo);
 #pragma unroll
-    for (int i = 0; i < kSvMaxKb; ++i) {
+    for (int i = 0; i < kKB; ++i) {
         if (i >= n_kb || !ok) break;
         ok = mbar_wait(&bar_a[i], 0, &abort_flag);
         if (!ok) break;
@@ -394,7 +397,7 @@ step_gemv_staged_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_
         __syncwarp();
         const int rr = lane >> 2, f4 = (lane & 3) * 4;
         const float4 v = *reinterpret_cast<const float4 *>(&t[rr][f4]);
-        const int r = nt * 8 + rr, o = a0 + warp * 16 + f4;
+        const int r = row0 + nt * 8 + rr, o = a0 + warp * 16 + f4;
         if (r < n_rows) {
             float *dst = out + static_cast<size_t>(r) * ldo + o;
             if (o + 3 < a_rows) sg::red_add_v4(dst, v);

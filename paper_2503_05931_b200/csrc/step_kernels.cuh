@@ -433,6 +433,14 @@ template <typename CT> struct LaneWidth { static constexpr int kE = 8; };
 template <typename CT> constexpr int fused_chunk() { return 4 * (32 / (kHeadDim / LaneWidth<CT>::kE)); }
 constexpr int kFusedMaxWarps = 8;
 
+// 2^x by the hardware approximation (relative error about 2^-22): softmax weights of the single-pass attention kernel
+__device__ __forceinline__ float exp2_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int N> __device__ __forceinline__ void load_n(const float *p, float (&v)[N])
 {
 #pragma unroll
@@ -528,7 +536,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             load_n<kE>(ln_c1 + 2 * d_model + qcol, vc1); load_n<kE>(ln_c2 + 2 * d_model + qcol, vc2);
         }
     }
-    AED_TRACE_RESERVE(tcur, state, (threadIdx.x == 0 && blockIdx.x == 0) ? 4u : 0u);
+    AED_TRACE_RESERVE(tcur, state, (threadIdx.x == 0 && blockIdx.x == 0) ? 6u : 0u);
     AED_TRACE_PUT_NS(state, tcur, 8 + (kCross ? 1 : 0));      // resident, first chunk requested
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -571,7 +579,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         for (int i = 0; i < kE; ++i) qv[i] = fmaf(st.y, qv[i] - st.x * qc1[i], qc2[i]);
     }
 #pragma unroll
-    for (int i = 0; i < kE; ++i) qv[i] *= scale;
+    for (int i = 0; i < kE; ++i) qv[i] *= scale * 1.4426950408889634f;      // scores in units of ln 2: exponentials below are 2^x
     RawLane<CT> new_k, new_v;
     if (owns_new) {
         if (fold) {
@@ -589,6 +597,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         }
     }
 
+    AED_TRACE_PUT(state, tcur, 4);                          // query ready (statistics, fold)
     float m = -INFINITY, l = 0.f, acc[kE];
 #pragma unroll
     for (int i = 0; i < kE; ++i) acc[i] = 0.f;
@@ -638,13 +647,13 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
 #pragma unroll
         for (int o = kDG; o < 32; o <<= 1) cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));     // chunk max, uniform over the warp, finite
         const float m_new = fmaxf(m, cmax);
-        const float corr = expf(m - m_new);
+        const float corr = exp2_fast(m - m_new);
         l *= corr;
 #pragma unroll
         for (int j = 0; j < kE; ++j) acc[j] *= corr;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float pr = expf(s[i] - m_new);      // exp(-inf) = 0 for positions past the end
+            const float pr = exp2_fast(s[i] - m_new);      // 2^(-inf) = 0 for positions past the end
             float vf[kE];
             rv[i].get(vf);
             l += pr;
@@ -657,6 +666,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
             for (int i = 0; i < 4; ++i) { rk[i] = nk[i]; rv[i] = nv[i]; }
         }
     }
+    AED_TRACE_PUT(state, tcur, 5);                          // all chunks of this warp reduced
     // sum the position groups (they share m)
 #pragma unroll
     for (int o = kDG; o < 32; o <<= 1) {
@@ -675,7 +685,7 @@ attn_fused_kernel(const DecState *state, const int4 *__restrict__ row_info, cons
         for (int w = 0; w < n_warps; ++w) big = fmaxf(big, sm_m[w]);
         float lsum = 0.f, a = 0.f;
         for (int w = 0; w < n_warps; ++w) {
-            const float wgt = (sm_m[w] == -INFINITY) ? 0.f : expf(sm_m[w] - big);
+            const float wgt = (sm_m[w] == -INFINITY) ? 0.f : exp2_fast(sm_m[w] - big);
             lsum = fmaf(sm_l[w], wgt, lsum);
             a = fmaf(sm_acc[w][threadIdx.x], wgt, a);
         }

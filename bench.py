@@ -103,12 +103,12 @@ KERNEL_OF_FAMILY = {
 # dram__bytes_write.sum of the captured launches over their algorithmic bytes).  An entry is removed when its kernel
 # changes, which turns the reported traffic back into null.
 NCU_TRAFFIC_RATIO = {
-    # five launches of one layer at 64 rows: 68.44 MB read for 29.36 MB of layer weights; the launches also read the
-    # composite cross-query matrix (2.1 MB) and each prefetches the next layer's matrices of its kind into L2, which
-    # under the profiler's serialised replay is a second DRAM read
-    "step_gemm_kernel": 2.33,
-    # the same five launches at 16 and at 4 rows: 63.82 MB and 62.82 MB read
-    "step_gemv_staged_kernel": 2.17,
+    # five launches of one layer at 128 rows (cfg3): 73.68 MB read for 29.36 MB of layer weights; the launches also read
+    # the composite cross-query matrix (2.1 MB), the fp32 activation rows, and each prefetches the next layer's matrices
+    # of its kind into L2, which under the profiler's serialised replay is a second DRAM read
+    "step_gemm_kernel": 2.51,
+    # the five launches at 16 and at 4 rows (cfg2): 63.24 MB and 62.97 MB read
+    "step_gemv_staged_kernel": 2.15,
     "step_gemv_kernel": 2.14,
     # self + cross attention of one layer at 64 rows: 0.84 + 31.05 MB for 0.52 + 30.49 MB of K/V
     "attn_fused_kernel": 1.03,

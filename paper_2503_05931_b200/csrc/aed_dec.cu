@@ -616,10 +616,8 @@ aed_status_t launch_vocab_gemm(aed_dec *dec, int rows_ub, tc::TcParams p, int ro
     int stages = kTcSmemBudget / stage_bytes;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     if (stages > k_blocks) stages = k_blocks;
-    // every ring stage belongs to one issuing thread: stages is a multiple of the number of producers (prefer the
-    // deeper ring: 6 stages with 3 producers rather than 4 with 4)
+    // every ring stage belongs to one issuing thread: as many producers as stages (at most one per producer warp)
     int producers = stages >= tc::kProducerWarps ? tc::kProducerWarps : stages;
-    if (stages > tc::kProducerWarps && stages % tc::kProducerWarps && stages % (tc::kProducerWarps - 1) == 0) producers = tc::kProducerWarps - 1;
     stages -= stages % producers;
     const CUtensorMap *acts = dec->tc_actd[ni];
     dim3 grid(m_tiles, 1, row_tiles);
@@ -767,10 +765,18 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
             embed_rows_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), dec->at<int4>(L.row_info), dec->at<int32_t>(L.row_tok),
                                                                    (const T *)dec->embed, dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d,
                                                                    qc, d);
-        else
-            embed_kernel<T><<<rows_ub, 256, 0, dec->stream>>>(dec->state(), active_list, tokens, t_u, (const T *)dec->embed,
-                                                              dec->at<float>(L.pe), d, V, sqrtf((float)d), x, qkv, 3 * d, qc, d);
-        AED_LAUNCHED(dec);
+        else {
+            // starts while the row compaction still runs and waits for it inside (programmatic launch)
+            const DecState *state = dec->state();
+            const T *emb = (const T *)dec->embed;
+            const float *pe = dec->at<float>(L.pe);
+            int dd = d, vv = V, zc = 3 * d, zc2 = d;
+            float sc = sqrtf((float)d);
+            float *zb = qkv, *zb2 = qc;
+            void *args[] = {&state, &active_list, &tokens, &t_u, &emb, &pe, &dd, &vv, &sc, &x, &zb, &zc, &zb2, &zc2};
+            AED_TRY(launch_pdl_impl(dec, (const void *)embed_kernel<T>, dim3(rows_ub), dim3(256), 0, args));
+        }
+        if (pf) AED_LAUNCHED(dec);
     }
     const bool pdl = dec->use_pdl;
     for (int l = 0; l < c.n_layers; ++l) {
@@ -792,6 +798,8 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.stats_src = x; p.stats_out = stats; p.stats_d = d;
         p.prefetch_ptr = wn.w_qkv; p.prefetch_bytes = (size_t)3 * d * d * e2;
         p.prefetch2_ptr = wn.w_q_c; p.prefetch2_bytes = (size_t)d * d * e2;
+        // the vocabulary matrix is as large as a layer: its way into L2 starts a whole layer ahead of the projection
+        if (l == c.n_layers - 1) { p.prefetch2_ptr = dec->w_out; p.prefetch2_bytes = (size_t)V * d * e2; }
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_QKV, m.qkv, dec->tc_src_x, 3 * d, d, rows_ub, p, nullptr, &m.qc, d));
         // 2. self-attention (applies LN1 to q, k, v; appends k, v)
         if (pf) {
@@ -844,7 +852,6 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         p.out = hid; p.ldo = F;
         p.stats_src = x; p.stats_out = stats + 2 * stats_stride; p.stats_d = d;
         p.prefetch_ptr = wn.w_ff1; p.prefetch_bytes = (size_t)F * d * e2;
-        if (l == c.n_layers - 1) { p.prefetch2_ptr = dec->w_out; p.prefetch2_bytes = (size_t)V * d * e2; }    // the vocabulary projection is next
         AED_TRY(launch_step_gemm<sg::B_GAMMA>(dec, KF_GEMM_FF1, m.ff1, dec->tc_src_x, F, d, rows_ub, p));
         // 7. x += relu(LN3-corrected hidden) W2^T + b2 ; side: clear the cross-query rows
         p = sg::StepGemmParams{};

@@ -22,6 +22,7 @@ __global__ void build_active_kernel(const uint8_t *__restrict__ mask, const int3
                                     int4 *__restrict__ row_info, int row_slots, const int32_t *__restrict__ order)
 {
     AED_TRACE_BEGIN(state, 1);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the next kernel may become resident; it waits for this one inside
     __shared__ int warp_counts[32];
     __shared__ int base;
     const int batch = state->batch;
@@ -79,6 +80,9 @@ __global__ void embed_kernel(const DecState *state, const int32_t *__restrict__ 
                              float *__restrict__ zero_buf2 = nullptr, int zero_cols2 = 0)
 {
     AED_TRACE_BEGIN(state, 2);
+    // may be launched with programmatic stream serialization, right behind the row compaction
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int r = blockIdx.x;
     if (r >= state->n_active) return;
     int u = active_list[r];

@@ -30,8 +30,8 @@ constexpr int kBlockK = 64;                    // bf16 elements per k-block = on
 constexpr int kTileM = 128;
 constexpr int kATileBytes = kTileM * kBlockK * 2;
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 288;                    // 4 producer warps, 1 MMA warp, 4 epilogue warps
-constexpr int kProducerWarps = 4;
+constexpr int kThreads = 416;                    // 8 producer warps, 1 MMA warp, 4 epilogue warps
+constexpr int kProducerWarps = 8;                // (a k-block is three copies, and a thread's copies complete one after the other)
 constexpr long long kWaitCycles = 2000000000ll;   // about a second at B200 clocks
 constexpr int kErrTimeout = 2;
 

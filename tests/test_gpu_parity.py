@@ -382,3 +382,21 @@ def test_small_batch_model_shapes(model):
     w = wl.make_custom(m, rng.integers(1, 200, size=batch), rng.integers(1, 20, size=batch), dtype="bf16", seed=77,
                        out_std=0.1, ln_std=0.2, out_bias_std=0.1)
     _run_both(w, rows=[0, 5, batch // 2, batch - 1])
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes_and_row_counts_bf16(seed):
+    """Model widths, k-block counts, row counts and lengths drawn at random: every projection form (warp-level with
+    fragments from global memory, with shared-memory planes at one or two row halves, tcgen05, ready-made planes) meets
+    k ranges of one, two and four k-blocks, partial feature tiles and partly filled row tiles."""
+    rng = np.random.default_rng(1000 + seed)
+    heads = int(rng.integers(1, 6))
+    d = 64 * heads
+    model = dict(n_layers=int(rng.integers(1, 4)), d_model=d, n_heads=heads, d_ffn=64 * int(rng.integers(1, 13)),
+                 vocab=int(rng.integers(130, 700)), d_enc=64 * int(rng.integers(1, 5)))
+    batch = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 15, 16, 17, 31, 32, 33, 40, 41, 48, 63, 64, 65, 90, 128, 129, 140]))
+    enc_lens = rng.integers(1, 160, size=batch)
+    dec_lens = rng.integers(1, 7, size=batch)
+    w = wl.make_custom(model, enc_lens, dec_lens, dtype="bf16", seed=2000 + seed, out_std=0.1, ln_std=0.2, bias_std=0.05)
+    rows = sorted({0, batch - 1, batch // 2, int(np.argmax(dec_lens)), int(np.argmax(enc_lens))})
+    _run_both(w, rows=rows, need_tokens=False, label=f"random shape {model} B={batch}")

@@ -518,6 +518,8 @@ def profile_dominant_kernel(dec, w, one_pass, peaks, ms_per_step):
     for fam, v in prof.items():
         base, _, variant = fam.partition("@")                  # "gemm_qkv@gemv_staged": call site and the kernel that ran it
         kernel = {"gemv": "step_gemv_kernel", "gemv_staged": "step_gemv_staged_kernel"}.get(variant, KERNEL_OF_FAMILY.get(base, base))
+        if base == "gemm_vocab" and variant:
+            kernel = "vocab_gemv_kernel"                       # final LayerNorm + vocabulary projection of steps with few rows
         k = kernels.setdefault(kernel, {"ms": 0.0, "launches": 0, "bytes": 0.0, "families": []})
         k["ms"] += v["ms"]; k["launches"] += v["launches"]; k["families"].append(fam)
         if base in site_weights:

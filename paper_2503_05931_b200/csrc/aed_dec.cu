@@ -18,6 +18,7 @@
 #include "tc_gemm.cuh"
 #include "step_gemm.cuh"
 #include "step_gemv.cuh"
+#include "vocab_gemv.cuh"
 #include "crosskv_gemm.cuh"
 #include "stream_schedule.h"
 
@@ -65,6 +66,7 @@ struct Layout {
     size_t actd_hi, actd_lo, actf_hi, actf_lo;
     size_t fold_c, ln_stats, qc;          // LayerNorm-fold constants per layer, row statistics (3 sets)
     size_t slot_tokens, slot_lens;        // aed_dec_decode_stream: token rows and lengths of the slots
+    size_t fold_out;                      // c1 | c2 of the vocabulary projection with the final LayerNorm folded in
     size_t comp_w, comp_b;                // per layer: Wqc diag(gamma2) Wo as bf16 [d, d], and Wqc (gamma2 * bo) as fp32 [d]
     size_t ckv_maps, ckv_bias;            // per-layer tensor maps and bias pointers of the cross-K/V weights
     size_t fold_layer_floats;
@@ -145,6 +147,7 @@ Layout make_layout(const aed_dec_config_t &c)
         L.qc = take(B * d * 4);
         L.ckv_maps = take((size_t)c.n_layers * sizeof(CUtensorMap));
         L.ckv_bias = take((size_t)c.n_layers * sizeof(void *));
+        L.fold_out = take((size_t)2 * c.vocab * 4);
         L.comp_w = take((size_t)c.n_layers * d * d * 2);
         L.comp_b = take((size_t)c.n_layers * d * 4);
     }
@@ -567,7 +570,16 @@ aed_status_t tc_setup(aed_dec *dec)
         sg::compose_bias_kernel<<<(d + 7) / 8, 256, 0, dec->stream>>>((const T *)w.w_q_c, (const T *)w.ln2_g, (const T *)w.b_o, (int)d, cb);
         dec->launches += 5;
     }
+    {
+        typedef __nv_bfloat16 T;
+        float *fo = dec->at<float>(L.fold_out);
+        sg::ln_fold_constants_kernel<<<(c.vocab + 7) / 8, 256, 0, dec->stream>>>((const T *)dec->w_out, (const T *)dec->final_ln_g, (const T *)dec->final_ln_b,
+                                                                                (const T *)dec->b_out, c.vocab, (int)d, fo, fo + c.vocab);
+        dec->launches += 1;
+    }
     e = cudaGetLastError();
+    if (e == cudaSuccess && vg::vg_smem((int)d) <= 227 * 1024)
+        e = cudaFuncSetAttribute(vg::vocab_gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, vg::vg_smem((int)d));
     if (e != cudaSuccess) return fail(nullptr, AED_ERR_CUDA, "fold constants: %s", cudaGetErrorString(e));
     {
         const char *v = getenv("AED_DEC_NO_PDL");
@@ -862,6 +874,22 @@ aed_status_t forward_step_fused(aed_dec *dec, int rows_ub, int self_len_ub, cons
         AED_TRY(launch_step_gemm<sg::B_LN_RELU>(dec, KF_GEMM_FF2, m.ff2, dec->tc_src_hid, d, F, rows_ub, p));
     }
     if (pf && !pf->last_chunk) return AED_OK;
+    if (!pf && dec->use_gemv && rows_ub <= vg::kVgRows && d % 128 == 0 && vg::vg_smem(d) <= 227 * 1024) {
+        // at most 16 rows: final LayerNorm, vocabulary projection and argmax keys in one kernel (vocab_gemv.cuh)
+        ProfScope ps(dec, KF_GEMM_VOCAB + KF_COUNT * KV_GEMV);
+        vg::VocabGemvParams vp{};
+        vp.vocab = V; vp.d_model = d;
+        vp.x = x; vp.gamma = (const T *)dec->final_ln_g;
+        vp.c1 = dec->at<float>(L.fold_out); vp.c2 = vp.c1 + V;
+        vp.eps = c.ln_eps;
+        vp.logits_out = logits_out;
+        vp.keys = dec->at<unsigned long long>(L.keys);
+        vp.active_list = active_list;
+        vp.state = dec->state();
+        void *args[] = {(void *)&dec->tc_w_out, &vp};
+        return launch_pdl_impl(dec, (const void *)vg::vocab_gemv_kernel, dim3((V + tc::kTileM - 1) / tc::kTileM), dim3(vg::kVgThreads),
+                               (size_t)vg::vg_smem(d), args);
+    }
     AED_TRY(launch_ln_planes(dec, rows_ub, x, dec->final_ln_g, dec->final_ln_b, nullptr, 0));
     tc::TcParams tp{};
     tp.bias = (const T *)dec->b_out;

@@ -112,8 +112,9 @@ NCU_TRAFFIC_RATIO = {
     "step_gemv_kernel": 2.14,
     # self + cross attention of one layer at 64 rows: 0.84 + 31.05 MB for 0.52 + 30.49 MB of K/V
     "attn_fused_kernel": 1.03,
-    # vocabulary projection: 33.85 MB for the 33.55 MB output matrix
+    # vocabulary projection: 33.85 MB for the 33.55 MB output matrix (tcgen05 kernel; 33.79 MB in the few-row kernel)
     "tc_gemm_kernel": 1.01,
+    "vocab_gemv_kernel": 1.01,
     # cross-K/V of 7444 frames: 117.2 MB read + 677.2 MB written for 847.7 MB (part of the output is still in L2 at exit)
     "crosskv_gemm_kernel": 0.94,
 }

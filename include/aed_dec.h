@@ -115,7 +115,11 @@ size_t aed_dec_workspace_bytes(const aed_dec_config_t *config);
  * "rtfx" variants are free parameters).  Validates the configuration, carves the caller's workspace into
  * self-attention K/V caches, the cross-attention K/V store, activation buffers and decode state, and fills
  * the positional table.  Supported shapes: head_dim = d_model / n_heads == 64; d_model, d_ffn, d_enc
- * multiples of 64; vocab >= 2.  Otherwise AED_ERR_UNSUPPORTED.  On success *out receives the handle.
+ * multiples of 64; vocab >= 2; cross_kv_format = AED_CROSS_KV_E4M3 only with dtype = AED_DTYPE_BF16.  Otherwise
+ * AED_ERR_UNSUPPORTED.  In the bf16 configuration the call also builds, in the workspace and on the caller's stream,
+ * the LayerNorm-fold constants of the folded projections and, per layer, the composite of the self-attention output
+ * projection and the cross-attention query projection (a d x d matrix product per layer: creation takes milliseconds,
+ * not microseconds).  On success *out receives the handle.
  */
 aed_status_t aed_dec_create(const aed_dec_config_t *config, const aed_dec_weights_t *weights, aed_dec_t **out);
 
